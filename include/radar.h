@@ -1,0 +1,230 @@
+/*
+ * radar.h - C ABI of the B200 (sm_100a) hot path of one RADAR speculative step.
+ *
+ * The four calls are the data-parallel stages of one speculative step as the paper
+ * states it (Sec. 4.1 "Inference Pipeline" and the appendix walkthrough): draft-tree
+ * expansion with the continue/stop prediction model, rerank + serialisation of the tree,
+ * tree-masked verification attention, and acceptance.
+ *
+ * Conventions for every call
+ *   - Returns an int status (0 = RADAR_OK, negative = error).  Host-detectable errors
+ *     (NULL pointers, unsupported sizes, workspace too small) are returned at once and
+ *     nothing is launched.  Errors only the device can see (NaN logits, a pool that is not
+ *     ancestor-closed, a wait that ran out) are recorded in a sticky device status word
+ *     that radar_read_device_status() returns; kernels never trap.
+ *   - Every pointer in an argument struct is a DEVICE pointer owned by the caller unless
+ *     its comment says "host".  The library keeps no reference after the call returns.
+ *   - Calls are asynchronous on the given CUDA stream (passed as void*, 0 = default stream),
+ *     perform no host synchronisation and allocate nothing; scratch memory is the caller's
+ *     `workspace` (size from the matching *_workspace_bytes function, 256-byte aligned).
+ *   - Outputs are fully overwritten for every processed sequence; padding entries are
+ *     written as documented.  Inputs are never modified except the documented in/out state.
+ *   - Tree rows: row 0 is the root (the last committed token), rows 1..n_nodes-1 the kept
+ *     draft nodes; at most RADAR_MAX_NODES rows so that an ancestor set is one 64-bit word.
+ */
+#ifndef RADAR_H
+#define RADAR_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define RADAR_MAX_NODES 64      /* tree rows incl. root */
+#define RADAR_GATE_HIDDEN 128   /* LSTM / MLP hidden size of the prediction model (App. "Implementation Details") */
+#define RADAR_MAX_K 32          /* branching factor limit */
+#define RADAR_MAX_POOL 8192     /* pool capacity limit for radar_rerank_build_tree */
+
+enum {
+    RADAR_OK = 0,
+    RADAR_ERR_INVALID_ARG = -1,
+    RADAR_ERR_UNSUPPORTED = -2,
+    RADAR_ERR_WORKSPACE = -3,
+    RADAR_ERR_CUDA = -4,
+    RADAR_ERR_TIMEOUT = -5,
+    RADAR_ERR_NUMERIC = -6,
+    RADAR_ERR_TREE = -7
+};
+
+enum { RADAR_F32 = 0, RADAR_BF16 = 1 };
+enum { RADAR_GREEDY = 0, RADAR_STOCHASTIC = 1 };
+
+typedef struct radar_ctx radar_ctx;
+
+/* Context: remembers the device, its SM count and owns the 4-byte device status word
+ * (the only allocation the library ever makes).  `out` is a host pointer. */
+int radar_create(radar_ctx** out, int device);
+int radar_destroy(radar_ctx* ctx);
+const char* radar_status_string(int status);
+/* Synchronises `stream`, returns the sticky device status (RADAR_OK or the first device-side
+ * error recorded since the last read) and clears it. */
+int radar_read_device_status(radar_ctx* ctx, void* stream);
+
+/* ------------------------------------------------------------------------------------------
+ * radar_expand_step - one draft call's worth of tree expansion for every active sequence.
+ * (Appendix walkthrough: each frontier token yields its k most probable tokens with their
+ * confidence scores; the k best candidates over all parents are kept; the prediction model
+ * of Sec. 4.2 then emits continue/stop.  State s_t of the MDP = those k confidence scores.)
+ *
+ * For sequence b with active[b] != 0, and each of its F frontier rows f:
+ *   log-softmax over the V logits, top-k by (logit desc, token id asc);
+ *   candidate score = parent_score[b,f] + log-prob; all F*k candidates are appended to the
+ *   pool in (f, j) order at pool_len[b]; the k best by (score desc, flat index asc) become the
+ *   frontier outputs.  If t < t_max the prediction model runs on x = exp(frontier_score):
+ *   single-layer LSTM (gate blocks i,f,g,o; state h,c) then Linear(H+k,H)-ReLU-Linear(H,2) on
+ *   [h';x]; cont = logit[1] > logit[0].  At t == t_max the model is skipped, cont = 0 and
+ *   gate_logits = 0.  If force_calls is given, cont = (t < force_calls[b]) instead.
+ *   active[b] <- cont[b].  Sequences with active[b] == 0 are skipped: nothing of theirs is
+ *   touched, except cont[b] <- 0.
+ * A NaN logit records RADAR_ERR_NUMERIC (outputs of that sequence unspecified).
+ * Limits: 1 <= k <= RADAR_MAX_K, 1 <= F <= 32, V >= k, pool_len[b] + F*k <= pool_capacity.
+ */
+typedef struct {
+    int B, F, V, k;
+    int t, t_max;                       /* 1-based index of this draft call, and the maximum */
+    const void* logits;                 /* [B][F][V] draft logits; element type logits_dtype */
+    int logits_dtype;                   /* RADAR_F32 or RADAR_BF16 */
+    int64_t logits_row_stride;          /* elements between consecutive rows f   (>= V)      */
+    int64_t logits_seq_stride;          /* elements between consecutive sequences b          */
+    const float* parent_score;          /* [B][F] cumulative log-prob of each frontier row   */
+    const int32_t* parent_pool_idx;     /* [B][F] pool index of each frontier row, -1 = root */
+    uint8_t* active;                    /* [B] in/out                                        */
+    const int32_t* force_calls;         /* [B] or NULL                                       */
+    const float *w_ih, *w_hh, *b_ih, *b_hh;   /* LSTM: [4H][k], [4H][H], [4H], [4H]          */
+    const float *w1, *b1, *w2, *b2;           /* MLP : [H][H+k], [H], [2][H], [2]            */
+    float* h;                           /* [B][H] in/out, caller zeroes before t = 1         */
+    float* c;                           /* [B][H] in/out                                     */
+    int pool_capacity;                  /* C                                                 */
+    int32_t *pool_tok, *pool_parent, *pool_depth, *pool_draft_row;   /* [B][C] in/out        */
+    float* pool_score;                  /* [B][C] in/out                                     */
+    int32_t* pool_len;                  /* [B] in/out                                        */
+    int32_t* frontier_tok;              /* [B][k] out */
+    float* frontier_score;              /* [B][k] out (also the next call's parent_score)    */
+    int32_t* frontier_pool_idx;         /* [B][k] out (also the next call's parent_pool_idx) */
+    int32_t* frontier_src_row;          /* [B][k] out: which row f produced the survivor     */
+    int32_t* topk_tok;                  /* [B][F][k] out */
+    float* topk_logp;                   /* [B][F][k] out */
+    float* gate_logits;                 /* [B][2] out */
+    uint8_t* cont;                      /* [B] out */
+    void* workspace;
+    size_t workspace_bytes;
+} radar_expand_args;
+
+size_t radar_expand_workspace_bytes(const radar_ctx* ctx, int B, int F, int V, int k);
+int radar_expand_step(radar_ctx* ctx, const radar_expand_args* args, void* stream);
+
+/* ------------------------------------------------------------------------------------------
+ * radar_rerank_build_tree - top-N rerank of the pool and serialisation for one masked pass.
+ * (Sec. 1: the candidates form a tree that is serialised and verified via masked attention
+ * in a single pass; Sec. 2.3: nodes are reordered and pruned by confidence.)
+ *
+ * Keeps the n = min(N_b, pool_len[b], 63) best pool entries by (score desc, pool index asc),
+ * N_b = n_keep[b] if given else N; lays them out after the root in ascending pool index;
+ * writes per tree row: token, parent row, depth, position id = prefix_len[b] + depth, pool
+ * index, score, draft row (row of the draft logits that produced the node's children, -1 if
+ * it has none), ancestor mask (bit j of mask[i] <=> row j is i or an ancestor of i).
+ * Rows >= n_nodes[b]: tok/parent/pool_idx/draft_row = -1, depth/pos = 0, score = 0, mask = 0.
+ * retrieve[b][l][0..depth] = rows from the root to the l-th leaf (leaves in ascending row
+ * order), -1 padded; rows l >= n_leaves[b] are all -1.
+ * A kept entry whose parent was not kept records RADAR_ERR_TREE.
+ * Limits: pool_capacity <= RADAR_MAX_POOL, 1 <= N < RADAR_MAX_NODES, t_max < 64.
+ */
+typedef struct {
+    int B, N, t_max, pool_capacity;
+    const int32_t *pool_tok, *pool_parent, *pool_depth, *pool_draft_row;   /* [B][C] */
+    const float* pool_score;            /* [B][C] */
+    const int32_t* pool_len;            /* [B] */
+    const int32_t* n_keep;              /* [B] or NULL */
+    const int32_t* root_tok;            /* [B] */
+    const int32_t* prefix_len;          /* [B] */
+    int32_t *tree_tok, *tree_parent, *tree_depth, *tree_pos, *tree_pool_idx, *tree_draft_row;  /* [B][64] out */
+    float* tree_score;                  /* [B][64] out */
+    uint64_t* tree_mask;                /* [B][64] out */
+    int32_t* n_nodes;                   /* [B] out */
+    int32_t* retrieve;                  /* [B][N][t_max+1] out */
+    int32_t* n_leaves;                  /* [B] out */
+} radar_tree_args;
+
+int radar_rerank_build_tree(radar_ctx* ctx, const radar_tree_args* args, void* stream);
+
+/* ------------------------------------------------------------------------------------------
+ * radar_tree_attention - tree-masked verification attention of one layer, GQA.
+ * (Sec. 3: the target model scores the whole draft in one parallel pass; Sec. 1: the
+ * serialised tree is verified via masked attention.)
+ *
+ * For sequence b, query head h (KV head h / (Hq/Hkv)) and tree row i < n_nodes[b]:
+ *   O[b,i,h,:] = sum_j softmax_j(scale * q.k_j) v_j over j in prefix[0, prefix_len[b]) and
+ *   tree rows t with bit t of mask[b,i] set.  Rows i >= n_nodes[b] of O are left untouched.
+ * Layouts: Q, O [B][64][Hq][d]; Kt, Vt [B][64][Hkv][d]; prefix cache Kc, Vc token-major
+ * [token][Hkv][d] where sequence b's tokens start at row kv_start[b] (dense caches:
+ * kv_start[b] = b * Pmax; packed: the cumulative lengths).  dtype applies to Q, K, V and O;
+ * accumulation is fp32.  lse (optional) [B][Hq][64] receives log sum_j exp(scale * q.k_j).
+ * max_prefix_len (host) bounds prefix_len[] and sizes the launch; a larger device value
+ * records RADAR_ERR_INVALID_ARG on the device status word and that sequence is skipped.
+ * Limits: d in {64, 128}; Hq a multiple of Hkv.
+ */
+typedef struct {
+    int B, Hq, Hkv, d;
+    int dtype;                          /* RADAR_F32 or RADAR_BF16 */
+    const void* Q;
+    const void *Kc, *Vc;
+    const int64_t* kv_start;            /* [B] */
+    const int32_t* prefix_len;          /* [B] */
+    int max_prefix_len;                 /* host value */
+    const void *Kt, *Vt;
+    const uint64_t* mask;               /* [B][64] */
+    const int32_t* n_nodes;             /* [B] */
+    float scale;                        /* <= 0 selects 1/sqrt(d) */
+    void* O;
+    float* lse;                         /* or NULL */
+    void* workspace;
+    size_t workspace_bytes;
+} radar_attn_args;
+
+size_t radar_attn_workspace_bytes(const radar_ctx* ctx, int B, int Hq, int Hkv, int d, int dtype, int max_prefix_len);
+int radar_tree_attention(radar_ctx* ctx, const radar_attn_args* args, void* stream);
+
+/* ------------------------------------------------------------------------------------------
+ * radar_verify_accept - acceptance of the verified tree.
+ * Greedy (temperature-0 rows of the paper's temperature study): a_i = argmax of the target
+ *   logits at row i (lowest token id on ties); from the root move to the child whose token is
+ *   a_cur, else stop; next_token = a at the last accepted row.
+ * Stochastic (Sec. 3, Eq. 1-2, applied sibling by sibling as Sec. 4.3, Eq. 13 assumes):
+ *   p = softmax(target[cur]/T), q = softmax(draft[tree_draft_row[cur]]/T); children in
+ *   ascending row order; child x accepted iff u_accept[row] < min(1, p(x)/q(x)) (q(x) = 0:
+ *   accepted iff p(x) > 0); on reject p <- norm(max(0, p - q)), q(x) <- 0, q <- q / sum q;
+ *   when every child is rejected next_token is drawn from the current p, when the path
+ *   reaches a row without children it is drawn from softmax(target[row]/T); draws use the
+ *   inverse CDF in token order with u_sample[b].  Probabilities are evaluated in fp64.
+ * Outputs: accept_len[b] = accepted draft rows (root excluded); path_nodes/path_tokens
+ * [B][t_max+1] (entry 0 = root, -1 padded); next_token[b]; best_retrieve_row[b] = lowest
+ * retrieve row that contains the accepted path (-1 if the tree has no leaves).
+ * target_logits [B][64][V] (rows >= n_nodes[b] are not read); draft_logits [B][R][V].
+ */
+typedef struct {
+    int B, V, t_max, N, mode;
+    float temperature;                  /* stochastic only, > 0 */
+    const void* target_logits;
+    int logits_dtype;                   /* RADAR_F32 or RADAR_BF16 (both logits tensors) */
+    const int32_t *tree_tok, *tree_parent, *tree_draft_row;   /* [B][64] */
+    const int32_t* n_nodes;             /* [B] */
+    const int32_t* retrieve;            /* [B][N][t_max+1] */
+    const int32_t* n_leaves;            /* [B] */
+    const void* draft_logits;           /* stochastic: [B][R][V] */
+    int R;
+    const float* u_accept;              /* stochastic: [B][64] */
+    const float* u_sample;              /* stochastic: [B] */
+    int32_t *accept_len, *path_nodes, *path_tokens, *next_token, *best_retrieve_row;
+    void* workspace;
+    size_t workspace_bytes;
+} radar_accept_args;
+
+size_t radar_accept_workspace_bytes(const radar_ctx* ctx, int B, int V, int mode);
+int radar_verify_accept(radar_ctx* ctx, const radar_accept_args* args, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* RADAR_H */

@@ -1,0 +1,109 @@
+// Shared device/host helpers of the RADAR hot-path library (sm_100a).
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <math_constants.h>
+#include <stdint.h>
+
+#include "../../include/radar.h"
+
+struct radar_ctx {
+    int device;
+    int sm_count;
+    int* d_status;          // sticky device status word
+};
+
+#define RADAR_CUDA_CHECK(expr)                         \
+    do {                                               \
+        cudaError_t _e = (expr);                       \
+        if (_e != cudaSuccess) return RADAR_ERR_CUDA;  \
+    } while (0)
+
+namespace radar {
+
+constexpr int kMaxNodes = RADAR_MAX_NODES;
+constexpr int kHidden = RADAR_GATE_HIDDEN;
+constexpr unsigned kFull = 0xffffffffu;
+
+// first error wins
+__device__ __forceinline__ void set_status(int* status, int code) { atomicCAS(status, 0, code); }
+
+__device__ __forceinline__ float to_float(float x) { return x; }
+__device__ __forceinline__ float to_float(__nv_bfloat16 x) { return __bfloat162float(x); }
+
+// (value desc, index asc) ordering: true if a precedes b
+__device__ __forceinline__ bool precedes(float va, int ia, float vb, int ib) {
+    return va > vb || (va == vb && ia < ib);
+}
+__device__ __forceinline__ bool precedes(double va, int ia, double vb, int ib) {
+    return va > vb || (va == vb && ia < ib);
+}
+
+template <typename T>
+__device__ __forceinline__ T warp_max(T v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = max(v, __shfl_xor_sync(kFull, v, o));
+    return v;
+}
+template <typename T>
+__device__ __forceinline__ T warp_sum(T v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(kFull, v, o);
+    return v;
+}
+
+// Sorted list of the 32 best (value, index) pairs seen by a warp, one per lane (lane 0 = best).
+// V is float or double.  Empty slots hold (-inf, INT_MAX).
+template <typename V>
+struct WarpTopList {
+    V v;
+    int i;
+    __device__ __forceinline__ void reset() {
+        v = -CUDART_INF_F;
+        i = 0x7fffffff;
+    }
+    // all lanes call with the same candidate
+    __device__ __forceinline__ void insert(V cv, int ci) {
+        const bool worse = precedes(cv, ci, v, i);               // this lane's entry comes after the candidate
+        const unsigned w = __ballot_sync(kFull, worse);
+        if (w == 0) return;
+        const int pos = __ffs(w) - 1;                             // entries are sorted: worse lanes are a suffix
+        const V uv = __shfl_up_sync(kFull, v, 1);
+        const int ui = __shfl_up_sync(kFull, i, 1);
+        const int lane = threadIdx.x & 31;
+        if (lane == pos) { v = cv; i = ci; }
+        else if (lane > pos) { v = uv; i = ui; }
+    }
+    __device__ __forceinline__ V value_at(int lane) const { return __shfl_sync(kFull, v, lane); }
+    __device__ __forceinline__ int index_at(int lane) const { return __shfl_sync(kFull, i, lane); }
+};
+
+// --- vocabulary pass (vocab_pass.cu) ------------------------------------------------------
+// One launch reduces every (row, chunk) of a [rows][V] logits matrix to a partial record:
+//   topv/topi [k] best (logit, token) of the chunk, sorted; m = max logit; s = sum exp(logit - m).
+// rows are addressed as base + seq * seq_stride + f * row_stride with row = seq * F + f; rows whose
+// sequence has skip[seq] == 0 (if skip != NULL) or whose index within the sequence is >= nrows[seq]
+// (if nrows != NULL) are not read.
+struct VocabPassParams {
+    const void* logits;
+    int dtype;
+    int64_t row_stride, seq_stride;
+    int n_seq, F, V, k;
+    int n_chunks, chunk;             // chunk = elements per chunk (multiple of 8)
+    int want_lse;                    // 0: top-k only (argmax pass), 1: also (m, s)
+    const uint8_t* seq_active;       // or NULL
+    const int32_t* seq_rows;         // or NULL: rows to process per sequence
+    float* part_v;                   // [rows][n_chunks][k]
+    int32_t* part_i;                 // [rows][n_chunks][k]
+    float* part_m;                   // [rows][n_chunks]
+    float* part_s;                   // [rows][n_chunks]
+    int* status;
+};
+int vocab_pass_plan_chunks(int sm_count, int rows, int V, int* chunk_out);   // returns n_chunks
+size_t vocab_pass_partial_bytes(int rows, int n_chunks, int k);
+void vocab_pass_carve(void* ws, int rows, int n_chunks, int k, VocabPassParams* p);
+cudaError_t vocab_pass_launch(const VocabPassParams& p, cudaStream_t stream);
+
+static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+}  // namespace radar

@@ -1,0 +1,241 @@
+// radar_expand_step: vocabulary pass (vocab_pass.cu) followed by one block per sequence that
+// merges the chunk partials into each row's top-k and log-normaliser, forms the candidate
+// scores, appends them to the pool, selects the k best over all parents and runs the
+// prediction model (LSTM cell + MLP head) on their confidence scores.
+#include "common.cuh"
+
+namespace radar {
+namespace {
+
+constexpr int kSelThreads = 512;
+constexpr int kSelWarps = kSelThreads / 32;
+constexpr int kMaxF = 32;
+
+struct SelectParams {
+    radar_expand_args a;
+    VocabPassParams vp;
+    int* status;
+};
+
+__device__ __forceinline__ float sigmoidf_(float x) { return 1.f / (1.f + expf(-x)); }
+
+// y[r] = bias[r] + sum_c W[r][c] * x[c], rows distributed over warps, columns over lanes
+__device__ __forceinline__ float row_dot(const float* __restrict__ w_row, const float* x, int n, int lane) {
+    float acc = 0.f;
+    for (int c = lane; c < n; c += 32) acc = fmaf(w_row[c], x[c], acc);
+    return warp_sum(acc);
+}
+
+__global__ void __launch_bounds__(kSelThreads) expand_select_gate_kernel(const SelectParams P) {
+    const radar_expand_args& a = P.a;
+    const int b = blockIdx.x;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    if (a.active[b] == 0) {
+        if (tid == 0) a.cont[b] = 0;
+        return;
+    }
+    const int F = a.F, k = a.k, H = kHidden;
+    const int n_chunks = P.vp.n_chunks;
+
+    __shared__ double s_cand[kMaxF * RADAR_MAX_K];     // candidate scores, flat (f, j)
+    __shared__ int s_ctok[kMaxF * RADAR_MAX_K];
+    __shared__ int s_sel[RADAR_MAX_K];
+    __shared__ float s_x[RADAR_MAX_K];                 // gate input
+    __shared__ float s_h[kHidden], s_hn[kHidden], s_pre[4 * kHidden], s_hid[kHidden];
+    __shared__ float s_y[2];
+    __shared__ int s_base;
+
+    if (tid == 0) s_base = a.pool_len[b];
+
+    // ---- 1. per row: merge chunk partials -> top-k tokens, log-normaliser, candidate scores ----
+    for (int f = warp; f < F; f += kSelWarps) {
+        const size_t row = (size_t)b * F + f;
+        const float* pv = P.vp.part_v + row * n_chunks * k;
+        const int* pi = P.vp.part_i + row * n_chunks * k;
+        WarpTopList<float> top;
+        top.reset();
+        float thr = -CUDART_INF_F;
+        int thr_i = 0x7fffffff;
+        for (int c = 0; c < n_chunks; ++c) {
+            for (int e = 0; e < k; ++e) {
+                const float cv = pv[c * k + e];
+                const int ci = pi[c * k + e];
+                if (!precedes(cv, ci, thr, thr_i)) break;          // each chunk's list is sorted
+                top.insert(cv, ci);
+                thr = top.value_at(k - 1);
+                thr_i = top.index_at(k - 1);
+            }
+        }
+        // log-sum-exp over the chunks in fp64
+        float mloc = -CUDART_INF_F;
+        for (int c = lane; c < n_chunks; c += 32) mloc = fmaxf(mloc, P.vp.part_m[row * n_chunks + c]);
+        const float M = warp_max(mloc);
+        double sloc = 0.0;
+        for (int c = lane; c < n_chunks; c += 32) {
+            const float mc = P.vp.part_m[row * n_chunks + c];
+            if (mc > -CUDART_INF_F) sloc += (double)P.vp.part_s[row * n_chunks + c] * exp((double)mc - (double)M);
+        }
+        const double S = warp_sum(sloc);
+        const double lse = (double)M + log(S);
+        if (lane < k) {
+            const double logp = (double)top.v - lse;
+            const double sc = (double)a.parent_score[(size_t)b * F + f] + logp;
+            a.topk_tok[row * k + lane] = top.i;
+            a.topk_logp[row * k + lane] = (float)logp;
+            s_cand[f * k + lane] = sc;
+            s_ctok[f * k + lane] = top.i;
+        }
+    }
+    __syncthreads();
+    const int base = s_base;
+    const int n_cand = F * k;
+    if (base + n_cand > a.pool_capacity) {             // never write past the pool
+        if (tid == 0) { set_status(P.status, RADAR_ERR_INVALID_ARG); a.cont[b] = 0; a.active[b] = 0; }
+        return;
+    }
+
+    // ---- 2. append every candidate to the pool ----
+    const size_t pb = (size_t)b * a.pool_capacity + base;
+    for (int e = tid; e < n_cand; e += kSelThreads) {
+        const int f = e / k;
+        a.pool_tok[pb + e] = s_ctok[e];
+        a.pool_parent[pb + e] = a.parent_pool_idx[(size_t)b * F + f];
+        a.pool_score[pb + e] = (float)s_cand[e];
+        a.pool_depth[pb + e] = a.t;
+        a.pool_draft_row[pb + e] = -1;
+    }
+    __syncthreads();      // draft_row = -1 must land before the survivors overwrite theirs
+
+    // ---- 3. the k best candidates over all parents (score desc, flat index asc) ----
+    if (warp == 0) {
+        WarpTopList<double> top;
+        top.reset();
+        double thr = -CUDART_INF_F;
+        int thr_i = 0x7fffffff;
+        for (int e0 = 0; e0 < n_cand; e0 += 32) {
+            const int e = e0 + lane;
+            const bool valid = e < n_cand;
+            const double v = valid ? s_cand[e] : -CUDART_INF_F;
+            unsigned mk = __ballot_sync(kFull, valid && precedes(v, e, thr, thr_i));
+            while (mk) {
+                const int src = __ffs(mk) - 1;
+                mk &= mk - 1;
+                top.insert(__shfl_sync(kFull, v, src), e0 + src);
+            }
+            thr = top.value_at(k - 1);
+            thr_i = top.index_at(k - 1);
+        }
+        if (lane < k) {
+            const int e = top.i;
+            const float sc = (float)top.v;
+            const size_t o = (size_t)b * k + lane;
+            a.frontier_tok[o] = s_ctok[e];
+            a.frontier_score[o] = sc;
+            a.frontier_pool_idx[o] = base + e;
+            a.frontier_src_row[o] = e / k;
+            a.pool_draft_row[pb + e] = 1 + (a.t - 1) * k + lane;
+            s_sel[lane] = e;
+            s_x[lane] = (float)exp((double)sc);                  // confidence score in [0,1]
+        }
+        if (lane == 0) a.pool_len[b] = base + n_cand;
+    }
+    if (tid < H) s_h[tid] = a.h[(size_t)b * H + tid];
+    __syncthreads();
+
+    // ---- 4. prediction model ----
+    bool cont = false;
+    if (a.t < a.t_max) {
+        for (int r = warp; r < 4 * H; r += kSelWarps) {
+            float acc = row_dot(a.w_ih + (size_t)r * k, s_x, k, lane) + row_dot(a.w_hh + (size_t)r * H, s_h, H, lane);
+            if (lane == 0) s_pre[r] = acc + a.b_ih[r] + a.b_hh[r];
+        }
+        __syncthreads();
+        if (tid < H) {
+            const float ig = sigmoidf_(s_pre[tid]);
+            const float fg = sigmoidf_(s_pre[H + tid]);
+            const float gg = tanhf(s_pre[2 * H + tid]);
+            const float og = sigmoidf_(s_pre[3 * H + tid]);
+            const float cn = fg * a.c[(size_t)b * H + tid] + ig * gg;
+            const float hn = og * tanhf(cn);
+            a.c[(size_t)b * H + tid] = cn;
+            a.h[(size_t)b * H + tid] = hn;
+            s_hn[tid] = hn;
+        }
+        __syncthreads();
+        for (int r = warp; r < H; r += kSelWarps) {
+            const float* w = a.w1 + (size_t)r * (H + k);
+            float acc = row_dot(w, s_hn, H, lane) + row_dot(w + H, s_x, k, lane);
+            if (lane == 0) s_hid[r] = fmaxf(acc + a.b1[r], 0.f);
+        }
+        __syncthreads();
+        if (warp < 2) {
+            const float acc = row_dot(a.w2 + (size_t)warp * H, s_hid, H, lane);
+            if (lane == 0) s_y[warp] = acc + a.b2[warp];
+        }
+        __syncthreads();
+        cont = s_y[1] > s_y[0];
+        if (tid < 2) a.gate_logits[(size_t)b * 2 + tid] = s_y[tid];
+        if (a.force_calls != nullptr) cont = a.t < a.force_calls[b];
+    } else {
+        if (tid < 2) a.gate_logits[(size_t)b * 2 + tid] = 0.f;
+    }
+    if (tid == 0) {
+        a.cont[b] = cont ? 1 : 0;
+        a.active[b] = cont ? 1 : 0;
+    }
+}
+
+}  // namespace
+}  // namespace radar
+
+using namespace radar;
+
+extern "C" size_t radar_expand_workspace_bytes(const radar_ctx* ctx, int B, int F, int V, int k) {
+    if (!ctx || B <= 0 || F <= 0 || V <= 0 || k <= 0) return 0;
+    int chunk;
+    const int n_chunks = vocab_pass_plan_chunks(ctx->sm_count, B * F, V, &chunk);
+    return vocab_pass_partial_bytes(B * F, n_chunks, k);
+}
+
+extern "C" int radar_expand_step(radar_ctx* ctx, const radar_expand_args* a, void* stream_) {
+    if (!ctx || !a) return RADAR_ERR_INVALID_ARG;
+    cudaStream_t stream = reinterpret_cast<cudaStream_t>(stream_);
+    if (a->B <= 0 || a->F <= 0 || a->V <= 0 || a->k <= 0 || a->t < 1 || a->t > a->t_max) return RADAR_ERR_INVALID_ARG;
+    if (a->k > RADAR_MAX_K || a->F > kMaxF || a->V < a->k) return RADAR_ERR_UNSUPPORTED;
+    if (a->logits_dtype != RADAR_F32 && a->logits_dtype != RADAR_BF16) return RADAR_ERR_UNSUPPORTED;
+    if (a->logits_row_stride < a->V) return RADAR_ERR_INVALID_ARG;
+    if (!a->logits || !a->parent_score || !a->parent_pool_idx || !a->active || !a->h || !a->c || !a->pool_tok ||
+        !a->pool_parent || !a->pool_depth || !a->pool_draft_row || !a->pool_score || !a->pool_len ||
+        !a->frontier_tok || !a->frontier_score || !a->frontier_pool_idx || !a->frontier_src_row || !a->topk_tok ||
+        !a->topk_logp || !a->gate_logits || !a->cont || !a->workspace)
+        return RADAR_ERR_INVALID_ARG;
+    if (a->t < a->t_max && (!a->w_ih || !a->w_hh || !a->b_ih || !a->b_hh || !a->w1 || !a->b1 || !a->w2 || !a->b2))
+        return RADAR_ERR_INVALID_ARG;
+    if (a->pool_capacity < a->F * a->k) return RADAR_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(a->workspace) & 255) != 0) return RADAR_ERR_WORKSPACE;
+
+    SelectParams sp;
+    sp.a = *a;
+    sp.status = ctx->d_status;
+    VocabPassParams& vp = sp.vp;
+    vp.logits = a->logits;
+    vp.dtype = a->logits_dtype;
+    vp.row_stride = a->logits_row_stride;
+    vp.seq_stride = a->logits_seq_stride;
+    vp.n_seq = a->B;
+    vp.F = a->F;
+    vp.V = a->V;
+    vp.k = a->k;
+    vp.n_chunks = vocab_pass_plan_chunks(ctx->sm_count, a->B * a->F, a->V, &vp.chunk);
+    vp.want_lse = 1;
+    vp.seq_active = a->active;
+    vp.seq_rows = nullptr;
+    vp.status = ctx->d_status;
+    if (vocab_pass_partial_bytes(a->B * a->F, vp.n_chunks, a->k) > a->workspace_bytes) return RADAR_ERR_WORKSPACE;
+    vocab_pass_carve(a->workspace, a->B * a->F, vp.n_chunks, a->k, &vp);
+
+    RADAR_CUDA_CHECK(vocab_pass_launch(vp, stream));
+    expand_select_gate_kernel<<<a->B, kSelThreads, 0, stream>>>(sp);
+    RADAR_CUDA_CHECK(cudaGetLastError());
+    return RADAR_OK;
+}

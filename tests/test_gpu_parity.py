@@ -1,0 +1,165 @@
+"""Parity of the CUDA library (through the C ABI) against the CPU oracle on the same seeded
+inputs.  Needs a B200.  Sizes: the two small paper configurations in full, the batched ones
+reduced so that the oracle finishes in seconds while every kernel still spans several tiles,
+chunks and a ragged tail."""
+import numpy as np
+import pytest
+
+import harness as H
+from paper_2512_14069_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    from paper_2512_14069_b200 import binding as rb
+    c = rb.Context(0)
+    yield c
+    c.close()
+
+
+def small(cid):
+    """Reduced copies of the batched configurations (same head layout, dtype, k, t_max, N, mode)."""
+    cfg = W.CONFIGS[cid]
+    if cid == 3:
+        return W.shrink(cfg, B=3, Hq=8, Hkv=8, P=(1500, 1500), V=32000)
+    if cid == 4:
+        return W.shrink(cfg, B=3, Hq=16, Hkv=2, P=(1100, 1100), V=20011)       # odd V: unaligned rows
+    if cid == 5:
+        return W.shrink(cfg, B=4, Hq=8, Hkv=2, P=(300, 2100), V=30002)
+    return cfg
+
+
+@pytest.mark.parametrize("cid", [1, 2, 3, 4, 5])
+def test_whole_step_matches_oracle(ctx, cid):
+    cfg = small(cid)
+    inp = H.make_inputs(cfg)
+    pools, traces, trees = H.oracle_expand_and_tree(cfg, inp)
+    target = H.make_target(cfg, inp, trees)
+    accepts = H.oracle_accept(cfg, inp, trees, target)
+    H.check_margins(cfg, traces, trees, accepts)
+
+    g = H.GpuRun(cfg, inp, ctx)
+    g.expand_and_tree()
+    H.compare_expansion(cfg, g, pools, traces)
+    H.compare_tree(cfg, g, trees)
+
+    g.upload_attention()
+    O_gpu, lse_gpu = g.attention()                      # masks from the CUDA tree build
+    O_ref, lse_ref = H.oracle_attention(cfg, inp, trees)
+    H.compare_attention(cfg, O_gpu, lse_gpu, O_ref, lse_ref, trees)
+
+    g.accept(target)
+    H.compare_accept(cfg, g, accepts)
+
+
+@pytest.mark.parametrize("cid", [1, 3])
+def test_bf16_logits_with_many_ties(ctx, cid):
+    """bf16 logits collide often: token order must still be (value desc, id asc) bit for bit."""
+    cfg = small(cid)
+    inp = H.make_inputs(cfg, with_attention=False)
+    inp["draft"] = W.bf16_bits_to_f32(W.f32_to_bf16_bits(inp["draft"])).reshape(inp["draft"].shape)
+    pools, traces, trees = H.oracle_expand_and_tree(cfg, inp)
+    target = H.make_target(cfg, inp, trees)
+    target = W.bf16_bits_to_f32(W.f32_to_bf16_bits(target)).reshape(target.shape)
+    gcfg = W.shrink(cfg, mode="greedy")
+    accepts = H.oracle_accept(gcfg, inp, trees, target)
+    g = H.GpuRun(gcfg, inp, ctx, logits_bf16=True)
+    g.expand_and_tree()
+    for b in range(cfg.B):
+        for tr in traces[b]:
+            i = tr["t"] - 1
+            got = g.step.topk_tok1[b] if tr["t"] == 1 else g.step.topk_tok[i, b]
+            assert np.array_equal(got.cpu().numpy(), tr["topk_tok"])
+    if all(tr["margin"] > H.TAU_SCORE for b in range(cfg.B) for tr in traces[b]):
+        H.compare_expansion(cfg, g, pools, traces)
+        H.compare_tree(cfg, g, trees)
+        g.accept(target)
+        H.compare_accept(gcfg, g, accepts)
+
+
+def test_attention_with_oracle_masks_and_ragged_trees(ctx):
+    """Attention alone, masks and tree sizes taken from the oracle: ragged prefixes and trees,
+    a root-only tree, a prefix shorter than one tile, GQA with G = 4."""
+    cfg = W.shrink(W.CONFIGS[5], B=5, Hq=8, Hkv=2, P=(1, 900), V=2000, k=4, t_max=5, N=40)
+    inp = H.make_inputs(cfg)
+    inp["prefix_len"][0] = 1
+    inp["Kc"][0], inp["Vc"][0] = inp["Kc"][0][:1], inp["Vc"][0][:1]
+    _, _, trees = H.oracle_expand_and_tree(cfg, inp)
+    trees[1] = dict(trees[1]); trees[1]["n_nodes"] = 1                        # root only
+    g = H.GpuRun(cfg, inp, ctx)
+    g.upload_attention()
+    O_gpu, lse_gpu = g.attention(trees)
+    O_ref, lse_ref = H.oracle_attention(cfg, inp, trees)
+    H.compare_attention(cfg, O_gpu, lse_gpu, O_ref, lse_ref, trees)
+
+
+def test_attention_fp32_head_dim_64_and_128(ctx):
+    for d in (64, 128):
+        cfg = W.shrink(W.CONFIGS[1], cid=40 + d, B=2, Hq=4, Hkv=2, d=d, P=(257, 257))
+        inp = H.make_inputs(cfg)
+        _, _, trees = H.oracle_expand_and_tree(cfg, inp)
+        g = H.GpuRun(cfg, inp, ctx)
+        g.upload_attention()
+        O_gpu, lse_gpu = g.attention(trees)
+        O_ref, lse_ref = H.oracle_attention(cfg, inp, trees)
+        H.compare_attention(cfg, O_gpu, lse_gpu, O_ref, lse_ref, trees)
+
+
+@pytest.mark.parametrize("k,V", [(1, 77), (32, 4099), (7, 33)])
+def test_expansion_edge_sizes(ctx, k, V):
+    t_max = 3 if k == 32 else 4
+    cfg = W.shrink(W.CONFIGS[1], cid=60 + k, V=V, k=k, t_max=t_max, N=min(63, 3 * k), B=2, gate_b2_offset=5.0)
+    inp = H.make_inputs(cfg, with_attention=False)
+    pools, traces, trees = H.oracle_expand_and_tree(cfg, inp)
+    H.check_margins(cfg, traces, trees)
+    g = H.GpuRun(cfg, inp, ctx)
+    g.expand_and_tree()
+    H.compare_expansion(cfg, g, pools, traces)
+    H.compare_tree(cfg, g, trees)
+
+
+def test_minus_inf_logits_and_nan_status(ctx):
+    import torch
+    cfg = W.shrink(W.CONFIGS[1], cid=70, B=1)
+    inp = H.make_inputs(cfg, with_attention=False)
+    inp["draft"][0, :, 5:200] = -np.inf
+    pools, traces, trees = H.oracle_expand_and_tree(cfg, inp)
+    g = H.GpuRun(cfg, inp, ctx)
+    g.expand_and_tree()
+    H.compare_expansion(cfg, g, pools, traces)
+    # a NaN is reported through the status word, nothing faults
+    inp["draft"][0, 0, 17] = np.nan
+    g2 = H.GpuRun(cfg, inp, ctx)
+    g2.step.run_expansion(g2.draft, g2.gate, g2.force)
+    from paper_2512_14069_b200 import binding as rb
+    assert ctx.read_device_status() == -6
+    assert ctx.read_device_status() == rb.RADAR_OK          # reading clears it
+    torch.cuda.synchronize()
+
+
+def test_host_side_argument_errors(ctx):
+    import torch
+    from paper_2512_14069_b200 import binding as rb
+    cfg = W.CONFIGS[1]
+    inp = H.make_inputs(cfg, with_attention=False)
+    g = H.GpuRun(cfg, inp, ctx)
+    s = g.step
+    with pytest.raises(rb.RadarError) as e:
+        s.k = 33
+        s.expand(1, g.draft, g.gate)
+    assert e.value.status == -2
+    s.k = cfg.k
+    with pytest.raises(rb.RadarError) as e:
+        ws = s.ws_expand
+        s.ws_expand = ws[:16]
+        s.expand(1, g.draft, g.gate)
+    assert e.value.status == -3
+    s.ws_expand = ws
+    with pytest.raises(rb.RadarError) as e:
+        s.d = 96
+        s.attention(s.O, s.O, s.O, torch.zeros(1, dtype=torch.int64, device="cuda"), g.prefix_len, s.O, s.O)
+    assert e.value.status == -2
+    torch.cuda.synchronize()
+    assert ctx.read_device_status() == 0
