@@ -1,0 +1,477 @@
+#!/usr/bin/env python
+"""Benchmark of one RADAR speculative step (expansion calls + gate, rerank/tree build, one layer of
+tree attention, acceptance) on seeded synthetic inputs.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--config C] [--impl ours|reference]
+
+Prints ONE JSON line (rank 0).  `value` = whole-job speculative steps per second with the
+inputs resident in HBM; `e2e` = the same through host buffers (H2D of every input and D2H of the
+result inside the timed region); `roofline` = the dominant kernel's algorithmic bytes / its
+CUDA-event duration against the measured HBM peak; `cpu_baseline` = the CPU oracle on the host.
+N > 1 runs independent replicas of the batch (the path has no cross-sequence exchange): weak
+scaling, no collective on the data path.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2512_14069_b200 import workloads as W  # noqa: E402
+
+METRIC, UNIT = "tree_verify_steps_per_s", "steps/s"
+L2_BYTES = 126 * 1024 * 1024
+# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under profiles/
+# (kernel name, config id) -> bytes; absent = not captured.
+NCU_TRAFFIC = {}
+
+
+def parse():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--config", type=int, default=2, choices=sorted(W.CONFIGS))
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-graph", action="store_true", help="launch eagerly instead of replaying CUDA graphs")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    return ap.parse_args()
+
+
+# ------------------------------------------------------------------------------------------------
+# workload (numpy, seeded) for `rank`: sequences rank*B .. rank*B+B-1 of the configuration
+# ------------------------------------------------------------------------------------------------
+def host_inputs(cfg, rank):
+    B = cfg.B
+    gb = lambda b: rank * B + b
+    plen_all = W.prefix_lens(W.shrink(cfg, B=B * (rank + 1)))[rank * B:]
+    inp = {
+        "draft": np.stack([W.draft_logits(cfg, gb(b)) for b in range(B)]),
+        "gate": W.gate_weights(cfg),
+        "force_calls": None if cfg.depth_plan == "gate" else W.forced_calls(W.shrink(cfg, B=B * (rank + 1)))[rank * B:],
+        "n_keep": np.minimum(W.keep_sizes(W.shrink(cfg, B=B * (rank + 1)))[rank * B:], cfg.N).astype(np.int32),
+        "root_tok": W.root_tokens(W.shrink(cfg, B=B * (rank + 1)))[rank * B:],
+        "prefix_len": plen_all.astype(np.int32),
+        "Q": np.stack([W.attn_q(cfg, gb(b)) for b in range(B)]),
+    }
+    kt, vt = zip(*[W.attn_tree_kv(cfg, gb(b)) for b in range(B)])
+    inp["Kt"], inp["Vt"] = np.stack(kt), np.stack(vt)
+    kc, vc = zip(*[W.attn_prefix_kv(cfg, gb(b), int(plen_all[b])) for b in range(B)])
+    inp["Kc"], inp["Vc"] = np.concatenate(kc, 0), np.concatenate(vc, 0)
+    inp["kv_start"] = np.concatenate([[0], np.cumsum(plen_all)[:-1]]).astype(np.int64)
+    ua, us = W.accept_uniforms(W.shrink(cfg, B=B * (rank + 1)))
+    inp["u_accept"], inp["u_sample"] = ua[rank * B:], us[rank * B:]
+    return inp
+
+
+def torch_of(x):
+    import torch
+    t = torch.from_numpy(np.ascontiguousarray(x))
+    if x.dtype == np.uint16:
+        t = t.view(torch.int16).view(torch.bfloat16)
+    return t
+
+
+class ClockSampler:
+    """nvidia-smi clocks / throttle reasons sampled every 100 ms while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.proc, self.path = index, None, None
+
+    def start(self):
+        try:
+            f = tempfile.NamedTemporaryFile("w", suffix=".csv", delete=False)
+            self.path = f.name
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q,
+                                          "--format=csv,noheader,nounits", "-lms", "100"], stdout=f,
+                                         stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": []}
+        if self.proc is None:
+            return out
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, reasons, mx = [], set(), None
+        try:
+            for line in open(self.path):
+                p = [x.strip() for x in line.split(",")]
+                if len(p) < 9:
+                    continue
+                try:
+                    sm.append(float(p[1])); mx = float(p[2])
+                except ValueError:
+                    continue
+                for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), p[5:9]):
+                    if v.lower().startswith("active"):
+                        reasons.add(name)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if sm:
+            out.update(sm_mhz=float(np.median(sm)), sm_max_mhz=mx, reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+def measured_peak_gbs():
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return 6650.0, "fallback"
+
+
+# ------------------------------------------------------------------------------------------------
+# our arm
+# ------------------------------------------------------------------------------------------------
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2512_14069_b200 import binding as rb
+    from paper_2512_14069_b200.pipeline import SpecStep
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    dev = torch.device("cuda", local)
+    cfg = W.CONFIGS[args.config]
+    B, V, k, t_max = cfg.B, cfg.V, cfg.k, cfg.t_max
+    sizeof_logit = 4
+
+    inp = host_inputs(cfg, rank)
+    ctx = rb.Context(local)
+    kvdt = torch.float32 if cfg.kv_dtype == "f32" else torch.bfloat16
+    mode = rb.RADAR_GREEDY if cfg.mode == "greedy" else rb.RADAR_STOCHASTIC
+    max_p = int(inp["prefix_len"].max())
+    step = SpecStep(ctx, B=B, V=V, k=k, t_max=t_max, N=cfg.N, Hq=cfg.Hq, Hkv=cfg.Hkv, d=cfg.d, kv_dtype=kvdt,
+                    max_prefix_len=max_p, mode=mode, temperature=float(np.float32(cfg.temperature)), device=dev)
+    gate = {n: torch_of(v).to(dev) for n, v in inp["gate"].items()}
+    force = None if inp["force_calls"] is None else torch_of(inp["force_calls"]).to(dev)
+    n_keep, root_tok = torch_of(inp["n_keep"]).to(dev), torch_of(inp["root_tok"]).to(dev)
+    prefix_len, kv_start = torch_of(inp["prefix_len"]).to(dev), torch_of(inp["kv_start"]).to(dev)
+    u_acc, u_smp = torch_of(inp["u_accept"]).to(dev), torch_of(inp["u_sample"]).to(dev)
+
+    # untimed pre-pass: the tree decides which draft row each target row is a noisy copy of
+    d0 = torch_of(inp["draft"]).to(dev)
+    step.run_expansion(d0, gate, force)
+    step.build_tree(root_tok, prefix_len, n_keep)
+    ctx.check_device_status()
+    n_nodes = step.n_nodes.cpu().numpy()
+    drow = step.tree_draft_row.cpu().numpy()
+    calls = np.array([int((step.pool_len[b].item() - k) // (k * k)) + 1 for b in range(B)])
+    inp["target"] = np.stack([W.target_logits(cfg, rank * B + b, inp["draft"][b], drow[b], int(n_nodes[b]))
+                              for b in range(B)])
+    del d0
+
+    # input copies: rotate through enough of them that the bytes touched between two uses of a copy exceed L2
+    names = ["draft", "target", "Q", "Kt", "Vt", "Kc", "Vc"]
+    host = {n: torch_of(inp[n]) for n in names}
+    bytes_per_copy = sum(t.numel() * t.element_size() for t in host.values())
+    free_b, _ = torch.cuda.mem_get_info(dev)
+    n_copies = int(min(max(2, -(-3 * L2_BYTES // bytes_per_copy) + 1), max(2, (free_b // 2) // bytes_per_copy), 16))
+    copies = [{n: host[n].to(dev) for n in names} for _ in range(n_copies)]
+
+    def one_step(c):
+        step.run_expansion(c["draft"], gate, force)
+        step.build_tree(root_tok, prefix_len, n_keep)
+        step.attention(c["Q"], c["Kc"], c["Vc"], kv_start, prefix_len, c["Kt"], c["Vt"])
+        if mode == rb.RADAR_GREEDY:
+            step.accept(c["target"])
+        else:
+            step.accept(c["target"], c["draft"], u_acc, u_smp)
+
+    stream = torch.cuda.Stream(dev)
+    graphs = None
+    with torch.cuda.stream(stream):
+        for i in range(max(args.warmup, 3)):
+            one_step(copies[i % n_copies])
+        stream.synchronize()
+        ctx.check_device_status(stream)
+        if not args.no_graph:
+            try:
+                graphs = []
+                for c in copies:
+                    g = torch.cuda.CUDAGraph()
+                    with torch.cuda.graph(g, stream=stream):
+                        one_step(c)
+                    graphs.append(g)
+                for g in graphs:
+                    g.replay()
+                stream.synchronize()
+            except Exception as e:  # pragma: no cover
+                sys.stderr.write("graph capture failed (%s); timing eager launches\n" % e)
+                graphs = None
+
+        def run(i):
+            if graphs is not None:
+                graphs[i % n_copies].replay()
+            else:
+                one_step(copies[i % n_copies])
+
+        sampler = ClockSampler(local)                 # samples through the warm-up and the timed region
+        if rank == 0:
+            sampler.start()
+        for i in range(max(args.warmup, 3)):
+            run(i)
+        stream.synchronize()
+
+        # ---- timed region: exactly K steps, device time, max over ranks ----
+        ctx.reset_launch_counts()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for i in range(args.steps):
+            run(i)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        ms_total = e0.elapsed_time(e1)
+        clocks = sampler.stop() if rank == 0 else None
+        # graph replays do not pass through the library's host-side counters: count what one step launches
+        if graphs is not None:
+            ctx.reset_launch_counts()
+            one_step(copies[0])
+            stream.synchronize()
+            launches_per_step = sum(v[0] for v in ctx.kernel_stats().values())
+        else:
+            launches_per_step = sum(v[0] for v in ctx.kernel_stats().values()) // max(args.steps, 1)
+        ctx.check_device_status(stream)
+
+        # ---- per-kernel durations (CUDA events around every kernel, eager launches, same rotation) ----
+        prof_steps = min(args.steps, 50)
+        ctx.profile_begin(prof_steps * (2 * t_max + 8))
+        for i in range(prof_steps):
+            one_step(copies[i % n_copies])
+        ctx.profile_end()
+        kstats = ctx.kernel_stats()
+
+        # ---- end to end through host buffers ----
+        pinned = {n: host[n].pin_memory() for n in names}
+        stage = copies[0]
+        res_dev = [step.accept_len, step.next_token, step.best_retrieve_row, step.path_nodes, step.path_tokens]
+        res_host = [torch.empty_like(t, device="cpu").pin_memory() for t in res_dev]
+        h2d = sum(t.numel() * t.element_size() for t in pinned.values())
+        d2h = sum(t.numel() * t.element_size() for t in res_host)
+
+        def e2e_step():
+            for n in names:
+                stage[n].copy_(pinned[n], non_blocking=True)
+            if graphs is not None:
+                graphs[0].replay()
+            else:
+                one_step(stage)
+            for hst, dv in zip(res_host, res_dev):
+                hst.copy_(dv, non_blocking=True)
+            stream.synchronize()
+
+        for _ in range(3):
+            e2e_step()
+        e2e_steps = max(3, min(args.steps, 30))
+        if world > 1:
+            dist.barrier()
+        t0 = time.perf_counter()
+        for _ in range(e2e_steps):
+            e2e_step()
+        e2e_s = time.perf_counter() - t0
+
+    t = torch.tensor([ms_total, e2e_s], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_total, e2e_s = float(t[0]), float(t[1])
+    ms_per_step = ms_total / args.steps
+    value = world * 1000.0 / ms_per_step
+    tree_rows = int(n_nodes.sum())
+
+    # ---- roofline of the dominant kernel ----
+    s = sizeof_logit
+    kv_b = 2 if cfg.kv_dtype == "bf16" else 4
+    plen = inp["prefix_len"].astype(np.int64)
+    rows_expand = int(sum(1 + (c - 1) * k for c in calls))
+    alg = {   # algorithmic bytes per STEP of each HBM-bound kernel
+        "vocab_pass(expand)": rows_expand * V * s,
+        "vocab_pass(accept)": int(n_nodes.sum()) * V * s,
+        "tree_attention": int(((plen + n_nodes) * cfg.Hkv * cfg.d * 2 * kv_b).sum()
+                              + 2 * n_nodes.sum() * cfg.Hq * cfg.d * kv_b),
+    }
+    if mode == rb.RADAR_STOCHASTIC:
+        alen = step.accept_len.cpu().numpy()
+        alg["stochastic_walk"] = int(((alen + 1) * 2 * V * s).sum())      # target + draft row of each visited node, once
+    timed = {n: v for n, v in kstats.items() if v[2] > 0}
+    dom = max(timed, key=lambda n: timed[n][1]) if timed else None
+    peak, peak_kind = measured_peak_gbs()
+    roofline = None
+    kernels = {n: {"launches_per_step": v[2] / prof_steps, "avg_us": 1000.0 * v[1] / v[2],
+                   "share": v[1] / sum(x[1] for x in timed.values())} for n, v in timed.items()}
+    for n in kernels:
+        if n in alg:
+            per_launch = alg[n] / kernels[n]["launches_per_step"]
+            kernels[n]["alg_bytes_per_launch"] = per_launch
+            kernels[n]["gbs"] = per_launch / (kernels[n]["avg_us"] * 1e-6) / 1e9
+    if dom is not None:
+        if dom in alg:
+            ach = kernels[dom]["gbs"]
+            roofline = {"kernel": dom, "bound": "hbm", "achieved": ach, "peak": peak, "unit": "GB/s",
+                        "frac": ach / peak, "peak_kind": "of " + peak_kind,
+                        "traffic": NCU_TRAFFIC.get((dom, cfg.cid)),
+                        "alg_bytes_per_launch": kernels[dom]["alg_bytes_per_launch"], "avg_us": kernels[dom]["avg_us"]}
+        else:
+            roofline = {"kernel": dom, "bound": "latency", "achieved": None, "peak": peak, "unit": "GB/s",
+                        "frac": None, "traffic": None, "avg_us": kernels[dom]["avg_us"]}
+
+    out = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32" if cfg.kv_dtype == "f32" else "bf16", "data": "synthetic",
+        "config": {"workload": "config %d (%s): B=%d, Hq/Hkv/d=%d/%d/%d, prefix %s, V=%d, k=%d, t_max=%d, N=%d, %s"
+                   % (cfg.cid, cfg.name, B, cfg.Hq, cfg.Hkv, cfg.d, "%d..%d" % (plen.min(), plen.max()), V, k, t_max,
+                      cfg.N, cfg.mode),
+                   "per_gpu_batch": B, "draft_calls_per_seq": calls.tolist(), "tree_rows_per_seq": n_nodes.tolist(),
+                   "logits_dtype": "f32", "kv_dtype": cfg.kv_dtype, "layers_of_attention": 1,
+                   "l2": "inputs rotate over %d copies (%.0f MB each), more than L2 between reuses" % (n_copies, bytes_per_copy / 1e6),
+                   "launch": "cuda graph replay" if graphs is not None else "eager"},
+        "tree_tokens_per_s": value * tree_rows,
+        "clocks": clocks,
+        "e2e": {"value": world * e2e_steps / e2e_s, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+        "gpu_launches": int(launches_per_step * args.steps),
+        "roofline": roofline,
+        "kernels": kernels,
+    }
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        out["cpu_baseline"] = cpu_baseline(cfg, budget_s=15.0)
+    if rank == 0:
+        print(json.dumps(out))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+# ------------------------------------------------------------------------------------------------
+# CPU oracle timing (reported baseline and the `--impl reference` arm)
+# ------------------------------------------------------------------------------------------------
+class OracleWorkload:
+    """The oracle's whole step on rank 0's batch, with a knob that runs only a fraction of the three
+    heavy loops (draft rows, attention (sequence, head) pairs, target rows)."""
+
+    def __init__(self, cfg):
+        sys.path.insert(0, os.path.join(ROOT, "tests"))
+        import harness as H
+        self.H, self.cfg = H, cfg
+        self.inp = H.make_inputs(cfg)
+        self.pools, self.traces, self.trees = H.oracle_expand_and_tree(cfg, self.inp)
+        self.target = H.make_target(cfg, self.inp, self.trees)
+
+    def full_step(self):
+        H, cfg = self.H, self.cfg
+        pools, traces, trees = H.oracle_expand_and_tree(cfg, self.inp)
+        H.oracle_attention(cfg, self.inp, trees)
+        H.oracle_accept(cfg, self.inp, trees, self.target)
+
+    def sampled_step(self, frac):
+        """Fraction `frac` of the heavy units; the light parts (frontier, gate, tree, walk: well under 1 %
+        of the oracle's time) are not repeated."""
+        from oracle import radar_oracle as O
+        cfg, inp = self.cfg, self.inp
+        rows = [(b, r) for b in range(cfg.B) for r in range(1 + (len(self.traces[b]) - 1) * cfg.k)]
+        for b, r in rows[: max(1, int(round(frac * len(rows))))]:
+            O.vocab_topk(inp["draft"][b, r], cfg.k)
+        pairs = [(b, h) for b in range(cfg.B) for h in range(cfg.Hq)]
+        self.H.oracle_attention(cfg, inp, self.trees, pairs=pairs[: max(1, int(round(frac * len(pairs))))])
+        trows = [(b, i) for b in range(cfg.B) for i in range(self.trees[b]["n_nodes"])]
+        for b, i in trows[: max(1, int(round(frac * len(trows))))]:
+            if cfg.mode == "greedy":
+                int(np.argmax(self.target[b, i]))
+            else:
+                O.log_softmax(self.target[b, i] / np.float32(cfg.temperature))
+
+
+def _single_thread():
+    try:
+        from threadpoolctl import threadpool_limits
+        return threadpool_limits(limits=1)
+    except Exception:
+        import contextlib
+        return contextlib.nullcontext()
+
+
+def cpu_baseline(cfg, budget_s):
+    with _single_thread():
+        wl = OracleWorkload(cfg)
+        t0 = time.perf_counter()
+        wl.full_step() if cfg.cid <= 2 else wl.sampled_step(0.02)
+        probe = time.perf_counter() - t0
+        full_est = probe if cfg.cid <= 2 else probe / 0.02
+        frac = 1.0 if full_est <= budget_s else max(budget_s / full_est, 1e-3)
+        reps = max(1, int(budget_s / max(full_est * frac, 1e-3))) if frac == 1.0 else 1
+        t0 = time.perf_counter()
+        for _ in range(reps):
+            wl.full_step() if frac == 1.0 else wl.sampled_step(frac)
+        dt = (time.perf_counter() - t0) / reps
+    return {"value": frac / dt, "unit": UNIT, "cores": 1, "kind": "oracle",
+            "sample": ("whole step, %d repetitions" % reps) if frac == 1.0 else
+            ("fraction %.4f of the draft rows, attention (sequence, head) pairs and target rows of one step" % frac)}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    cfg = W.CONFIGS[args.config]
+    with _single_thread():
+        wl = OracleWorkload(cfg)
+        t0 = time.perf_counter()
+        wl.sampled_step(0.05)
+        full_est = (time.perf_counter() - t0) / 0.05
+        budget = 150.0 / (args.steps + args.warmup)
+        frac = min(1.0, max(budget / full_est, 1e-4))
+        stepf = (lambda: wl.full_step()) if frac >= 1.0 else (lambda: wl.sampled_step(frac))
+        for _ in range(args.warmup):
+            stepf()
+        t0 = time.perf_counter()
+        for _ in range(args.steps):
+            stepf()
+        dt = (time.perf_counter() - t0) / args.steps
+    value = min(frac, 1.0) / dt
+    sample = "whole step" if frac >= 1.0 else \
+        "fraction %.4f of the draft rows, attention (sequence, head) pairs and target rows per step" % frac
+    n_rows = int(sum(t["n_nodes"] for t in wl.trees))
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": 1000.0 / value, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": "config %d (%s), CPU oracle" % (cfg.cid, cfg.name)},
+        "tree_tokens_per_s": value * n_rows,
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+if __name__ == "__main__":
+    a = parse()
+    if a.impl == "reference":
+        run_reference(a)
+    else:
+        run_ours(a)

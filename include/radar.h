@@ -62,6 +62,18 @@ const char* radar_status_string(int status);
  * error recorded since the last read) and clears it. */
 int radar_read_device_status(radar_ctx* ctx, void* stream);
 
+/* Measurement helpers (no counterpart in the paper): host-side launch counts per kernel and,
+ * between radar_profile_begin and radar_profile_end, a CUDA-event pair around every kernel the
+ * library launches (on the launching stream).  radar_profile_begin creates 2 * max_records events;
+ * radar_profile_end synchronises the device, accumulates the durations and destroys the events.
+ * Do not profile inside a stream capture.  radar_kernel_stats: all out-pointers are host, optional. */
+int radar_profile_begin(radar_ctx* ctx, int max_records);
+int radar_profile_end(radar_ctx* ctx);
+int radar_kernel_count(void);
+const char* radar_kernel_name(int id);
+int radar_kernel_stats(const radar_ctx* ctx, int id, long long* launches, double* timed_ms, long long* timed_launches);
+int radar_reset_launch_counts(radar_ctx* ctx);
+
 /* ------------------------------------------------------------------------------------------
  * radar_expand_step - one draft call's worth of tree expansion for every active sequence.
  * (Appendix walkthrough: each frontier token yields its k most probable tokens with their
@@ -76,8 +88,10 @@ int radar_read_device_status(radar_ctx* ctx, void* stream);
  *   single-layer LSTM (gate blocks i,f,g,o; state h,c) then Linear(H+k,H)-ReLU-Linear(H,2) on
  *   [h';x]; cont = logit[1] > logit[0].  At t == t_max the model is skipped, cont = 0 and
  *   gate_logits = 0.  If force_calls is given, cont = (t < force_calls[b]) instead.
- *   active[b] <- cont[b].  Sequences with active[b] == 0 are skipped: nothing of theirs is
- *   touched, except cont[b] <- 0.
+ *   active[b] <- cont[b].  For t > 1, sequences with active[b] == 0 are skipped: nothing of
+ *   theirs is touched, except cont[b] <- 0.  Call t == 1 starts a new speculative step for every
+ *   sequence: the incoming active, h, c and pool_len are ignored (taken as 1, 0, 0 and 0), so a
+ *   step needs no separate reset.
  * A NaN logit records RADAR_ERR_NUMERIC (outputs of that sequence unspecified).
  * Limits: 1 <= k <= RADAR_MAX_K, 1 <= F <= 32, V >= k, pool_len[b] + F*k <= pool_capacity.
  */
@@ -90,11 +104,11 @@ typedef struct {
     int64_t logits_seq_stride;          /* elements between consecutive sequences b          */
     const float* parent_score;          /* [B][F] cumulative log-prob of each frontier row   */
     const int32_t* parent_pool_idx;     /* [B][F] pool index of each frontier row, -1 = root */
-    uint8_t* active;                    /* [B] in/out                                        */
+    uint8_t* active;                    /* [B] in/out (out only at t = 1)                    */
     const int32_t* force_calls;         /* [B] or NULL                                       */
     const float *w_ih, *w_hh, *b_ih, *b_hh;   /* LSTM: [4H][k], [4H][H], [4H], [4H]          */
     const float *w1, *b1, *w2, *b2;           /* MLP : [H][H+k], [H], [2][H], [2]            */
-    float* h;                           /* [B][H] in/out, caller zeroes before t = 1         */
+    float* h;                           /* [B][H] in/out (out only at t = 1)                 */
     float* c;                           /* [B][H] in/out                                     */
     int pool_capacity;                  /* C                                                 */
     int32_t *pool_tok, *pool_parent, *pool_depth, *pool_draft_row;   /* [B][C] in/out        */

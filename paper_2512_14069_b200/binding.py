@@ -104,6 +104,18 @@ def lib() -> ctypes.CDLL:
         L.radar_accept_workspace_bytes.argtypes = [_vp, _c_int, _c_int, _c_int]
         L.radar_verify_accept.restype = _c_int
         L.radar_verify_accept.argtypes = [_vp, ctypes.POINTER(AcceptArgs), _vp]
+        L.radar_profile_begin.restype = _c_int
+        L.radar_profile_begin.argtypes = [_vp, _c_int]
+        L.radar_profile_end.restype = _c_int
+        L.radar_profile_end.argtypes = [_vp]
+        L.radar_kernel_count.restype = _c_int
+        L.radar_kernel_name.restype = ctypes.c_char_p
+        L.radar_kernel_name.argtypes = [_c_int]
+        L.radar_kernel_stats.restype = _c_int
+        L.radar_kernel_stats.argtypes = [_vp, _c_int, ctypes.POINTER(ctypes.c_longlong),
+                                         ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_longlong)]
+        L.radar_reset_launch_counts.restype = _c_int
+        L.radar_reset_launch_counts.argtypes = [_vp]
         _lib = L
     return _lib
 
@@ -169,6 +181,26 @@ class Context:
 
     def check_device_status(self, stream=None):
         _check("device status", self.read_device_status(stream))
+
+    # ---- measurement helpers ----
+    def profile_begin(self, max_records: int):
+        _check("radar_profile_begin", lib().radar_profile_begin(self.handle, max_records))
+
+    def profile_end(self):
+        _check("radar_profile_end", lib().radar_profile_end(self.handle))
+
+    def reset_launch_counts(self):
+        _check("radar_reset_launch_counts", lib().radar_reset_launch_counts(self.handle))
+
+    def kernel_stats(self) -> dict:
+        """{kernel name: (launches since reset, event-timed ms, event-timed launches)}"""
+        out = {}
+        for i in range(lib().radar_kernel_count()):
+            n, ms, tn = ctypes.c_longlong(), ctypes.c_double(), ctypes.c_longlong()
+            _check("radar_kernel_stats", lib().radar_kernel_stats(self.handle, i, ctypes.byref(n), ctypes.byref(ms),
+                                                                  ctypes.byref(tn)))
+            out[lib().radar_kernel_name(i).decode()] = (n.value, ms.value, tn.value)
+        return out
 
 
 def radar_expand_workspace_bytes(ctx: Context, B, F, V, k) -> int:

@@ -7,10 +7,50 @@
 
 #include "../../include/radar.h"
 
+// kernels the library launches (index into the profiling tables)
+enum radar_kernel_id {
+    RADAR_K_VOCAB_EXPAND = 0,   // vocabulary pass of radar_expand_step
+    RADAR_K_SELECT_GATE,        // partial merge + frontier selection + prediction model
+    RADAR_K_TREE_BUILD,
+    RADAR_K_ATTN,               // tree attention main kernel
+    RADAR_K_ATTN_COMBINE,
+    RADAR_K_VOCAB_ACCEPT,       // row-argmax pass of greedy acceptance
+    RADAR_K_GREEDY_WALK,
+    RADAR_K_STOCH_WALK,
+    RADAR_K_COUNT
+};
+
 struct radar_ctx {
     int device;
     int sm_count;
     int* d_status;          // sticky device status word
+    // launch accounting (host side)
+    long long launches[RADAR_K_COUNT];
+    // optional per-kernel CUDA-event timing
+    bool profiling;
+    cudaEvent_t* ev;        // 2 * ev_cap events
+    int* ev_kernel;         // kernel id of record i
+    int ev_cap, ev_used;
+    double prof_ms[RADAR_K_COUNT];
+    long long prof_n[RADAR_K_COUNT];
+};
+
+// Brackets one kernel launch: counts it and, while profiling, records an event pair on its stream.
+struct radar_launch_scope {
+    radar_ctx* c;
+    cudaStream_t s;
+    int slot;
+    radar_launch_scope(radar_ctx* ctx, int kernel, cudaStream_t stream) : c(ctx), s(stream), slot(-1) {
+        c->launches[kernel]++;
+        if (c->profiling && c->ev_used < c->ev_cap) {
+            slot = c->ev_used++;
+            c->ev_kernel[slot] = kernel;
+            cudaEventRecord(c->ev[2 * slot], s);
+        }
+    }
+    ~radar_launch_scope() {
+        if (slot >= 0) cudaEventRecord(c->ev[2 * slot + 1], s);
+    }
 };
 
 #define RADAR_CUDA_CHECK(expr)                         \
@@ -102,7 +142,7 @@ struct VocabPassParams {
 int vocab_pass_plan_chunks(int sm_count, int rows, int V, int* chunk_out);   // returns n_chunks
 size_t vocab_pass_partial_bytes(int rows, int n_chunks, int k);
 void vocab_pass_carve(void* ws, int rows, int n_chunks, int k, VocabPassParams* p);
-cudaError_t vocab_pass_launch(const VocabPassParams& p, cudaStream_t stream);
+cudaError_t vocab_pass_launch(radar_ctx* ctx, int kernel_id, const VocabPassParams& p, cudaStream_t stream);
 
 static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 

@@ -30,7 +30,7 @@ __global__ void __launch_bounds__(kSelThreads) expand_select_gate_kernel(const S
     const radar_expand_args& a = P.a;
     const int b = blockIdx.x;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    if (a.active[b] == 0) {
+    if (a.t > 1 && a.active[b] == 0) {                 // call 1 always runs: it (re)starts every sequence
         if (tid == 0) a.cont[b] = 0;
         return;
     }
@@ -39,13 +39,12 @@ __global__ void __launch_bounds__(kSelThreads) expand_select_gate_kernel(const S
 
     __shared__ double s_cand[kMaxF * RADAR_MAX_K];     // candidate scores, flat (f, j)
     __shared__ int s_ctok[kMaxF * RADAR_MAX_K];
-    __shared__ int s_sel[RADAR_MAX_K];
     __shared__ float s_x[RADAR_MAX_K];                 // gate input
     __shared__ float s_h[kHidden], s_hn[kHidden], s_pre[4 * kHidden], s_hid[kHidden];
     __shared__ float s_y[2];
     __shared__ int s_base;
 
-    if (tid == 0) s_base = a.pool_len[b];
+    if (tid == 0) s_base = a.t > 1 ? a.pool_len[b] : 0;
 
     // ---- 1. per row: merge chunk partials -> top-k tokens, log-normaliser, candidate scores ----
     for (int f = warp; f < F; f += kSelWarps) {
@@ -134,12 +133,11 @@ __global__ void __launch_bounds__(kSelThreads) expand_select_gate_kernel(const S
             a.frontier_pool_idx[o] = base + e;
             a.frontier_src_row[o] = e / k;
             a.pool_draft_row[pb + e] = 1 + (a.t - 1) * k + lane;
-            s_sel[lane] = e;
             s_x[lane] = (float)exp((double)sc);                  // confidence score in [0,1]
         }
         if (lane == 0) a.pool_len[b] = base + n_cand;
     }
-    if (tid < H) s_h[tid] = a.h[(size_t)b * H + tid];
+    if (tid < H) s_h[tid] = a.t > 1 ? a.h[(size_t)b * H + tid] : 0.f;
     __syncthreads();
 
     // ---- 4. prediction model ----
@@ -155,7 +153,7 @@ __global__ void __launch_bounds__(kSelThreads) expand_select_gate_kernel(const S
             const float fg = sigmoidf_(s_pre[H + tid]);
             const float gg = tanhf(s_pre[2 * H + tid]);
             const float og = sigmoidf_(s_pre[3 * H + tid]);
-            const float cn = fg * a.c[(size_t)b * H + tid] + ig * gg;
+            const float cn = fg * (a.t > 1 ? a.c[(size_t)b * H + tid] : 0.f) + ig * gg;
             const float hn = og * tanhf(cn);
             a.c[(size_t)b * H + tid] = cn;
             a.h[(size_t)b * H + tid] = hn;
@@ -228,14 +226,17 @@ extern "C" int radar_expand_step(radar_ctx* ctx, const radar_expand_args* a, voi
     vp.k = a->k;
     vp.n_chunks = vocab_pass_plan_chunks(ctx->sm_count, a->B * a->F, a->V, &vp.chunk);
     vp.want_lse = 1;
-    vp.seq_active = a->active;
+    vp.seq_active = a->t > 1 ? a->active : nullptr;
     vp.seq_rows = nullptr;
     vp.status = ctx->d_status;
     if (vocab_pass_partial_bytes(a->B * a->F, vp.n_chunks, a->k) > a->workspace_bytes) return RADAR_ERR_WORKSPACE;
     vocab_pass_carve(a->workspace, a->B * a->F, vp.n_chunks, a->k, &vp);
 
-    RADAR_CUDA_CHECK(vocab_pass_launch(vp, stream));
-    expand_select_gate_kernel<<<a->B, kSelThreads, 0, stream>>>(sp);
+    RADAR_CUDA_CHECK(vocab_pass_launch(ctx, RADAR_K_VOCAB_EXPAND, vp, stream));
+    {
+        radar_launch_scope scope(ctx, RADAR_K_SELECT_GATE, stream);
+        expand_select_gate_kernel<<<a->B, kSelThreads, 0, stream>>>(sp);
+    }
     RADAR_CUDA_CHECK(cudaGetLastError());
     return RADAR_OK;
 }

@@ -271,18 +271,27 @@ void plan(const radar_ctx* ctx, int B, int Hq, int Hkv, int max_prefix_len, int*
 }
 
 template <typename T, int D>
-int launch(const AttnParams& P, cudaStream_t stream) {
+int launch(radar_ctx* ctx, const AttnParams& P, cudaStream_t stream) {
     const radar_attn_args& a = P.a;
     const int rblocks = (kMaxNodes * P.G + kRowsPerBlock - 1) / kRowsPerBlock;
     const size_t smem = sizeof(float) * (kRowsPerBlock * D + kTile * (D + 4) + kTile * D);
-    if (smem > 48 * 1024)
+    static bool attr_done = false;                  // once per process: not a stream operation
+    if (smem > 48 * 1024 && !attr_done) {
         RADAR_CUDA_CHECK(cudaFuncSetAttribute(tree_attn_fp32_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                               (int)smem));
+        attr_done = true;
+    }
     dim3 grid((unsigned)(rblocks * P.n_splits), (unsigned)a.Hkv, (unsigned)a.B);
-    tree_attn_fp32_kernel<T, D><<<grid, kThreads, smem, stream>>>(P);
+    {
+        radar_launch_scope scope(ctx, RADAR_K_ATTN, stream);
+        tree_attn_fp32_kernel<T, D><<<grid, kThreads, smem, stream>>>(P);
+    }
     RADAR_CUDA_CHECK(cudaGetLastError());
     const int64_t items = (int64_t)a.B * a.Hq * kMaxNodes;
-    tree_attn_combine_kernel<T, D><<<(unsigned)((items + 3) / 4), 128, 0, stream>>>(P);
+    {
+        radar_launch_scope scope(ctx, RADAR_K_ATTN_COMBINE, stream);
+        tree_attn_combine_kernel<T, D><<<(unsigned)((items + 3) / 4), 128, 0, stream>>>(P);
+    }
     RADAR_CUDA_CHECK(cudaGetLastError());
     return RADAR_OK;
 }
@@ -328,7 +337,7 @@ extern "C" int radar_tree_attention(radar_ctx* ctx, const radar_attn_args* a, vo
     P.part_o = reinterpret_cast<float*>(reinterpret_cast<char*>(a->workspace) + align_up(rec * sizeof(float2), 256));
 
     if (a->dtype == RADAR_F32) {
-        return a->d == 128 ? launch<float, 128>(P, stream) : launch<float, 64>(P, stream);
+        return a->d == 128 ? launch<float, 128>(ctx, P, stream) : launch<float, 64>(ctx, P, stream);
     }
-    return a->d == 128 ? launch<__nv_bfloat16, 128>(P, stream) : launch<__nv_bfloat16, 64>(P, stream);
+    return a->d == 128 ? launch<__nv_bfloat16, 128>(ctx, P, stream) : launch<__nv_bfloat16, 64>(ctx, P, stream);
 }

@@ -177,10 +177,16 @@ extern "C" int radar_rerank_build_tree(radar_ctx* ctx, const radar_tree_args* a,
     p.a = *a;
     p.status = ctx->d_status;
     const size_t smem = (size_t)a->pool_capacity * 6;
-    if (smem > 48 * 1024)
+    static size_t attr_smem = 48 * 1024;            // raised at most a few times per process
+    if (smem > attr_smem) {
         RADAR_CUDA_CHECK(cudaFuncSetAttribute(rerank_build_tree_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                               (int)smem));
-    rerank_build_tree_kernel<<<a->B, kThreads, smem, stream>>>(p);
+        attr_smem = smem;
+    }
+    {
+        radar_launch_scope scope(ctx, RADAR_K_TREE_BUILD, stream);
+        rerank_build_tree_kernel<<<a->B, kThreads, smem, stream>>>(p);
+    }
     RADAR_CUDA_CHECK(cudaGetLastError());
     return RADAR_OK;
 }

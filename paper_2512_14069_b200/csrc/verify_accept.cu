@@ -341,8 +341,11 @@ extern "C" int radar_verify_accept(radar_ctx* ctx, const radar_accept_args* a, v
         vp.seq_rows = a->n_nodes;
         vp.status = ctx->d_status;
         vocab_pass_carve(a->workspace, a->B * kMaxNodes, vp.n_chunks, 1, &vp);
-        RADAR_CUDA_CHECK(vocab_pass_launch(vp, stream));
-        greedy_walk_kernel<<<a->B, 64, 0, stream>>>(gp);
+        RADAR_CUDA_CHECK(vocab_pass_launch(ctx, RADAR_K_VOCAB_ACCEPT, vp, stream));
+        {
+            radar_launch_scope scope(ctx, RADAR_K_GREEDY_WALK, stream);
+            greedy_walk_kernel<<<a->B, 64, 0, stream>>>(gp);
+        }
         RADAR_CUDA_CHECK(cudaGetLastError());
         return RADAR_OK;
     }
@@ -354,8 +357,11 @@ extern "C" int radar_verify_accept(radar_ctx* ctx, const radar_accept_args* a, v
     sp.q_cache = reinterpret_cast<double*>(reinterpret_cast<char*>(a->workspace) +
                                            align_up((size_t)a->B * a->V * sizeof(double), 256));
     sp.status = ctx->d_status;
-    if (a->logits_dtype == RADAR_F32) stochastic_walk_kernel<float><<<a->B, kSThreads, 0, stream>>>(sp);
-    else stochastic_walk_kernel<__nv_bfloat16><<<a->B, kSThreads, 0, stream>>>(sp);
+    {
+        radar_launch_scope scope(ctx, RADAR_K_STOCH_WALK, stream);
+        if (a->logits_dtype == RADAR_F32) stochastic_walk_kernel<float><<<a->B, kSThreads, 0, stream>>>(sp);
+        else stochastic_walk_kernel<__nv_bfloat16><<<a->B, kSThreads, 0, stream>>>(sp);
+    }
     RADAR_CUDA_CHECK(cudaGetLastError());
     return RADAR_OK;
 }

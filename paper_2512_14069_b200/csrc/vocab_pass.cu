@@ -221,10 +221,11 @@ void vocab_pass_carve(void* ws, int rows, int n_chunks, int k, VocabPassParams* 
     p->part_s = reinterpret_cast<float*>(c);
 }
 
-cudaError_t vocab_pass_launch(const VocabPassParams& p, cudaStream_t stream) {
+cudaError_t vocab_pass_launch(radar_ctx* ctx, int kernel_id, const VocabPassParams& p, cudaStream_t stream) {
     const int rows = p.n_seq * p.F;
     const unsigned grid = (unsigned)rows * (unsigned)p.n_chunks;
     if (grid == 0) return cudaSuccess;
+    radar_launch_scope scope(ctx, kernel_id, stream);
     if (p.dtype == RADAR_F32) {
         if (p.want_lse) vocab_pass_kernel<float, true><<<grid, kThreads, 0, stream>>>(p);
         else vocab_pass_kernel<float, false><<<grid, kThreads, 0, stream>>>(p);

@@ -66,12 +66,6 @@ class SpecStep:
             setattr(self, n, t[off:off + t.numel() - 255])
 
     # ---- expansion -------------------------------------------------------------------
-    def reset(self):
-        self.active.fill_(1)
-        self.h.zero_()
-        self.c.zero_()
-        self.pool_len.zero_()
-
     def expand(self, t, draft_logits, gate, force_calls=None):
         """Draft call t (1-based) on draft_logits [B,R,V]: row 0 for t = 1, rows 1+(t-2)k.. for t >= 2."""
         k, B, V = self.k, self.B, self.V
@@ -93,8 +87,7 @@ class SpecStep:
             gate_logits=self.gate_logits[s], cont=self.cont_hist[s], workspace=self.ws_expand)
 
     def run_expansion(self, draft_logits, gate, force_calls=None):
-        self.reset()
-        for t in range(1, self.t_max + 1):
+        for t in range(1, self.t_max + 1):          # call 1 restarts the state on the device
             self.expand(t, draft_logits, gate, force_calls)
 
     # ---- tree, attention, acceptance ------------------------------------------------------
