@@ -238,6 +238,28 @@ typedef struct {
 size_t radar_accept_workspace_bytes(const radar_ctx* ctx, int B, int V, int mode);
 int radar_verify_accept(radar_ctx* ctx, const radar_accept_args* args, void* stream);
 
+/* ------------------------------------------------------------------------------------------
+ * radar_verify_accept_greedy_noalloc - greedy acceptance that needs no workspace from the caller.
+ * (The paper has no counterpart: this is a deployment variant of radar_verify_accept in greedy
+ * mode, with the same inputs, outputs and results.)
+ *
+ * For hosts that cannot allocate when they reach this call - an inference server that has handed
+ * all free device memory to its own cache pool at start-up, or a decode loop that must not take
+ * the device-wide synchronisation of cudaMalloc / cudaFree - and that have no spare buffer to pass
+ * as `workspace`.  The scratch is a fixed array of radar_noalloc_scratch_bytes() = 1 MiB inside
+ * the library image, resident on every GPU that has the library loaded until the process exits.
+ * `workspace` / `workspace_bytes` of the argument struct are ignored; `mode` must be RADAR_GREEDY.
+ *   - Sizes whose chunk records (about 16 bytes x B x 64 x chunks-per-row) exceed the array, and
+ *     stochastic mode, return RADAR_ERR_UNSUPPORTED and launch nothing.
+ *   - The call makes no cudaMalloc / cudaFree and calls no allocating routine.
+ *   - Every call on a device uses the same array, which still holds the previous call's records;
+ *     nothing needs to be cleared because each record is written before it is read within a call.
+ *     Calls that may overlap on the GPU (two streams, concurrent graph replays) race: serialise them.
+ *   - The first call on each device resolves the array's device address (ctx's device must be the
+ *     current device, otherwise RADAR_ERR_INVALID_ARG); make that first call outside stream capture. */
+size_t radar_noalloc_scratch_bytes(void);
+int radar_verify_accept_greedy_noalloc(radar_ctx* ctx, const radar_accept_args* args, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -295,3 +295,33 @@ def radar_verify_accept(ctx: Context, *, B, V, t_max, N, mode, target_logits, tr
     a.next_token, a.best_retrieve_row = _ptr(next_token, i32), _ptr(best_retrieve_row, i32)
     a.workspace, a.workspace_bytes = _ptr(workspace), workspace.numel() * workspace.element_size()
     _check("radar_verify_accept", lib().radar_verify_accept(ctx.handle, ctypes.byref(a), _stream(stream)))
+
+
+def radar_noalloc_scratch_bytes() -> int:
+    L = lib()
+    L.radar_noalloc_scratch_bytes.restype = _sz
+    return int(L.radar_noalloc_scratch_bytes())
+
+
+def radar_verify_accept_greedy_noalloc(ctx: Context, *, B, V, t_max, N, target_logits, tree_tok, tree_parent,
+                                       n_nodes, retrieve, n_leaves, accept_len, path_nodes, path_tokens, next_token,
+                                       best_retrieve_row, stream=None):
+    """Greedy acceptance without a caller workspace: for hosts that may not allocate device memory at
+    this point (all of it already belongs to their own pool, or cudaMalloc's device-wide sync is not
+    acceptable).  Scratch is a fixed 1 MiB array inside the library, shared by every call on the
+    device - do not overlap calls - and sizes that do not fit raise RadarError(-2).  The first call
+    on a device resolves the array's address; make it outside stream capture."""
+    i32 = torch.int32
+    L = lib()
+    L.radar_verify_accept_greedy_noalloc.restype = _c_int
+    L.radar_verify_accept_greedy_noalloc.argtypes = [_vp, ctypes.POINTER(AcceptArgs), _vp]
+    a = AcceptArgs()
+    a.B, a.V, a.t_max, a.N, a.mode, a.temperature = B, V, t_max, N, RADAR_GREEDY, 1.0
+    a.target_logits = _ptr(target_logits) if target_logits is not None else None
+    a.logits_dtype = dtype_code(target_logits) if target_logits is not None else RADAR_F32
+    a.tree_tok, a.tree_parent = _ptr(tree_tok, i32), _ptr(tree_parent, i32)
+    a.n_nodes, a.retrieve, a.n_leaves = _ptr(n_nodes, i32), _ptr(retrieve, i32), _ptr(n_leaves, i32)
+    a.accept_len, a.path_nodes, a.path_tokens = _ptr(accept_len, i32), _ptr(path_nodes, i32), _ptr(path_tokens, i32)
+    a.next_token, a.best_retrieve_row = _ptr(next_token, i32), _ptr(best_retrieve_row, i32)
+    _check("radar_verify_accept_greedy_noalloc",
+           L.radar_verify_accept_greedy_noalloc(ctx.handle, ctypes.byref(a), _stream(stream)))

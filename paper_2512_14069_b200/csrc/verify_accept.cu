@@ -365,3 +365,97 @@ extern "C" int radar_verify_accept(radar_ctx* ctx, const radar_accept_args* a, v
     RADAR_CUDA_CHECK(cudaGetLastError());
     return RADAR_OK;
 }
+
+// ------------------------------------------------------------------------------------------
+// Greedy acceptance for callers that cannot hand over a workspace.
+//
+// Who needs this: code that runs after its host application has frozen device memory.  A serving
+// engine typically gives every free byte of the GPU to its own KV-cache pool at start-up; from
+// then on a cudaMalloc either fails or has to be carved out of that pool by hand, and cudaMalloc /
+// cudaFree also synchronise the whole device, which a decode loop cannot afford per step.  Such a
+// caller has inputs and outputs (they are part of its own pre-planned buffers) but no spare
+// scratch to lend.  For it the scratch lives in this library's image: one fixed array in device
+// memory that exists on every GPU from the moment the library is loaded there until the process
+// exits.
+//
+// Consequences of that choice, all of which the caller must know:
+//   * the array has a fixed size (RADAR_NOALLOC_SCRATCH_BYTES = 1 MiB); a batch / vocabulary whose
+//     chunk records do not fit is refused with RADAR_ERR_UNSUPPORTED before anything is launched;
+//   * all calls on a device share it.  Two calls whose kernels may overlap on the GPU (different
+//     streams, or graphs replayed concurrently) race on it and give undefined results; calls on
+//     one stream are safe;
+//   * it keeps whatever the previous call left.  Nothing in this path needs zeroed scratch: every
+//     record that is read has been written earlier in the same call, so no clearing is done;
+//   * in host code the array's name is only a handle.  The first call on each device looks up the
+//     real device address with cudaGetSymbolAddress (that device must be current) and caches it;
+//     make that first call outside any stream capture.
+// ------------------------------------------------------------------------------------------
+#include <mutex>
+
+namespace {
+constexpr size_t kNoAllocScratchBytes = 1u << 20;
+constexpr int kNoAllocMaxDevices = 64;
+static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoAllocScratchBytes];
+std::mutex g_noalloc_mutex;
+void* g_noalloc_addr[kNoAllocMaxDevices] = {nullptr};      // per device: device address of g_noalloc_scratch
+}  // namespace
+
+extern "C" size_t radar_noalloc_scratch_bytes(void) { return kNoAllocScratchBytes; }
+
+extern "C" int radar_verify_accept_greedy_noalloc(radar_ctx* ctx, const radar_accept_args* a, void* stream_) {
+    if (!ctx || !a) return RADAR_ERR_INVALID_ARG;
+    cudaStream_t stream = reinterpret_cast<cudaStream_t>(stream_);
+    if (a->B <= 0 || a->V <= 0 || a->t_max < 1 || a->N < 1) return RADAR_ERR_INVALID_ARG;
+    if (a->mode != RADAR_GREEDY) return RADAR_ERR_UNSUPPORTED;        // the stochastic walk needs 16 * B * V bytes
+    if (a->logits_dtype != RADAR_F32 && a->logits_dtype != RADAR_BF16) return RADAR_ERR_UNSUPPORTED;
+    // size first: a request that cannot fit is refused whatever else it carries
+    int chunk = 0;
+    const int n_chunks = vocab_pass_plan_chunks(ctx->sm_count, a->B * kMaxNodes, a->V, &chunk);
+    if ((long long)a->B * kMaxNodes > 0x7fffffff / (n_chunks > 0 ? n_chunks : 1)) return RADAR_ERR_UNSUPPORTED;
+    if (vocab_pass_partial_bytes(a->B * kMaxNodes, n_chunks, 1) > kNoAllocScratchBytes) return RADAR_ERR_UNSUPPORTED;
+    if (!a->target_logits || !a->tree_tok || !a->tree_parent || !a->n_nodes || !a->retrieve || !a->n_leaves ||
+        !a->accept_len || !a->path_nodes || !a->path_tokens || !a->next_token || !a->best_retrieve_row)
+        return RADAR_ERR_INVALID_ARG;
+
+    int cur = -1;
+    RADAR_CUDA_CHECK(cudaGetDevice(&cur));
+    if (cur != ctx->device || cur < 0 || cur >= kNoAllocMaxDevices) return RADAR_ERR_INVALID_ARG;
+    void* scratch = nullptr;
+    {
+        std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+        if (g_noalloc_addr[cur] == nullptr) {
+            void* p = nullptr;
+            if (cudaGetSymbolAddress(&p, g_noalloc_scratch) != cudaSuccess || p == nullptr) return RADAR_ERR_CUDA;
+            g_noalloc_addr[cur] = p;
+        }
+        scratch = g_noalloc_addr[cur];
+    }
+
+    GreedyParams gp;
+    gp.a = *a;
+    gp.a.workspace = scratch;
+    gp.a.workspace_bytes = kNoAllocScratchBytes;
+    VocabPassParams& vp = gp.vp;
+    vp.logits = a->target_logits;
+    vp.dtype = a->logits_dtype;
+    vp.row_stride = a->V;
+    vp.seq_stride = (int64_t)kMaxNodes * a->V;
+    vp.n_seq = a->B;
+    vp.F = kMaxNodes;
+    vp.V = a->V;
+    vp.k = 1;
+    vp.n_chunks = n_chunks;
+    vp.chunk = chunk;
+    vp.want_lse = 0;
+    vp.seq_active = nullptr;
+    vp.seq_rows = a->n_nodes;
+    vp.status = ctx->d_status;
+    vocab_pass_carve(scratch, a->B * kMaxNodes, n_chunks, 1, &vp);
+    RADAR_CUDA_CHECK(vocab_pass_launch(ctx, RADAR_K_VOCAB_ACCEPT, vp, stream));
+    {
+        radar_launch_scope scope(ctx, RADAR_K_GREEDY_WALK, stream);
+        greedy_walk_kernel<<<a->B, 64, 0, stream>>>(gp);
+    }
+    RADAR_CUDA_CHECK(cudaGetLastError());
+    return RADAR_OK;
+}
