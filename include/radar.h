@@ -175,9 +175,14 @@ int radar_rerank_build_tree(radar_ctx* ctx, const radar_tree_args* args, void* s
  * [token][Hkv][d] where sequence b's tokens start at row kv_start[b] (dense caches:
  * kv_start[b] = b * Pmax; packed: the cumulative lengths).  dtype applies to Q, K, V and O;
  * accumulation is fp32.  lse (optional) [B][Hq][64] receives log sum_j exp(scale * q.k_j).
- * max_prefix_len (host) bounds prefix_len[] and sizes the launch; a larger device value
- * records RADAR_ERR_INVALID_ARG on the device status word and that sequence is skipped.
- * Limits: d in {64, 128}; Hq a multiple of Hkv.
+ * max_prefix_len (host) bounds prefix_len[] and sizes the launch; cache_rows (host) is the number
+ * of token rows allocated in Kc / Vc and bounds every read of them.  A sequence whose device-side
+ * prefix_len is negative or larger than max_prefix_len, or whose kv_start + prefix_len exceeds
+ * cache_rows, records RADAR_ERR_INVALID_ARG on the device status word and is skipped.
+ * bf16 with Hq / Hkv a power of two (<= 128) and 16-byte aligned tensors runs on the tensor cores
+ * (TMA-staged K/V tiles, tcgen05 MMA for QK^T and PV); every other case, and all of fp32, runs on
+ * an fp32 FMA kernel.
+ * Limits: d in {64, 128}; Hq a multiple of Hkv; cache_rows < 2^31.
  */
 typedef struct {
     int B, Hq, Hkv, d;
@@ -187,6 +192,7 @@ typedef struct {
     const int64_t* kv_start;            /* [B] */
     const int32_t* prefix_len;          /* [B] */
     int max_prefix_len;                 /* host value */
+    int64_t cache_rows;                 /* host value: token rows in Kc / Vc */
     const void *Kt, *Vt;
     const uint64_t* mask;               /* [B][64] */
     const int32_t* n_nodes;             /* [B] */

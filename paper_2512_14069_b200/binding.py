@@ -54,7 +54,7 @@ class AttnArgs(ctypes.Structure):
     _fields_ = [
         ("B", _c_int), ("Hq", _c_int), ("Hkv", _c_int), ("d", _c_int), ("dtype", _c_int),
         ("Q", _vp), ("Kc", _vp), ("Vc", _vp), ("kv_start", _vp), ("prefix_len", _vp), ("max_prefix_len", _c_int),
-        ("Kt", _vp), ("Vt", _vp), ("mask", _vp), ("n_nodes", _vp), ("scale", _c_f), ("O", _vp), ("lse", _vp),
+        ("cache_rows", _c_i64), ("Kt", _vp), ("Vt", _vp), ("mask", _vp), ("n_nodes", _vp), ("scale", _c_f), ("O", _vp), ("lse", _vp),
         ("workspace", _vp), ("workspace_bytes", _sz),
     ]
 
@@ -271,6 +271,7 @@ def radar_tree_attention(ctx: Context, *, B, Hq, Hkv, d, Q, Kc, Vc, kv_start, pr
     a.Q, a.Kc, a.Vc = _ptr(Q), _ptr(Kc), _ptr(Vc)
     a.kv_start, a.prefix_len = _ptr(kv_start, torch.int64), _ptr(prefix_len, torch.int32)
     a.max_prefix_len = max_prefix_len
+    a.cache_rows = 0 if Kc is None else min(Kc.numel(), Vc.numel()) // (Hkv * d)      # token rows [Hkv][d]
     a.Kt, a.Vt, a.mask, a.n_nodes = _ptr(Kt), _ptr(Vt), _ptr(mask, torch.int64), _ptr(n_nodes, torch.int32)
     a.scale, a.O, a.lse = scale, _ptr(O), _ptr(lse, torch.float32)
     a.workspace, a.workspace_bytes = _ptr(workspace), workspace.numel() * workspace.element_size()

@@ -144,6 +144,11 @@ size_t vocab_pass_partial_bytes(int rows, int n_chunks, int k);
 void vocab_pass_carve(void* ws, int rows, int n_chunks, int k, VocabPassParams* p);
 cudaError_t vocab_pass_launch(radar_ctx* ctx, int kernel_id, const VocabPassParams& p, cudaStream_t stream);
 
+// --- tensor-core tree attention (tree_attention_tc.cu) --------------------------------------
+bool tree_attn_tc_supported(const radar_attn_args* a);
+size_t tree_attn_tc_workspace_bytes(const radar_ctx* ctx, int B, int Hq, int Hkv, int d, int max_prefix_len);
+int tree_attn_tc_launch(radar_ctx* ctx, const radar_attn_args* a, cudaStream_t stream);
+
 static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 }  // namespace radar

@@ -5,6 +5,8 @@
 // serving bf16 storage) and the split-KV combine.  Work is split over (sequence, KV head,
 // block of 32 query rows, KV split); all G query heads that share a KV head are rows of the
 // same block so that a K/V tile staged in shared memory is reused G * rows times.
+#include <algorithm>
+
 #include "common.cuh"
 
 namespace radar {
@@ -303,12 +305,14 @@ using namespace radar;
 
 extern "C" size_t radar_attn_workspace_bytes(const radar_ctx* ctx, int B, int Hq, int Hkv, int d, int dtype,
                                              int max_prefix_len) {
-    (void)dtype;
     if (!ctx || B <= 0 || Hq <= 0 || Hkv <= 0 || Hq % Hkv != 0 || max_prefix_len < 0) return 0;
     int split_len, n_splits;
     plan(ctx, B, Hq, Hkv, max_prefix_len, &split_len, &n_splits);
     const size_t rec = (size_t)B * Hq * kMaxNodes * n_splits;
-    return align_up(rec * sizeof(float2), 256) + align_up(rec * d * sizeof(float), 256);
+    size_t need = align_up(rec * sizeof(float2), 256) + align_up(rec * d * sizeof(float), 256);
+    // the same buffer serves whichever kernel the call dispatches to
+    if (dtype == RADAR_BF16) need = std::max(need, tree_attn_tc_workspace_bytes(ctx, B, Hq, Hkv, d, max_prefix_len));
+    return need;
 }
 
 extern "C" int radar_tree_attention(radar_ctx* ctx, const radar_attn_args* a, void* stream_) {
@@ -323,6 +327,8 @@ extern "C" int radar_tree_attention(radar_ctx* ctx, const radar_attn_args* a, vo
         return RADAR_ERR_INVALID_ARG;
     if (a->max_prefix_len > 0 && (!a->Kc || !a->Vc)) return RADAR_ERR_INVALID_ARG;
     if ((reinterpret_cast<uintptr_t>(a->workspace) & 255) != 0) return RADAR_ERR_WORKSPACE;
+    if (a->max_prefix_len > 0 && a->cache_rows <= 0) return RADAR_ERR_INVALID_ARG;
+    if (tree_attn_tc_supported(a)) return tree_attn_tc_launch(ctx, a, stream);
 
     AttnParams P;
     P.a = *a;
