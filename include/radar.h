@@ -93,7 +93,8 @@ int radar_reset_launch_counts(radar_ctx* ctx);
  *   sequence: the incoming active, h, c and pool_len are ignored (taken as 1, 0, 0 and 0), so a
  *   step needs no separate reset.
  * A NaN logit records RADAR_ERR_NUMERIC (outputs of that sequence unspecified).
- * Limits: 1 <= k <= RADAR_MAX_K, 1 <= F <= 32, V >= k, pool_len[b] + F*k <= pool_capacity.
+ * Limits: 1 <= k <= RADAR_MAX_K, 1 <= F <= 32, V >= k, pool_len[b] + F*k <= pool_capacity;
+ * w_hh 16-byte aligned.
  */
 typedef struct {
     int B, F, V, k;

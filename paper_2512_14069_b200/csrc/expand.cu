@@ -1,32 +1,36 @@
 // radar_expand_step: vocabulary pass (vocab_pass.cu) followed by one block per sequence that
 // merges the chunk partials into each row's top-k and log-normaliser, forms the candidate
 // scores, appends them to the pool, selects the k best over all parents and runs the
-// prediction model (LSTM cell + MLP head) on their confidence scores.
+// prediction model (LSTM cell + MLP head) on their confidence scores.  The block is built for
+// latency: everything it reads from global memory is fetched in a few wide, independent batches.
 #include "common.cuh"
 
 namespace radar {
 namespace {
 
-constexpr int kSelThreads = 512;
+constexpr int kSelThreads = 1024;
 constexpr int kSelWarps = kSelThreads / 32;
+constexpr int kMergeWarps = 16;                      // warps 0..15 merge chunk records, warps 16..31 prepare the gate
 constexpr int kMaxF = 32;
+constexpr size_t kStageLimit = 96 * 1024;            // chunk records are staged in shared memory up to this size
 
 struct SelectParams {
     radar_expand_args a;
     VocabPassParams vp;
     int* status;
+    int staged;                                      // 1: the block's chunk records fit the staging area
 };
 
 __device__ __forceinline__ float sigmoidf_(float x) { return 1.f / (1.f + expf(-x)); }
 
-// y[r] = bias[r] + sum_c W[r][c] * x[c], rows distributed over warps, columns over lanes
-__device__ __forceinline__ float row_dot(const float* __restrict__ w_row, const float* x, int n, int lane) {
-    float acc = 0.f;
-    for (int c = lane; c < n; c += 32) acc = fmaf(w_row[c], x[c], acc);
-    return warp_sum(acc);
-}
+__device__ __forceinline__ void group_barrier(int id) { asm volatile("bar.sync %0, 512;" ::"r"(id) : "memory"); }
 
-__global__ void __launch_bounds__(kSelThreads) expand_select_gate_kernel(const SelectParams P) {
+// One block per sequence.  Phase 1 runs two things side by side: warps 0-15 merge the vocabulary pass's
+// chunk records into each row's top-k and log-normaliser, warps 16-31 do everything of the prediction
+// model that does not depend on this call's candidates (W_hh h + biases, weights into shared memory).
+// Phase 2 appends the candidates to the pool and selects the frontier; phase 3 finishes the LSTM cell
+// and the MLP head from shared memory only.
+__global__ void __launch_bounds__(kSelThreads, 1) expand_select_gate_kernel(const SelectParams P) {
     const radar_expand_args& a = P.a;
     const int b = blockIdx.x;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -36,54 +40,103 @@ __global__ void __launch_bounds__(kSelThreads) expand_select_gate_kernel(const S
     }
     const int F = a.F, k = a.k, H = kHidden;
     const int n_chunks = P.vp.n_chunks;
+    const int per_row = n_chunks * k;
+    const bool run_gate = a.t < a.t_max;
+
+    extern __shared__ __align__(16) unsigned char sel_smem[];
+    float* st_v = reinterpret_cast<float*>(sel_smem);                              // [F][n_chunks][k] if staged
+    int* st_i = reinterpret_cast<int*>(st_v + (P.staged ? (size_t)F * per_row : 0));
+    float* s_wih = reinterpret_cast<float*>(st_i + (P.staged ? (size_t)F * per_row : 0));   // [4H][k]
+    float* s_w1 = s_wih + 4 * H * k;                                                // [H][H + k]
 
     __shared__ double s_cand[kMaxF * RADAR_MAX_K];     // candidate scores, flat (f, j)
     __shared__ int s_ctok[kMaxF * RADAR_MAX_K];
     __shared__ float s_x[RADAR_MAX_K];                 // gate input
-    __shared__ float s_h[kHidden], s_hn[kHidden], s_pre[4 * kHidden], s_hid[kHidden];
+    __shared__ __align__(16) float s_h[kHidden];
+    __shared__ float s_hn[kHidden], s_pre[4 * kHidden], s_hid[kHidden];
+    __shared__ float s_b1[kHidden], s_w2[2 * kHidden], s_b2[2];
     __shared__ float s_y[2];
     __shared__ int s_base;
 
     if (tid == 0) s_base = a.t > 1 ? a.pool_len[b] : 0;
 
-    // ---- 1. per row: merge chunk partials -> top-k tokens, log-normaliser, candidate scores ----
-    for (int f = warp; f < F; f += kSelWarps) {
-        const size_t row = (size_t)b * F + f;
-        const float* pv = P.vp.part_v + row * n_chunks * k;
-        const int* pi = P.vp.part_i + row * n_chunks * k;
-        WarpTopList<float> top;
-        top.reset();
-        float thr = -CUDART_INF_F;
-        int thr_i = 0x7fffffff;
-        for (int c = 0; c < n_chunks; ++c) {
-            for (int e = 0; e < k; ++e) {
-                const float cv = pv[c * k + e];
-                const int ci = pi[c * k + e];
-                if (!precedes(cv, ci, thr, thr_i)) break;          // each chunk's list is sorted
-                top.insert(cv, ci);
-                thr = top.value_at(k - 1);
-                thr_i = top.index_at(k - 1);
+    if (warp < kMergeWarps) {
+        // ---- 1a. chunk records -> shared memory (coalesced), then per row: top-k, log-normaliser, scores ----
+        const size_t row0 = (size_t)b * F;
+        const float* gv = P.vp.part_v + row0 * per_row;
+        const int* gi = P.vp.part_i + row0 * per_row;
+        if (P.staged) {
+            for (int e = tid; e < F * per_row; e += kMergeWarps * 32) { st_v[e] = gv[e]; st_i[e] = gi[e]; }
+            group_barrier(2);
+        }
+        const float* pv_all = P.staged ? st_v : gv;
+        const int* pi_all = P.staged ? st_i : gi;
+        for (int f = warp; f < F; f += kMergeWarps) {
+            const size_t row = row0 + f;
+            const float* pv = pv_all + (size_t)f * per_row;
+            const int* pi = pi_all + (size_t)f * per_row;
+            // log-sum-exp over the chunks in fp64 (loads first: they overlap the merge below)
+            float mloc = -CUDART_INF_F;
+            for (int c = lane; c < n_chunks; c += 32) mloc = fmaxf(mloc, P.vp.part_m[row * n_chunks + c]);
+            WarpTopList<float> top;
+            top.reset();
+            float thr = -CUDART_INF_F;
+            int thr_i = 0x7fffffff;
+            for (int c = 0; c < n_chunks; ++c) {
+                for (int e = 0; e < k; ++e) {
+                    const float cv = pv[c * k + e];
+                    const int ci = pi[c * k + e];
+                    if (!precedes(cv, ci, thr, thr_i)) break;          // each chunk's list is sorted
+                    top.insert(cv, ci);
+                    thr = top.value_at(k - 1);
+                    thr_i = top.index_at(k - 1);
+                }
+            }
+            const float M = warp_max(mloc);
+            double sloc = 0.0;
+            for (int c = lane; c < n_chunks; c += 32) {
+                const float mc = P.vp.part_m[row * n_chunks + c];
+                if (mc > -CUDART_INF_F) sloc += (double)P.vp.part_s[row * n_chunks + c] * exp((double)mc - (double)M);
+            }
+            const double S = warp_sum(sloc);
+            const double lse = (double)M + log(S);
+            if (lane < k) {
+                const double logp = (double)top.v - lse;
+                const double sc = (double)a.parent_score[(size_t)b * F + f] + logp;
+                a.topk_tok[row * k + lane] = top.i;
+                a.topk_logp[row * k + lane] = (float)logp;
+                s_cand[f * k + lane] = sc;
+                s_ctok[f * k + lane] = top.i;
             }
         }
-        // log-sum-exp over the chunks in fp64
-        float mloc = -CUDART_INF_F;
-        for (int c = lane; c < n_chunks; c += 32) mloc = fmaxf(mloc, P.vp.part_m[row * n_chunks + c]);
-        const float M = warp_max(mloc);
-        double sloc = 0.0;
-        for (int c = lane; c < n_chunks; c += 32) {
-            const float mc = P.vp.part_m[row * n_chunks + c];
-            if (mc > -CUDART_INF_F) sloc += (double)P.vp.part_s[row * n_chunks + c] * exp((double)mc - (double)M);
+    } else if (run_gate) {
+        // ---- 1b. the part of the prediction model that only needs the previous state ----
+        const int gt = tid - kMergeWarps * 32;          // 0..511
+        const int gw = warp - kMergeWarps;              // 0..15
+        if (gt < H) s_h[gt] = a.t > 1 ? a.h[(size_t)b * H + gt] : 0.f;
+        group_barrier(3);
+        const float4 h4 = *reinterpret_cast<const float4*>(&s_h[lane * 4]);
+        constexpr int kBatch = 8;
+        for (int r0 = gw * 32; r0 < gw * 32 + 32; r0 += kBatch) {
+            float4 w[kBatch];
+#pragma unroll
+            for (int i = 0; i < kBatch; ++i)
+                w[i] = __ldg(reinterpret_cast<const float4*>(a.w_hh + (size_t)(r0 + i) * H) + lane);
+#pragma unroll
+            for (int i = 0; i < kBatch; ++i) {
+                float acc = w[i].x * h4.x;
+                acc = fmaf(w[i].y, h4.y, acc);
+                acc = fmaf(w[i].z, h4.z, acc);
+                acc = fmaf(w[i].w, h4.w, acc);
+                acc = warp_sum(acc);
+                if (lane == 0) s_pre[r0 + i] = acc + a.b_ih[r0 + i] + a.b_hh[r0 + i];
+            }
         }
-        const double S = warp_sum(sloc);
-        const double lse = (double)M + log(S);
-        if (lane < k) {
-            const double logp = (double)top.v - lse;
-            const double sc = (double)a.parent_score[(size_t)b * F + f] + logp;
-            a.topk_tok[row * k + lane] = top.i;
-            a.topk_logp[row * k + lane] = (float)logp;
-            s_cand[f * k + lane] = sc;
-            s_ctok[f * k + lane] = top.i;
-        }
+        for (int e = gt; e < 4 * H * k; e += 512) s_wih[e] = __ldg(a.w_ih + e);
+        for (int e = gt; e < H * (H + k); e += 512) s_w1[e] = __ldg(a.w1 + e);
+        if (gt < H) s_b1[gt] = a.b1[gt];
+        if (gt < 2 * H) s_w2[gt] = a.w2[gt];
+        if (gt < 2) s_b2[gt] = a.b2[gt];
     }
     __syncthreads();
     const int base = s_base;
@@ -137,15 +190,16 @@ __global__ void __launch_bounds__(kSelThreads) expand_select_gate_kernel(const S
         }
         if (lane == 0) a.pool_len[b] = base + n_cand;
     }
-    if (tid < H) s_h[tid] = a.t > 1 ? a.h[(size_t)b * H + tid] : 0.f;
     __syncthreads();
 
-    // ---- 4. prediction model ----
+    // ---- 4. prediction model, from shared memory ----
     bool cont = false;
-    if (a.t < a.t_max) {
-        for (int r = warp; r < 4 * H; r += kSelWarps) {
-            float acc = row_dot(a.w_ih + (size_t)r * k, s_x, k, lane) + row_dot(a.w_hh + (size_t)r * H, s_h, H, lane);
-            if (lane == 0) s_pre[r] = acc + a.b_ih[r] + a.b_hh[r];
+    if (run_gate) {
+        if (tid < 4 * H) {
+            float acc = s_pre[tid];
+            const float* w = s_wih + tid * k;
+            for (int j = 0; j < k; ++j) acc = fmaf(w[j], s_x[j], acc);
+            s_pre[tid] = acc;
         }
         __syncthreads();
         if (tid < H) {
@@ -161,14 +215,19 @@ __global__ void __launch_bounds__(kSelThreads) expand_select_gate_kernel(const S
         }
         __syncthreads();
         for (int r = warp; r < H; r += kSelWarps) {
-            const float* w = a.w1 + (size_t)r * (H + k);
-            float acc = row_dot(w, s_hn, H, lane) + row_dot(w + H, s_x, k, lane);
-            if (lane == 0) s_hid[r] = fmaxf(acc + a.b1[r], 0.f);
+            const float* w = s_w1 + r * (H + k);
+            float acc = 0.f;
+            for (int c = lane; c < H; c += 32) acc = fmaf(w[c], s_hn[c], acc);
+            if (lane < k) acc = fmaf(w[H + lane], s_x[lane], acc);
+            acc = warp_sum(acc);
+            if (lane == 0) s_hid[r] = fmaxf(acc + s_b1[r], 0.f);
         }
         __syncthreads();
         if (warp < 2) {
-            const float acc = row_dot(a.w2 + (size_t)warp * H, s_hid, H, lane);
-            if (lane == 0) s_y[warp] = acc + a.b2[warp];
+            float acc = 0.f;
+            for (int c = lane; c < H; c += 32) acc = fmaf(s_w2[warp * H + c], s_hid[c], acc);
+            acc = warp_sum(acc);
+            if (lane == 0) s_y[warp] = acc + s_b2[warp];
         }
         __syncthreads();
         cont = s_y[1] > s_y[0];
@@ -209,6 +268,7 @@ extern "C" int radar_expand_step(radar_ctx* ctx, const radar_expand_args* a, voi
         return RADAR_ERR_INVALID_ARG;
     if (a->t < a->t_max && (!a->w_ih || !a->w_hh || !a->b_ih || !a->b_hh || !a->w1 || !a->b1 || !a->w2 || !a->b2))
         return RADAR_ERR_INVALID_ARG;
+    if (a->t < a->t_max && (reinterpret_cast<uintptr_t>(a->w_hh) & 15) != 0) return RADAR_ERR_INVALID_ARG;
     if (a->pool_capacity < a->F * a->k) return RADAR_ERR_INVALID_ARG;
     if ((reinterpret_cast<uintptr_t>(a->workspace) & 255) != 0) return RADAR_ERR_WORKSPACE;
 
@@ -233,9 +293,19 @@ extern "C" int radar_expand_step(radar_ctx* ctx, const radar_expand_args* a, voi
     vocab_pass_carve(a->workspace, a->B * a->F, vp.n_chunks, a->k, &vp);
 
     RADAR_CUDA_CHECK(vocab_pass_launch(ctx, RADAR_K_VOCAB_EXPAND, vp, stream));
+    const size_t stage_bytes = (size_t)a->F * vp.n_chunks * a->k * 8;
+    sp.staged = stage_bytes <= kStageLimit ? 1 : 0;
+    const size_t smem = (sp.staged ? stage_bytes : 0) +
+                        sizeof(float) * ((size_t)4 * kHidden * a->k + (size_t)kHidden * (kHidden + a->k));
+    static size_t attr_smem = 0;                    // raised at most a few times per process
+    if (smem > attr_smem) {
+        RADAR_CUDA_CHECK(cudaFuncSetAttribute(expand_select_gate_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                              (int)smem));
+        attr_smem = smem;
+    }
     {
         radar_launch_scope scope(ctx, RADAR_K_SELECT_GATE, stream);
-        expand_select_gate_kernel<<<a->B, kSelThreads, 0, stream>>>(sp);
+        expand_select_gate_kernel<<<a->B, kSelThreads, smem, stream>>>(sp);
     }
     RADAR_CUDA_CHECK(cudaGetLastError());
     return RADAR_OK;

@@ -1,8 +1,14 @@
 // Vocabulary pass: one coalesced, vectorised read of every logits row produces, per
 // (row, chunk), the chunk's k best (logit, token) pairs and its (max, sum exp) pair.
-// The pass is HBM-bound: each logit is read exactly once with 16-byte loads; selection keeps
-// a sorted 32-entry list per warp (one entry per lane) that is touched only when an element
-// beats the current k-th best, which after the first few vectors is rare.
+//
+// The pass is HBM-bound, so each logit is read exactly once, with 16-byte streaming loads, and a
+// block keeps its whole chunk (16 or 32 values per thread) in registers: every load of the chunk is
+// in flight at once, and nothing is re-read from memory for the selection.  Selection is a filter,
+// not a running list: the k-th best of each warp's 32 per-thread maxima is a lower bound of the
+// chunk's k-th best value; the best such bound over the warps becomes the threshold, the few
+// register values that reach it go to a shared-memory candidate list, and their exact ranks by
+// (logit desc, token asc) are counted there.  If an adversarial chunk overflows the list, k rounds
+// of a block-wide arg-best over the registers give the same result.
 #include "common.cuh"
 
 namespace radar {
@@ -11,6 +17,8 @@ namespace {
 
 constexpr int kThreads = 256;
 constexpr int kWarps = kThreads / 32;
+constexpr int kCandCap = 1024;
+constexpr int kEmptyIdx = 0x40000000;          // empty slots sort after every real token id
 
 template <typename T> struct Vec;
 template <> struct Vec<float> {
@@ -33,42 +41,28 @@ template <> struct Vec<__nv_bfloat16> {
     }
 };
 
-struct Scan {
-    WarpTopList<float> top;
-    float thr;      // k-th best value so far (warp-uniform)
-    int thr_i;
-    float m, s;     // per-thread running max and sum of exp(x - m)
-    bool nan;
-    int k;
+__device__ __forceinline__ float fast_exp2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
 
-    __device__ __forceinline__ void init(int k_) {
-        top.reset();
-        thr = -CUDART_INF_F;
-        thr_i = 0x7fffffff;
-        m = -CUDART_INF_F;
-        s = 0.f;
-        nan = false;
-        k = k_;
+// best (value desc, index asc) pair over the warp, in every lane
+__device__ __forceinline__ void warp_best(float& v, int& i) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const float ov = __shfl_xor_sync(kFull, v, o);
+        const int oi = __shfl_xor_sync(kFull, i, o);
+        if (precedes(ov, oi, v, i)) { v = ov; i = oi; }
     }
-    // warp-collective: offer one element per lane
-    __device__ __forceinline__ void offer(float v, int idx, bool valid) {
-        const bool cand = valid && precedes(v, idx, thr, thr_i);
-        unsigned mk = __ballot_sync(kFull, cand);
-        if (mk == 0) return;
-        while (mk) {
-            const int src = __ffs(mk) - 1;
-            mk &= mk - 1;
-            top.insert(__shfl_sync(kFull, v, src), __shfl_sync(kFull, idx, src));
-        }
-        thr = top.value_at(k - 1);
-        thr_i = top.index_at(k - 1);
-    }
-};
+}
 
-template <typename T, bool WANT_LSE>
-__global__ void __launch_bounds__(kThreads) vocab_pass_kernel(const VocabPassParams p) {
+// EPT = values per thread kept in registers (a multiple of the vector width), chunk = kThreads * EPT
+template <typename T, int EPT, bool WANT_LSE>
+__global__ void __launch_bounds__(kThreads, EPT == 32 ? 3 : 4) vocab_pass_kernel(const VocabPassParams p) {
     using VT = Vec<T>;
     constexpr int N = VT::N;
+    constexpr int NV = EPT / N;
     const int row = blockIdx.x / p.n_chunks;
     const int chunk_id = blockIdx.x - row * p.n_chunks;
     const int seq = row / p.F;
@@ -80,129 +74,207 @@ __global__ void __launch_bounds__(kThreads) vocab_pass_kernel(const VocabPassPar
     const int e0 = min(chunk_id * p.chunk, p.V);
     const int e1 = min(e0 + p.chunk, p.V);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-
-    Scan sc;
-    sc.init(p.k);
+    const int k = p.k;
 
     // scalar head up to the first 16-byte boundary, vector body, scalar tail
     const uintptr_t addr = reinterpret_cast<uintptr_t>(base + e0);
     int head = (int)(((16 - (addr & 15)) & 15) / sizeof(T));
     head = min(head, e1 - e0);
     const int body0 = e0 + head;
-    const int nvec = (e1 - body0) / N;
+    const int nvec = (e1 - body0) / N;             // <= kThreads * NV because chunk == kThreads * EPT
     const int tail0 = body0 + nvec * N;
+    const int ntail = e1 - tail0;
 
-    auto scalar = [&](int idx, bool valid) {
-        float v = valid ? to_float(base[idx]) : -CUDART_INF_F;
-        if (valid) {
-            if (v != v) sc.nan = true;
-            if (WANT_LSE) {
-                if (v > sc.m) { sc.s *= __expf(sc.m - v); sc.m = v; }
-                if (sc.m > -CUDART_INF_F) sc.s += __expf(v - sc.m);
-            }
-        }
-        sc.offer(v, idx, valid);
-    };
-    if (warp == 0) {                        // head and tail are shorter than one vector
-        scalar(e0 + lane, lane < head);
-        scalar(tail0 + lane, tail0 + lane < e1);
-    }
-
+    // ---- every load of the chunk in flight ----
+    float x[NV][N];
     const T* vbase = base + body0;
-    constexpr int U = 4;                    // independent 16-byte loads in flight per thread
-    for (int j0 = 0; j0 < nvec; j0 += kThreads * U) {
-        float x[U][N];
-        bool ok[U];
 #pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const int j = j0 + u * kThreads + tid;
-            ok[u] = j < nvec;
-            if (ok[u]) VT::load(vbase + (int64_t)j * N, x[u]);
+    for (int u = 0; u < NV; ++u) {
+        const int j = tid + u * kThreads;
+        if (j < nvec) {
+            VT::load(vbase + (int64_t)j * N, x[u]);
+        } else {
+#pragma unroll
+            for (int e = 0; e < N; ++e) x[u][e] = -CUDART_INF_F;
         }
+    }
+    // head and tail (each shorter than one vector): one value for threads 0..N-1 and N..2N-1
+    float xs = -CUDART_INF_F;
+    int xs_idx = -1;
+    if (tid < head) xs_idx = e0 + tid;
+    else if (tid >= N && tid - N < ntail) xs_idx = tail0 + tid - N;
+    if (xs_idx >= 0) xs = to_float(base[xs_idx]);
+
+    // ---- per-thread best and (max, sum exp) ----
+    float bv = xs;
+    int bi = xs_idx >= 0 ? xs_idx : kEmptyIdx + tid;
+    bool nan = xs != xs;
 #pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const int j = j0 + u * kThreads + tid;
-            bool any = false;
-            if (ok[u]) {
-                float vmax = x[u][0];
+    for (int u = 0; u < NV; ++u) {
+        const int idx0 = body0 + (tid + u * kThreads) * N;
 #pragma unroll
-                for (int e = 1; e < N; ++e) vmax = fmaxf(vmax, x[u][e]);
-                bool bad = false;
+        for (int e = 0; e < N; ++e) {
+            const float v = x[u][e];
+            nan |= (v != v);
+            // a later element only wins when strictly larger: the lowest index of the maximum is kept,
+            // except against the scalar slot, whose index may be higher (tail) - handled by precedes
+            if (v > bv || (v == bv && idx0 + e < bi)) { bv = v; bi = idx0 + e; }
+        }
+    }
+    float ssum = 0.f;
+    if (WANT_LSE) {
+        if (bv > -CUDART_INF_F) {
+            const float mb = bv * 1.4426950408889634f;
 #pragma unroll
-                for (int e = 0; e < N; ++e) bad |= (x[u][e] != x[u][e]);
-                sc.nan |= bad;
-                if (WANT_LSE) {
-                    if (vmax > sc.m) { sc.s *= __expf(sc.m - vmax); sc.m = vmax; }
-                    if (sc.m > -CUDART_INF_F) {
+            for (int u = 0; u < NV; ++u)
 #pragma unroll
-                        for (int e = 0; e < N; ++e) sc.s += __expf(x[u][e] - sc.m);
-                    }
-                }
-                any = vmax >= sc.thr;
-            }
-            if (__any_sync(kFull, any)) {
-                const int idx0 = body0 + j * N;
-#pragma unroll
-                for (int e = 0; e < N; ++e) sc.offer(ok[u] ? x[u][e] : -CUDART_INF_F, idx0 + e, ok[u]);
-            }
+                for (int e = 0; e < N; ++e) ssum += fast_exp2(fmaf(x[u][e], 1.4426950408889634f, -mb));
+            if (xs_idx >= 0) ssum += fast_exp2(fmaf(xs, 1.4426950408889634f, -mb));
         }
     }
 
-    // ---- combine the warps of the block ----
-    __shared__ float sh_v[kWarps][32];
-    __shared__ int sh_i[kWarps][32];
     __shared__ float sh_m[kWarps], sh_s[kWarps];
-    __shared__ int sh_nan;
-    if (tid == 0) sh_nan = 0;
-    sh_v[warp][lane] = sc.top.v;
-    sh_i[warp][lane] = sc.top.i;
+    __shared__ float sh_tv[kWarps];
+    __shared__ int sh_ti[kWarps];
+    __shared__ int sh_nan, sh_cnt;
+    __shared__ float sh_cv[kCandCap];
+    __shared__ int sh_ci[kCandCap];
+    if (tid == 0) { sh_nan = 0; sh_cnt = 0; }
+
+    const size_t rec = (size_t)row * p.n_chunks + chunk_id;
     if (WANT_LSE) {
-        const float wm = warp_max(sc.m);
-        const float ws = warp_sum(wm > -CUDART_INF_F ? sc.s * __expf(sc.m - wm) : 0.f);
+        const float wm = warp_max(bv);
+        const float ws = warp_sum(wm > -CUDART_INF_F ? ssum * __expf(bv - wm) : 0.f);
         if (lane == 0) { sh_m[warp] = wm; sh_s[warp] = ws; }
     }
-    __syncthreads();
-    if (sc.nan) atomicOr(&sh_nan, 1);
-    __syncthreads();
-    if (warp == 0) {
-        for (int w = 1; w < kWarps; ++w) {
-            for (int e = 0; e < p.k; ++e) {
-                const float cv = sh_v[w][e];
-                const int ci = sh_i[w][e];
-                if (!precedes(cv, ci, sc.thr, sc.thr_i)) break;      // that warp's list is sorted
-                sc.top.insert(cv, ci);
-                sc.thr = sc.top.value_at(p.k - 1);
-                sc.thr_i = sc.top.index_at(p.k - 1);
+
+    if (k == 1) {
+        // ---- arg-best only ----
+        float wv = bv;
+        int wi = bi;
+        warp_best(wv, wi);
+        if (lane == 0) { sh_tv[warp] = wv; sh_ti[warp] = wi; }
+        __syncthreads();
+        if (nan) atomicOr(&sh_nan, 1);
+        __syncthreads();
+        if (warp == 0) {
+            float v = lane < kWarps ? sh_tv[lane] : -CUDART_INF_F;
+            int i = lane < kWarps ? sh_ti[lane] : 0x7fffffff;
+            warp_best(v, i);
+            if (lane == 0) {
+                p.part_v[rec] = v;
+                p.part_i[rec] = i >= kEmptyIdx ? 0x7fffffff : i;
             }
         }
-        const size_t rec = (size_t)row * p.n_chunks + chunk_id;
-        if (lane < p.k) {
-            p.part_v[rec * p.k + lane] = sc.top.v;
-            p.part_i[rec * p.k + lane] = sc.top.i;
+    } else {
+        // ---- threshold: k-th best of this warp's per-thread bests (k <= 32), best over the warps ----
+        {
+            int rank = 0;
+#pragma unroll
+            for (int l = 0; l < 32; ++l) {
+                const float ov = __shfl_sync(kFull, bv, l);
+                const int oi = __shfl_sync(kFull, bi, l);
+                rank += precedes(ov, oi, bv, bi) ? 1 : 0;
+            }
+            if (rank == k - 1) { sh_tv[warp] = bv; sh_ti[warp] = bi; }
         }
-        if (WANT_LSE && lane == 0) {
-            float M = sh_m[0];
-            for (int w = 1; w < kWarps; ++w) M = fmaxf(M, sh_m[w]);
-            float S = 0.f;
-            if (M > -CUDART_INF_F)
-                for (int w = 0; w < kWarps; ++w) S += sh_s[w] * __expf(sh_m[w] - M);
-            p.part_m[rec] = M;
-            p.part_s[rec] = S;
+        __syncthreads();
+        if (nan) atomicOr(&sh_nan, 1);
+        float tv = sh_tv[0];
+        int ti = sh_ti[0];
+#pragma unroll
+        for (int w = 1; w < kWarps; ++w)
+            if (precedes(sh_tv[w], sh_ti[w], tv, ti)) { tv = sh_tv[w]; ti = sh_ti[w]; }
+        // ---- candidates: everything that is not after the threshold pair ----
+        auto push = [&](float v, int idx) {
+            if (v > tv || (v == tv && idx <= ti)) {
+                const int slot = atomicAdd(&sh_cnt, 1);
+                if (slot < kCandCap) { sh_cv[slot] = v; sh_ci[slot] = idx; }
+            }
+        };
+#pragma unroll
+        for (int u = 0; u < NV; ++u) {
+            const int idx0 = body0 + (tid + u * kThreads) * N;
+            if (tid + u * kThreads < nvec) {
+#pragma unroll
+                for (int e = 0; e < N; ++e)
+                    if (x[u][e] >= tv) push(x[u][e], idx0 + e);
+            }
         }
-        if (lane == 0 && sh_nan) set_status(p.status, RADAR_ERR_NUMERIC);
+        if (xs_idx >= 0 && xs >= tv) push(xs, xs_idx);
+        __syncthreads();
+        const int C = sh_cnt;
+        float* out_v = p.part_v + rec * k;
+        int32_t* out_i = p.part_i + rec * k;
+        if (C <= kCandCap) {
+            for (int c = tid; c < C; c += kThreads) {
+                const float cv = sh_cv[c];
+                const int ci = sh_ci[c];
+                int rank = 0;
+                for (int j = 0; j < C; ++j) rank += precedes(sh_cv[j], sh_ci[j], cv, ci) ? 1 : 0;
+                if (rank < k) { out_v[rank] = cv; out_i[rank] = ci; }
+            }
+            for (int r = C + tid; r < k; r += kThreads) { out_v[r] = -CUDART_INF_F; out_i[r] = 0x7fffffff; }
+        } else {
+            // ---- exact fallback: k rounds of a block-wide arg-best over the registers ----
+            float pv = CUDART_INF_F;                   // previous winner: everything real comes after it
+            int pi = -1;
+            for (int r = 0; r < k; ++r) {
+                float cv = -CUDART_INF_F;
+                int ci = 0x7fffffff;
+                auto offer = [&](float v, int idx) {
+                    if (precedes(pv, pi, v, idx) && precedes(v, idx, cv, ci)) { cv = v; ci = idx; }
+                };
+#pragma unroll
+                for (int u = 0; u < NV; ++u) {
+                    const int idx0 = body0 + (tid + u * kThreads) * N;
+                    if (tid + u * kThreads < nvec) {
+#pragma unroll
+                        for (int e = 0; e < N; ++e) offer(x[u][e], idx0 + e);
+                    }
+                }
+                if (xs_idx >= 0) offer(xs, xs_idx);
+                warp_best(cv, ci);
+                __syncthreads();                        // previous round's readers are done
+                if (lane == 0) { sh_tv[warp] = cv; sh_ti[warp] = ci; }
+                __syncthreads();
+                cv = sh_tv[0];
+                ci = sh_ti[0];
+#pragma unroll
+                for (int w = 1; w < kWarps; ++w)
+                    if (precedes(sh_tv[w], sh_ti[w], cv, ci)) { cv = sh_tv[w]; ci = sh_ti[w]; }
+                if (tid == 0) { out_v[r] = cv; out_i[r] = ci; }
+                pv = cv;
+                pi = ci;
+            }
+        }
     }
+
+    if (WANT_LSE && tid == 0) {
+        float M = sh_m[0];
+        for (int w = 1; w < kWarps; ++w) M = fmaxf(M, sh_m[w]);
+        float S = 0.f;
+        if (M > -CUDART_INF_F)
+            for (int w = 0; w < kWarps; ++w) S += sh_s[w] * __expf(sh_m[w] - M);
+        p.part_m[rec] = M;
+        p.part_s[rec] = S;
+    }
+    if (tid == 0 && sh_nan) set_status(p.status, RADAR_ERR_NUMERIC);
+}
+
+template <typename T, bool WANT_LSE>
+void launch_ept(const VocabPassParams& p, unsigned grid, cudaStream_t stream) {
+    if (p.chunk / kThreads == 16) vocab_pass_kernel<T, 16, WANT_LSE><<<grid, kThreads, 0, stream>>>(p);
+    else vocab_pass_kernel<T, 32, WANT_LSE><<<grid, kThreads, 0, stream>>>(p);
 }
 
 }  // namespace
 
+// chunk is 8192 values (32 per thread, three blocks per SM), or 4096 (16 per thread, four blocks) when
+// the larger one would leave SMs without work
 int vocab_pass_plan_chunks(int sm_count, int rows, int V, int* chunk_out) {
-    const int min_chunk = 2048, max_chunk = 16384;
-    int want = (2 * sm_count + rows - 1) / rows;                 // about two blocks per SM for small inputs
-    if (want < 1) want = 1;
-    int chunk = (V + want - 1) / want;
-    if (chunk < min_chunk) chunk = min_chunk;
-    if (chunk > max_chunk) chunk = max_chunk;
-    chunk = (chunk + 255) / 256 * 256;
+    int chunk = 8192;
+    if ((long long)rows * ((V + chunk - 1) / chunk) < 3LL * sm_count) chunk = 4096;
     *chunk_out = chunk;
     return (V + chunk - 1) / chunk;
 }
@@ -227,11 +299,11 @@ cudaError_t vocab_pass_launch(radar_ctx* ctx, int kernel_id, const VocabPassPara
     if (grid == 0) return cudaSuccess;
     radar_launch_scope scope(ctx, kernel_id, stream);
     if (p.dtype == RADAR_F32) {
-        if (p.want_lse) vocab_pass_kernel<float, true><<<grid, kThreads, 0, stream>>>(p);
-        else vocab_pass_kernel<float, false><<<grid, kThreads, 0, stream>>>(p);
+        if (p.want_lse) launch_ept<float, true>(p, grid, stream);
+        else launch_ept<float, false>(p, grid, stream);
     } else {
-        if (p.want_lse) vocab_pass_kernel<__nv_bfloat16, true><<<grid, kThreads, 0, stream>>>(p);
-        else vocab_pass_kernel<__nv_bfloat16, false><<<grid, kThreads, 0, stream>>>(p);
+        if (p.want_lse) launch_ept<__nv_bfloat16, true>(p, grid, stream);
+        else launch_ept<__nv_bfloat16, false>(p, grid, stream);
     }
     return cudaGetLastError();
 }
