@@ -94,7 +94,7 @@ int radar_reset_launch_counts(radar_ctx* ctx);
  *   step needs no separate reset.
  * A NaN logit records RADAR_ERR_NUMERIC (outputs of that sequence unspecified).
  * Limits: 1 <= k <= RADAR_MAX_K, 1 <= F <= 32, V >= k, pool_len[b] + F*k <= pool_capacity;
- * w_hh 16-byte aligned.
+ * w_ih, w_hh and w1 16-byte aligned.
  */
 typedef struct {
     int B, F, V, k;

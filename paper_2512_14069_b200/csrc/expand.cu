@@ -13,6 +13,7 @@ constexpr int kSelWarps = kSelThreads / 32;
 constexpr int kMergeWarps = 16;                      // warps 0..15 merge chunk records, warps 16..31 prepare the gate
 constexpr int kMaxF = 32;
 constexpr size_t kStageLimit = 96 * 1024;            // chunk records are staged in shared memory up to this size
+constexpr int kSurvCap = 256;                        // per-row survivor list of the parallel merge
 
 struct SelectParams {
     radar_expand_args a;
@@ -24,6 +25,14 @@ struct SelectParams {
 __device__ __forceinline__ float sigmoidf_(float x) { return 1.f / (1.f + expf(-x)); }
 
 __device__ __forceinline__ void group_barrier(int id) { asm volatile("bar.sync %0, 512;" ::"r"(id) : "memory"); }
+__device__ __forceinline__ void cp_async4(void* smem, const void* gmem) {
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"((uint32_t)__cvta_generic_to_shared(smem)), "l"(gmem) : "memory");
+}
+__device__ __forceinline__ void cp_async16(void* smem, const void* gmem) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(smem)), "l"(gmem) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
+__host__ __device__ inline size_t up16(size_t x) { return (x + 15) & ~(size_t)15; }
 
 // One block per sequence.  Phase 1 runs two things side by side: warps 0-15 merge the vocabulary pass's
 // chunk records into each row's top-k and log-normaliser, warps 16-31 do everything of the prediction
@@ -44,9 +53,12 @@ __global__ void __launch_bounds__(kSelThreads, 1) expand_select_gate_kernel(cons
     const bool run_gate = a.t < a.t_max;
 
     extern __shared__ __align__(16) unsigned char sel_smem[];
+    const size_t stage_elems = P.staged ? (size_t)F * per_row : 0;
     float* st_v = reinterpret_cast<float*>(sel_smem);                              // [F][n_chunks][k] if staged
-    int* st_i = reinterpret_cast<int*>(st_v + (P.staged ? (size_t)F * per_row : 0));
-    float* s_wih = reinterpret_cast<float*>(st_i + (P.staged ? (size_t)F * per_row : 0));   // [4H][k]
+    int* st_i = reinterpret_cast<int*>(sel_smem + up16(stage_elems * 4));
+    float* sv_v = reinterpret_cast<float*>(sel_smem + 2 * up16(stage_elems * 4));   // [kMergeWarps][kSurvCap]
+    int* sv_i = reinterpret_cast<int*>(sv_v + kMergeWarps * kSurvCap);
+    float* s_wih = reinterpret_cast<float*>(sv_i + kMergeWarps * kSurvCap);         // [4H][k]
     float* s_w1 = s_wih + 4 * H * k;                                                // [H][H + k]
 
     __shared__ double s_cand[kMaxF * RADAR_MAX_K];     // candidate scores, flat (f, j)
@@ -57,6 +69,8 @@ __global__ void __launch_bounds__(kSelThreads, 1) expand_select_gate_kernel(cons
     __shared__ float s_b1[kHidden], s_w2[2 * kHidden], s_b2[2];
     __shared__ float s_y[2];
     __shared__ int s_base;
+    __shared__ float s_tv[kMergeWarps], s_rv[kMergeWarps][32];
+    __shared__ int s_ti[kMergeWarps], s_ri[kMergeWarps][32];
 
     if (tid == 0) s_base = a.t > 1 ? a.pool_len[b] : 0;
 
@@ -66,30 +80,87 @@ __global__ void __launch_bounds__(kSelThreads, 1) expand_select_gate_kernel(cons
         const float* gv = P.vp.part_v + row0 * per_row;
         const int* gi = P.vp.part_i + row0 * per_row;
         if (P.staged) {
-            for (int e = tid; e < F * per_row; e += kMergeWarps * 32) { st_v[e] = gv[e]; st_i[e] = gi[e]; }
+            for (int e = tid; e < F * per_row; e += kMergeWarps * 32) { cp_async4(st_v + e, gv + e); cp_async4(st_i + e, gi + e); }
+            cp_async_wait_all();
             group_barrier(2);
         }
-        const float* pv_all = P.staged ? st_v : gv;
-        const int* pi_all = P.staged ? st_i : gi;
         for (int f = warp; f < F; f += kMergeWarps) {
             const size_t row = row0 + f;
-            const float* pv = pv_all + (size_t)f * per_row;
-            const int* pi = pi_all + (size_t)f * per_row;
             // log-sum-exp over the chunks in fp64 (loads first: they overlap the merge below)
             float mloc = -CUDART_INF_F;
             for (int c = lane; c < n_chunks; c += 32) mloc = fmaxf(mloc, P.vp.part_m[row * n_chunks + c]);
             WarpTopList<float> top;
             top.reset();
-            float thr = -CUDART_INF_F;
-            int thr_i = 0x7fffffff;
-            for (int c = 0; c < n_chunks; ++c) {
-                for (int e = 0; e < k; ++e) {
-                    const float cv = pv[c * k + e];
-                    const int ci = pi[c * k + e];
-                    if (!precedes(cv, ci, thr, thr_i)) break;          // each chunk's list is sorted
-                    top.insert(cv, ci);
-                    thr = top.value_at(k - 1);
-                    thr_i = top.index_at(k - 1);
+            bool merged = false;
+            if (P.staged) {
+                // Parallel merge of the sorted chunk lists.  The k-th best chunk head bounds the row's k-th
+                // best from below; what is not after it survives, and survivors are ranked by counting.
+                const float* pv = st_v + (size_t)f * per_row;
+                const int* pi = st_i + (size_t)f * per_row;
+                float* lv = sv_v + warp * kSurvCap;
+                int* li = sv_i + warp * kSurvCap;
+                if (lane == 0) { s_tv[warp] = -CUDART_INF_F; s_ti[warp] = 0x7fffffff; }
+                s_rv[warp][lane] = -CUDART_INF_F;
+                s_ri[warp][lane] = 0x7fffffff;
+                __syncwarp();
+                for (int c = lane; c < n_chunks; c += 32) {
+                    const float hv = pv[c * k];
+                    const int hi = pi[c * k];
+                    int rank = 0;
+                    for (int o = 0; o < n_chunks; ++o) rank += precedes(pv[o * k], pi[o * k], hv, hi) ? 1 : 0;
+                    if (rank == k - 1) { s_tv[warp] = hv; s_ti[warp] = hi; }
+                }
+                __syncwarp();
+                const float tv = s_tv[warp];
+                const int ti = s_ti[warp];
+                int total = 0;
+                for (int c0 = 0; c0 < n_chunks; c0 += 32) {
+                    const int c = c0 + lane;
+                    int cnt = 0;
+                    if (c < n_chunks)
+                        while (cnt < k && !precedes(tv, ti, pv[c * k + cnt], pi[c * k + cnt])) ++cnt;
+                    int incl = cnt;
+#pragma unroll
+                    for (int o = 1; o < 32; o <<= 1) {
+                        const int v = __shfl_up_sync(kFull, incl, o);
+                        if (lane >= o) incl += v;
+                    }
+                    const int off = total + incl - cnt;
+                    for (int e = 0; e < cnt; ++e)
+                        if (off + e < kSurvCap) { lv[off + e] = pv[c * k + e]; li[off + e] = pi[c * k + e]; }
+                    total += __shfl_sync(kFull, incl, 31);
+                }
+                __syncwarp();
+                if (total <= kSurvCap) {
+                    for (int e = lane; e < total; e += 32) {
+                        const float cv = lv[e];
+                        const int ci = li[e];
+                        int rank = 0;
+                        for (int j = 0; j < total; ++j) rank += precedes(lv[j], li[j], cv, ci) ? 1 : 0;
+                        if (rank < k) { s_rv[warp][rank] = cv; s_ri[warp][rank] = ci; }
+                    }
+                    __syncwarp();
+                    top.v = s_rv[warp][lane];
+                    top.i = s_ri[warp][lane];
+                    merged = true;
+                }
+                __syncwarp();
+            }
+            if (!merged) {
+                // serial merge (records too large to stage, or a survivor list that overflowed)
+                const float* pv = (P.staged ? st_v : gv) + (size_t)f * per_row;
+                const int* pi = (P.staged ? st_i : gi) + (size_t)f * per_row;
+                float thr = -CUDART_INF_F;
+                int thr_i = 0x7fffffff;
+                for (int c = 0; c < n_chunks; ++c) {
+                    for (int e = 0; e < k; ++e) {
+                        const float cv = pv[c * k + e];
+                        const int ci = pi[c * k + e];
+                        if (!precedes(cv, ci, thr, thr_i)) break;          // each chunk's list is sorted
+                        top.insert(cv, ci);
+                        thr = top.value_at(k - 1);
+                        thr_i = top.index_at(k - 1);
+                    }
                 }
             }
             const float M = warp_max(mloc);
@@ -113,6 +184,8 @@ __global__ void __launch_bounds__(kSelThreads, 1) expand_select_gate_kernel(cons
         // ---- 1b. the part of the prediction model that only needs the previous state ----
         const int gt = tid - kMergeWarps * 32;          // 0..511
         const int gw = warp - kMergeWarps;              // 0..15
+        for (int e = gt; e < H * k; e += 512) cp_async16(s_wih + 4 * e, a.w_ih + 4 * e);          // 4H*k floats
+        for (int e = gt; e < H * (H + k) / 4; e += 512) cp_async16(s_w1 + 4 * e, a.w1 + 4 * e);
         if (gt < H) s_h[gt] = a.t > 1 ? a.h[(size_t)b * H + gt] : 0.f;
         group_barrier(3);
         const float4 h4 = *reinterpret_cast<const float4*>(&s_h[lane * 4]);
@@ -132,11 +205,10 @@ __global__ void __launch_bounds__(kSelThreads, 1) expand_select_gate_kernel(cons
                 if (lane == 0) s_pre[r0 + i] = acc + a.b_ih[r0 + i] + a.b_hh[r0 + i];
             }
         }
-        for (int e = gt; e < 4 * H * k; e += 512) s_wih[e] = __ldg(a.w_ih + e);
-        for (int e = gt; e < H * (H + k); e += 512) s_w1[e] = __ldg(a.w1 + e);
         if (gt < H) s_b1[gt] = a.b1[gt];
         if (gt < 2 * H) s_w2[gt] = a.w2[gt];
         if (gt < 2) s_b2[gt] = a.b2[gt];
+        cp_async_wait_all();
     }
     __syncthreads();
     const int base = s_base;
@@ -159,37 +231,22 @@ __global__ void __launch_bounds__(kSelThreads, 1) expand_select_gate_kernel(cons
     __syncthreads();      // draft_row = -1 must land before the survivors overwrite theirs
 
     // ---- 3. the k best candidates over all parents (score desc, flat index asc) ----
-    if (warp == 0) {
-        WarpTopList<double> top;
-        top.reset();
-        double thr = -CUDART_INF_F;
-        int thr_i = 0x7fffffff;
-        for (int e0 = 0; e0 < n_cand; e0 += 32) {
-            const int e = e0 + lane;
-            const bool valid = e < n_cand;
-            const double v = valid ? s_cand[e] : -CUDART_INF_F;
-            unsigned mk = __ballot_sync(kFull, valid && precedes(v, e, thr, thr_i));
-            while (mk) {
-                const int src = __ffs(mk) - 1;
-                mk &= mk - 1;
-                top.insert(__shfl_sync(kFull, v, src), e0 + src);
-            }
-            thr = top.value_at(k - 1);
-            thr_i = top.index_at(k - 1);
-        }
-        if (lane < k) {
-            const int e = top.i;
-            const float sc = (float)top.v;
-            const size_t o = (size_t)b * k + lane;
+    for (int e = tid; e < n_cand; e += kSelThreads) {
+        const double v = s_cand[e];
+        int rank = 0;
+        for (int j = 0; j < n_cand; ++j) rank += precedes(s_cand[j], j, v, e) ? 1 : 0;
+        if (rank < k) {
+            const float sc = (float)v;
+            const size_t o = (size_t)b * k + rank;
             a.frontier_tok[o] = s_ctok[e];
             a.frontier_score[o] = sc;
             a.frontier_pool_idx[o] = base + e;
             a.frontier_src_row[o] = e / k;
-            a.pool_draft_row[pb + e] = 1 + (a.t - 1) * k + lane;
-            s_x[lane] = (float)exp((double)sc);                  // confidence score in [0,1]
+            a.pool_draft_row[pb + e] = 1 + (a.t - 1) * k + rank;
+            s_x[rank] = (float)exp((double)sc);                  // confidence score in [0,1]
         }
-        if (lane == 0) a.pool_len[b] = base + n_cand;
     }
+    if (tid == 0) a.pool_len[b] = base + n_cand;
     __syncthreads();
 
     // ---- 4. prediction model, from shared memory ----
@@ -268,7 +325,9 @@ extern "C" int radar_expand_step(radar_ctx* ctx, const radar_expand_args* a, voi
         return RADAR_ERR_INVALID_ARG;
     if (a->t < a->t_max && (!a->w_ih || !a->w_hh || !a->b_ih || !a->b_hh || !a->w1 || !a->b1 || !a->w2 || !a->b2))
         return RADAR_ERR_INVALID_ARG;
-    if (a->t < a->t_max && (reinterpret_cast<uintptr_t>(a->w_hh) & 15) != 0) return RADAR_ERR_INVALID_ARG;
+    if (a->t < a->t_max && ((reinterpret_cast<uintptr_t>(a->w_hh) | reinterpret_cast<uintptr_t>(a->w_ih) |
+                             reinterpret_cast<uintptr_t>(a->w1)) & 15) != 0)
+        return RADAR_ERR_INVALID_ARG;
     if (a->pool_capacity < a->F * a->k) return RADAR_ERR_INVALID_ARG;
     if ((reinterpret_cast<uintptr_t>(a->workspace) & 255) != 0) return RADAR_ERR_WORKSPACE;
 
@@ -295,7 +354,7 @@ extern "C" int radar_expand_step(radar_ctx* ctx, const radar_expand_args* a, voi
     RADAR_CUDA_CHECK(vocab_pass_launch(ctx, RADAR_K_VOCAB_EXPAND, vp, stream));
     const size_t stage_bytes = (size_t)a->F * vp.n_chunks * a->k * 8;
     sp.staged = stage_bytes <= kStageLimit ? 1 : 0;
-    const size_t smem = (sp.staged ? stage_bytes : 0) +
+    const size_t smem = 2 * up16(sp.staged ? stage_bytes / 2 : 0) + (size_t)kMergeWarps * kSurvCap * 8 +
                         sizeof(float) * ((size_t)4 * kHidden * a->k + (size_t)kHidden * (kHidden + a->k));
     static size_t attr_smem = 0;                    // raised at most a few times per process
     if (smem > attr_smem) {

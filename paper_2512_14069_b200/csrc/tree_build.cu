@@ -1,6 +1,6 @@
-// radar_rerank_build_tree: one block per sequence ranks the pool by exact comparison counting
-// (score desc, pool index asc), keeps the best n, compacts them in pool order with a block scan
-// and derives parent rows, depths, position ids, ancestor masks, leaves and retrieve rows.
+// radar_rerank_build_tree: one block per sequence sorts the pool's (score desc, pool index asc) keys
+// with a shared-memory bitonic network, keeps the best n, compacts them in pool order with a block
+// scan and derives parent rows, depths, position ids, ancestor masks, leaves and retrieve rows.
 #include "common.cuh"
 
 namespace radar {
@@ -11,13 +11,22 @@ constexpr int kThreads = 1024;
 struct TreeParams {
     radar_tree_args a;
     int* status;
+    int n2;              // pool capacity rounded up to a power of two
 };
+
+// ascending order of this key == (score descending, pool index ascending); -0 and +0 compare equal
+__device__ __forceinline__ unsigned long long sort_key(float score, int idx) {
+    unsigned u = __float_as_uint(score == 0.f ? 0.f : score);
+    u ^= (u >> 31) ? 0xffffffffu : 0x80000000u;          // monotone map of the float order onto unsigned
+    return ((unsigned long long)(~u) << 32) | (unsigned)idx;
+}
 
 __global__ void __launch_bounds__(kThreads) rerank_build_tree_kernel(const TreeParams P) {
     const radar_tree_args& a = P.a;
     extern __shared__ unsigned char smem_raw[];
-    float* s_score = reinterpret_cast<float*>(smem_raw);                       // [C]
-    short* s_node = reinterpret_cast<short*>(smem_raw + (size_t)a.pool_capacity * 4);   // [C] tree row or 0
+    unsigned long long* s_key = reinterpret_cast<unsigned long long*>(smem_raw);        // [n2] sort keys
+    float* s_score = reinterpret_cast<float*>(smem_raw + (size_t)P.n2 * 8);              // [C]
+    short* s_node = reinterpret_cast<short*>(smem_raw + (size_t)P.n2 * 8 + (size_t)a.pool_capacity * 4);   // [C] tree row or 0
     __shared__ int s_warp_cnt[kThreads / 32];
     __shared__ int s_parent[kMaxNodes], s_depth[kMaxNodes], s_haschild[kMaxNodes], s_leaf_rank[kMaxNodes];
     __shared__ int s_nleaves;
@@ -36,22 +45,32 @@ __global__ void __launch_bounds__(kThreads) rerank_build_tree_kernel(const TreeP
     for (int i = tid; i < L; i += kThreads) s_score[i] = a.pool_score[pb + i];
     if (tid < kMaxNodes) { s_parent[tid] = -1; s_depth[tid] = 0; s_haschild[tid] = 0; }
     __syncthreads();
+    // smallest power of two that holds the live entries; the rest of the network is padding
+    int n2 = 2;
+    while (n2 < L) n2 <<= 1;
+    for (int i = tid; i < n2; i += kThreads) s_key[i] = i < L ? sort_key(s_score[i], i) : ~0ull;
+    for (int i = tid; i < L; i += kThreads) s_node[i] = 0;
+    __syncthreads();
+    for (int size = 2; size <= n2; size <<= 1) {
+        for (int stride = size >> 1; stride > 0; stride >>= 1) {
+            for (int t = tid; t < (n2 >> 1); t += kThreads) {
+                const int lo = ((t & ~(stride - 1)) << 1) | (t & (stride - 1));
+                const int hi = lo | stride;
+                const bool up = (lo & size) == 0;
+                const unsigned long long x = s_key[lo], y = s_key[hi];
+                if ((x > y) == up) { s_key[lo] = y; s_key[hi] = x; }
+            }
+            __syncthreads();
+        }
+    }
+    for (int p = tid; p < n_eff; p += kThreads) s_node[(int)(s_key[p] & 0xffffffffu)] = 1;
+    __syncthreads();
 
     // each thread owns a contiguous run of pool entries so that the scan keeps pool order
     const int per = (L + kThreads - 1) / kThreads;
     const int i0 = min(tid * per, L), i1 = min(i0 + per, L);
     int kept_cnt = 0;
-    for (int i = i0; i < i1; ++i) {
-        const float si = s_score[i];
-        int rank = 0;
-        for (int j = 0; j < L; ++j) {
-            const float sj = s_score[j];
-            rank += (sj > si || (sj == si && j < i)) ? 1 : 0;
-        }
-        const bool kept = rank < n_eff;
-        s_node[i] = kept ? 1 : 0;
-        kept_cnt += kept ? 1 : 0;
-    }
+    for (int i = i0; i < i1; ++i) kept_cnt += s_node[i];
     // exclusive scan of kept_cnt over threads
     int incl = kept_cnt;
 #pragma unroll
@@ -176,7 +195,9 @@ extern "C" int radar_rerank_build_tree(radar_ctx* ctx, const radar_tree_args* a,
     TreeParams p;
     p.a = *a;
     p.status = ctx->d_status;
-    const size_t smem = (size_t)a->pool_capacity * 6;
+    p.n2 = 2;
+    while (p.n2 < a->pool_capacity) p.n2 <<= 1;
+    const size_t smem = (size_t)p.n2 * 8 + (size_t)a->pool_capacity * 6;
     static size_t attr_smem = 48 * 1024;            // raised at most a few times per process
     if (smem > attr_smem) {
         RADAR_CUDA_CHECK(cudaFuncSetAttribute(rerank_build_tree_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,

@@ -59,7 +59,7 @@ __device__ __forceinline__ void warp_best(float& v, int& i) {
 
 // EPT = values per thread kept in registers (a multiple of the vector width), chunk = kThreads * EPT
 template <typename T, int EPT, bool WANT_LSE>
-__global__ void __launch_bounds__(kThreads, EPT == 32 ? 3 : 4) vocab_pass_kernel(const VocabPassParams p) {
+__global__ void __launch_bounds__(kThreads, WANT_LSE ? (EPT == 32 ? 3 : 4) : 5) vocab_pass_kernel(const VocabPassParams p) {
     using VT = Vec<T>;
     constexpr int N = VT::N;
     constexpr int NV = EPT / N;
@@ -148,8 +148,8 @@ __global__ void __launch_bounds__(kThreads, EPT == 32 ? 3 : 4) vocab_pass_kernel
         if (lane == 0) { sh_m[warp] = wm; sh_s[warp] = ws; }
     }
 
-    if (k == 1) {
-        // ---- arg-best only ----
+    if (!WANT_LSE || k == 1) {
+        // ---- arg-best only (the pass without the normaliser is always run with k = 1) ----
         float wv = bv;
         int wi = bi;
         warp_best(wv, wi);
@@ -297,6 +297,7 @@ cudaError_t vocab_pass_launch(radar_ctx* ctx, int kernel_id, const VocabPassPara
     const int rows = p.n_seq * p.F;
     const unsigned grid = (unsigned)rows * (unsigned)p.n_chunks;
     if (grid == 0) return cudaSuccess;
+    if (!p.want_lse && p.k != 1) return cudaErrorInvalidValue;
     radar_launch_scope scope(ctx, kernel_id, stream);
     if (p.dtype == RADAR_F32) {
         if (p.want_lse) launch_ept<float, true>(p, grid, stream);
