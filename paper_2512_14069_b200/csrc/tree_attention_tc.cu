@@ -2,25 +2,32 @@
 // with K/V tiles staged by TMA.
 //
 // Work decomposition.  All G query heads of one KV head, for all tree rows, form R = n_nodes * G
-// query rows (row r = node * G + head-in-group).  They are cut into row blocks of 128 (the MMA M
-// dimension); one CTA owns (sequence, KV head, row block, KV split) and streams its range of the
-// prefix in tiles of 128 keys, plus - in the last split - one tile holding the tree's own 64 keys.
+// query rows (row r = node * G + head-in-group), cut into row blocks of 128 (the MMA M dimension)
+// and these into pairs.  A unit is (sequence, KV head, row-block pair); it has to visit the
+// sequence's prefix in tiles of 128 keys plus one tile holding the tree's own 64 keys.  The tiles of
+// all units, weighted by their cost, are laid end to end and cut into equal ranges, one per CTA, so
+// every CTA gets about the same amount of time whatever the mix of prefix lengths and tree sizes;
+// the grid is one CTA per SM.  A CTA therefore works through a few segments (unit, tile range).  A
+// unit that falls into one CTA is normalised and written to O directly; the pieces of a unit that
+// was cut are written as fp32 partials (m, l, O) and merged by tree_attn_tc_combine_kernel.  When
+// there are several pairs per KV head, CTAs alternate between them so that they stream the same K/V
+// at the same time and all but the first read hit L2.
 //
 // Inside the CTA (10 warps):
-//   warp 8     TMA producer: Q once, then K and V tiles into two 3-slot rings (128-byte swizzle).
+//   warp 8     TMA producer: per segment the Q rows, then K and V tiles into two rings (128-byte
+//              swizzle), in the order the MMA warp consumes them.
 //   warp 9     MMA issuer (one lane): S = Q K^T into one of two tensor-memory score buffers, and
 //              O (+)= P V with P read back from tensor memory (bf16, overlaying S) and V consumed
 //              N-major straight from the row-major tile.
-//   warps 0-3  softmax group 0: tiles 0, 2, 4, ... of the CTA's range;  warps 4-7: group 1, odd tiles.
-//              One thread per query row: S row from tensor memory, prefix-boundary / ancestor-bit
-//              masking in registers, running max with lazy rescaling of the O accumulator, exp2,
-//              P back to tensor memory.  The two groups keep separate (m, l, O) and are merged
-//              through shared memory at the end, so tile t+1's QK^T and softmax overlap tile t's PV.
-// A sequence that fits one split is normalised and written to O directly; otherwise the CTA writes
-// an fp32 partial (m, l, O) that tree_attn_tc_combine_kernel merges.
-//
+//   warps 0-3 / 4-7  softmax groups 0 / 1, one thread per query row: S row from tensor memory,
+//              prefix-boundary / ancestor-bit masking in registers, running max with lazy rescaling
+//              of the O accumulator, exp2, P back to tensor memory.
+//              Unit with two live row blocks: group s owns row block s and sees every tile, so each
+//              K/V tile is loaded once for 256 query rows.  Unit with one live row block: the
+//              groups take alternate tiles with separate (m, l, O) and are merged at the end.
+//              Either way one group's softmax overlaps the other's MMAs.
 // Every mbarrier wait is bounded; a wait that runs out sets RADAR_ERR_TIMEOUT on the device status
-// word, the CTA drains, frees its tensor memory and returns.
+// word, the CTA drains without skipping any hardware barrier, frees its tensor memory and returns.
 #include <cuda.h>
 
 #include "common.cuh"
@@ -31,20 +38,35 @@ namespace {
 
 using namespace tc05;
 
-constexpr int kTcThreads = 320;
+constexpr int kTcThreads = 320;      // 8 softmax warps, TMA producer, MMA issuer
+constexpr int kProducerWarp = 8, kMmaWarp = 9;
 constexpr int kTileKeys = 128;       // keys per prefix tile
 constexpr int kTreeKeys = 64;        // keys of the tree tile (RADAR_MAX_NODES)
-constexpr int kRing = 3;
+constexpr int kPairRows = 256;       // query rows of a row-block pair (and the stride of partial records)
 constexpr float kRescaleThreshold = 8.f;   // in log2 units: P stays below 2^8
+
+// Written by every CTA of the attention kernel, read by the combine kernel.
+struct CutUnit {
+    int valid;           // 1: this CTA's last segment starts a unit that continues in the following CTAs
+    int b, g, nt;        // the unit and its number of tiles
+    int slot;            // partial slot of that first piece in this CTA (0 or 1)
+    int rows;            // live query rows of the unit
+    int w;               // cost of one of its tiles
+    long long u0;        // position of the unit's first tile in the class's space
+    long long tot;       // size of that space
+};
 
 struct TcParams {
     radar_attn_args a;
-    int G, nodes_per_rb, nrb_max;
-    int tiles_per_split, n_splits_max;
+    int G, nodes_per_rb;
+    int pair_rows;       // query rows of a class's units: 256 (two row blocks share each K/V tile) or 128
+    int n_cls;           // classes = units per KV head
+    int ncc;             // CTAs per class; grid = n_cls * ncc
     float scale_log2;
     long long cache_rows;
-    float2* part_ml;     // [B][Hq][64][n_splits_max]  (m natural-log units, l)
-    float* part_o;       // [B][Hq][64][n_splits_max][D]
+    float2* part_ml;     // [grid][2][256]     (m in natural-log units, l)
+    float* part_o;       // [grid][2][256][D]
+    CutUnit* cut;        // [grid]
     int* status;
 };
 
@@ -54,70 +76,165 @@ __device__ __forceinline__ float ex2(float x) {
     return y;
 }
 
-template <int D>
+// ---- the tile space of one class (unit index pp within a KV head) ---------------------------------
+// Positions are in cost units: a tile of a unit with two live row blocks (four MMAs) weighs kCostTwo,
+// a tile of a unit with one live row block weighs kCostOne; equal position ranges are then about
+// equal amounts of time.  A tile belongs to the CTA whose range contains the tile's start position.
+constexpr int kCostOne = 3, kCostTwo = 5;
+
+struct SeqInfo {
+    int M, Pb, nt;       // tree rows, prefix length, tiles of a unit (prefix tiles + the tree tile)
+    int rows;            // live query rows of this class's unit (0: it does not exist for this sequence)
+    int w;               // cost of one tile
+    long long kv0;
+};
+
+__device__ __forceinline__ SeqInfo seq_info(const TcParams& P, int b, int pp) {
+    const radar_attn_args& a = P.a;
+    SeqInfo s;
+    s.M = min(max(a.n_nodes[b], 0), kMaxNodes);
+    s.Pb = a.prefix_len[b];
+    s.kv0 = a.kv_start[b];
+    const bool ok = s.Pb >= 0 && s.Pb <= a.max_prefix_len && s.kv0 >= 0 && s.kv0 + s.Pb <= P.cache_rows;
+    s.rows = ok ? min(max(s.M * P.G - pp * P.pair_rows, 0), P.pair_rows) : 0;
+    s.nt = (max(s.Pb, 0) + kTileKeys - 1) / kTileKeys + 1;
+    s.w = s.rows > 128 ? kCostTwo : kCostOne;
+    return s;
+}
+__device__ __forceinline__ long long seq_cost(const TcParams& P, int b, int pp) {
+    const SeqInfo s = seq_info(P, b, pp);
+    return s.rows > 0 ? (long long)P.a.Hkv * s.nt * s.w : 0;
+}
+// number of tiles of a unit (start position U, nt tiles of cost w) that start before position x
+__device__ __forceinline__ int tiles_before(long long x, long long U, int nt, int w) {
+    if (x <= U) return 0;
+    const long long n = (x - U + w - 1) / w;
+    return n > nt ? nt : (int)n;
+}
+
+// One CTA's walk over its range [.., hi) of the class's space: segments (sequence b, KV head g, tiles [t0, t1)).
+struct Cursor {
+    int b, g, t0, t1;
+    long long U, hi;     // start position of the current unit, end of the CTA's range
+    SeqInfo s;
+    __device__ __forceinline__ bool valid() const { return t1 > t0; }
+    __device__ __forceinline__ void clip() { t1 = tiles_before(hi, U, s.nt, s.w); }
+    __device__ __forceinline__ void next_unit(const TcParams& P, int pp) {
+        U += (long long)s.nt * s.w;
+        t0 = 0;
+        if (++g == P.a.Hkv) {
+            g = 0;
+            do { ++b; if (b >= P.a.B) { t1 = 0; return; } s = seq_info(P, b, pp); } while (s.rows == 0);
+        }
+        clip();
+    }
+    __device__ __forceinline__ void next(const TcParams& P, int pp) {
+        if (t1 < s.nt) { t0 = t1; return; }                  // the range ended inside this unit
+        next_unit(P, pp);
+    }
+    __device__ __forceinline__ bool complete() const { return t0 == 0 && t1 == s.nt; }
+    __device__ __forceinline__ bool two_rb() const { return s.rows > 128; }
+};
+
+template <int D, bool TWO>
 struct Smem {
     static constexpr int kHalves = D / 64;
-    static constexpr int kQBytes = 128 * D * 2;
+    static constexpr int kQBlock = 128 * D * 2;
+    static constexpr int kQBytes = (TWO ? 2 : 1) * kQBlock;
     static constexpr int kTileBytes = kTileKeys * D * 2;
-    static constexpr int kRingBytes = kRing * kTileBytes;
-    static constexpr int kTotal = kQBytes + 2 * kRingBytes;
+    static constexpr int kRingK = 3;
+    static constexpr int kRingV = TWO ? 2 : 3;
+    static constexpr int kTotal = kQBytes + (kRingK + kRingV) * kTileBytes;
     static constexpr int kDynamic = kTotal + 1024;          // slack for the 1024-byte alignment
 };
 
-template <int D>
+// TWO: the launch may contain units with two live row blocks; decides the shared-memory layout
+template <int D, bool TWO>
 __global__ void __launch_bounds__(kTcThreads, 1)
 tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmKc,
                     const __grid_constant__ CUtensorMap tmVc, const __grid_constant__ CUtensorMap tmKt,
                     const __grid_constant__ CUtensorMap tmVt, const TcParams P) {
-    using SM = Smem<D>;
+    using SM = Smem<D, TWO>;
     constexpr int H = SM::kHalves;
+    constexpr int RK = SM::kRingK, RV = SM::kRingV;
     const radar_attn_args& a = P.a;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int rb = blockIdx.x % P.nrb_max;
-    const int split = blockIdx.x / P.nrb_max;
-    const int g = blockIdx.y, b = blockIdx.z;
+    const int pp = blockIdx.x % P.n_cls;                    // class
+    const int ci = blockIdx.x / P.n_cls;
     const int G = P.G;
-
-    // ---- which part of the problem is ours (uniform over the CTA) ----
-    const int M = min(max(a.n_nodes[b], 0), kMaxNodes);
-    const int Pb = a.prefix_len[b];
-    const long long kv0 = a.kv_start[b];
-    if (Pb < 0 || Pb > a.max_prefix_len || kv0 < 0 || kv0 + Pb > P.cache_rows) {
-        if (tid == 0) set_status(P.status, RADAR_ERR_INVALID_ARG);
-        return;
-    }
-    const int R = M * G;
-    if (rb * 128 >= R) return;
-    const int ntp_all = (Pb + kTileKeys - 1) / kTileKeys;                       // prefix tiles of the sequence
-    const int n_splits = max(1, (ntp_all + P.tiles_per_split - 1) / P.tiles_per_split);
-    if (split >= n_splits) return;
-    const int tile0 = split * P.tiles_per_split;
-    const int ntp = min(P.tiles_per_split, ntp_all - tile0);                     // prefix tiles of this CTA (may be 0)
-    const bool has_tree = split == n_splits - 1;
-    const int nt = max(ntp, 0) + (has_tree ? 1 : 0);                              // >= 1
 
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     unsigned char* sQ = smem;
     unsigned char* sK = smem + SM::kQBytes;
-    unsigned char* sV = sK + SM::kRingBytes;
-    __shared__ uint64_t bar_q, bar_kfull[kRing], bar_kempty[kRing], bar_vfull[kRing], bar_vempty[kRing];
-    __shared__ uint64_t bar_sfull[2], bar_pready[2], bar_odone[2];
+    unsigned char* sV = sK + RK * SM::kTileBytes;
+    __shared__ uint64_t bar_qfull, bar_qempty, bar_kfull[3], bar_kempty[3], bar_vfull[3], bar_vempty[3];
+    __shared__ uint64_t bar_sfull[2], bar_pready[2], bar_odone[2], bar_ofree[2];
     __shared__ uint32_t s_tmem_base;
     __shared__ int s_abort;
     __shared__ float s_xm[128], s_xl[128];
+    __shared__ long long s_range[4];     // this CTA's range [lo, hi), size of the class's space, start of its first unit
+    __shared__ int s_start[2];           // sequence and KV head of the unit that contains lo
 
-    if (tid == 0) {
-        s_abort = 0;
-        mbar_init(&bar_q, 1);
-        for (int i = 0; i < kRing; ++i) {
-            mbar_init(&bar_kfull[i], 1); mbar_init(&bar_kempty[i], 1);
-            mbar_init(&bar_vfull[i], 1); mbar_init(&bar_vempty[i], 1);
+    // ---- set-up: warp 0 finds this CTA's range while the barriers and tensor memory are prepared ----
+    if (warp == 0) {
+        long long tot = 0;
+        for (int b0 = 0; b0 < a.B; b0 += 32) {
+            const int b = b0 + lane;
+            long long sz = b < a.B ? seq_cost(P, b, pp) : 0;
+            if (pp == 0 && ci == 0 && b < a.B) {
+                const int Pb = a.prefix_len[b];
+                const long long kv0 = a.kv_start[b];
+                if (Pb < 0 || Pb > a.max_prefix_len || kv0 < 0 || kv0 + Pb > P.cache_rows) set_status(P.status, RADAR_ERR_INVALID_ARG);
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) sz += __shfl_xor_sync(kFull, sz, o);
+            tot += sz;
         }
-        for (int i = 0; i < 2; ++i) { mbar_init(&bar_sfull[i], 1); mbar_init(&bar_pready[i], 4); mbar_init(&bar_odone[i], 1); }
-        fence_barrier_init();
-    }
-    if (warp == 8) {
+        const long long lo = tot * ci / P.ncc, hi = tot * (ci + 1) / P.ncc;
+        long long cum = 0, fU = 0;
+        int fb = -1, fg = 0;
+        for (int b0 = 0; b0 < a.B && fb < 0; b0 += 32) {
+            const int b = b0 + lane;
+            const long long sz = b < a.B ? seq_cost(P, b, pp) : 0;
+            long long incl = sz;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const long long v = __shfl_up_sync(kFull, incl, o);
+                if (lane >= o) incl += v;
+            }
+            const unsigned hit = __ballot_sync(kFull, cum + incl > lo);
+            if (hit) {
+                const int src = __ffs(hit) - 1;
+                const long long before = cum + __shfl_sync(kFull, incl - sz, src);
+                fb = b0 + src;
+                const SeqInfo si = seq_info(P, fb, pp);
+                const long long unit = (long long)si.nt * si.w;
+                fg = (int)((lo - before) / unit);
+                fU = before + fg * unit;
+            }
+            cum += __shfl_sync(kFull, incl, 31);
+        }
+        if (lane == 0) {
+            s_range[0] = lo; s_range[1] = hi; s_range[2] = tot; s_range[3] = fU;
+            s_start[0] = fb; s_start[1] = fg;
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            s_abort = 0;
+            mbar_init(&bar_qfull, 1);
+            mbar_init(&bar_qempty, 1);
+            for (int i = 0; i < 3; ++i) {
+                mbar_init(&bar_kfull[i], 1); mbar_init(&bar_kempty[i], 1);
+                mbar_init(&bar_vfull[i], 1); mbar_init(&bar_vempty[i], 1);
+            }
+            for (int i = 0; i < 2; ++i) {
+                mbar_init(&bar_sfull[i], 1); mbar_init(&bar_pready[i], 4);
+                mbar_init(&bar_odone[i], 1); mbar_init(&bar_ofree[i], 4);
+            }
+            fence_barrier_init();
+        }
+    } else if (warp == kProducerWarp) {
         tmem_alloc(&s_tmem_base, 512);
         tmem_relinquish();
         if (lane == 0) {
@@ -128,107 +245,186 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
-    const uint32_t tmem = s_tmem_base;
-    // tensor-memory columns: S/P buffers at 0 and 128, O accumulators at 256 and 384
+    const uint32_t tmem = s_tmem_base;      // columns: S/P buffers at 0 and 128, O accumulators at 256 and 384
     volatile int* ab = &s_abort;
 
-    // tile t of this CTA: prefix tile (128 keys) or, last, the tree tile (64 keys)
-    auto tile_is_tree = [&](int t) { return has_tree && t == nt - 1; };
+    // first segment: the unit that contains the range's start, from its first tile starting at or after it
+    Cursor cur;
+    cur.b = s_start[0]; cur.g = s_start[1];
+    cur.hi = s_range[1];
+    cur.U = s_range[3];
+    cur.t0 = cur.t1 = 0;
+    if (cur.b >= 0) {
+        cur.s = seq_info(P, cur.b, pp);
+        cur.t0 = tiles_before(s_range[0], cur.U, cur.s.nt, cur.s.w);
+        if (cur.t0 >= cur.s.nt) cur.next_unit(P, pp);       // every tile of that unit starts before the range
+        else cur.clip();
+    }
+    if (!cur.valid()) {                                     // nothing for this CTA (uniform)
+        if (tid == 0) P.cut[blockIdx.x].valid = 0;
+        tc_fence_before_sync();
+        __syncthreads();
+        if (warp == kProducerWarp) tmem_dealloc(tmem, 512);
+        return;
+    }
 
-    if (warp == 8) {
+    if (warp == kProducerWarp) {
         // =================================== TMA producer ===================================
         if (lane == 0) {
-            mbar_arrive_expect_tx(&bar_q, SM::kQBytes);
-            for (int h = 0; h < H; ++h)
-                tma_load_3d(sQ + h * (128 * 128), &tmQ, &bar_q, h * 64, g * G, b * kMaxNodes + rb * P.nodes_per_rb);
-            auto load_tile = [&](int t, bool is_k) {
-                const int slot = t % kRing;
-                uint64_t* full = is_k ? &bar_kfull[slot] : &bar_vfull[slot];
-                uint64_t* empty = is_k ? &bar_kempty[slot] : &bar_vempty[slot];
-                unsigned char* dst = (is_k ? sK : sV) + slot * SM::kTileBytes;
-                if (!mbar_wait(empty, ((t / kRing) & 1) ^ 1, ab)) return false;
-                if (tile_is_tree(t)) {
-                    mbar_arrive_expect_tx(full, kTreeKeys * D * 2);
-                    for (int h = 0; h < H; ++h)
-                        tma_load_3d(dst + h * (kTreeKeys * 128), is_k ? &tmKt : &tmVt, full, h * 64, g, b * kMaxNodes);
-                } else {
-                    mbar_arrive_expect_tx(full, kTileKeys * D * 2);
-                    const int row = (int)(kv0 + (long long)(tile0 + t) * kTileKeys);
-                    for (int h = 0; h < H; ++h)
-                        tma_load_3d(dst + h * (kTileKeys * 128), is_k ? &tmKc : &tmVc, full, h * 64, g, row);
+            uint32_t kc = 0, vc = 0;
+            bool ok = true;
+            CutUnit cu;
+            cu.valid = 0;
+            for (uint32_t seg = 0; cur.valid(); cur.next(P, pp), ++seg) {
+                const int b = cur.b, g = cur.g, n = cur.t1 - cur.t0;
+                const bool two = TWO && cur.two_rb();
+                if (cur.t0 == 0 && cur.t1 < cur.s.nt) {          // necessarily the last segment of this CTA
+                    cu.valid = 1; cu.b = b; cu.g = g; cu.nt = cur.s.nt; cu.slot = seg == 0 ? 0 : 1;
+                    cu.rows = cur.s.rows; cu.w = cur.s.w; cu.u0 = cur.U; cu.tot = s_range[2];
                 }
-                return true;
-            };
-            // same order as the MMA warp consumes: K0, K1, then V(t), K(t+2)
-            bool ok = load_tile(0, true);
-            if (ok && nt > 1) ok = load_tile(1, true);
-            for (int t = 0; ok && t < nt; ++t) {
-                ok = load_tile(t, false);
-                if (ok && t + 2 < nt) ok = load_tile(t + 2, true);
+                ok = ok && mbar_wait(&bar_qempty, (seg & 1) ^ 1, ab);
+                if (ok) {
+                    mbar_arrive_expect_tx(&bar_qfull, two ? 2 * SM::kQBlock : SM::kQBlock);
+                    for (int q = 0; q < (two ? 2 : 1); ++q)
+                        for (int h = 0; h < H; ++h)
+                            tma_load_3d(sQ + q * SM::kQBlock + h * (128 * 128), &tmQ, &bar_qfull, h * 64, g * G,
+                                        b * kMaxNodes + (pp * (P.pair_rows / 128) + q) * P.nodes_per_rb);
+                }
+                auto load_tile = [&](int t, bool is_k) {
+                    uint32_t& cnt = is_k ? kc : vc;
+                    const int ring = is_k ? RK : RV;
+                    const int slot = cnt % ring;
+                    const uint32_t use = cnt / ring;
+                    ++cnt;
+                    uint64_t* full = is_k ? &bar_kfull[slot] : &bar_vfull[slot];
+                    uint64_t* empty = is_k ? &bar_kempty[slot] : &bar_vempty[slot];
+                    unsigned char* dst = (is_k ? sK : sV) + slot * SM::kTileBytes;
+                    if (!ok || !mbar_wait(empty, (use & 1) ^ 1, ab)) { ok = false; return; }
+                    if (t == cur.s.nt - 1) {
+                        mbar_arrive_expect_tx(full, kTreeKeys * D * 2);
+                        for (int h = 0; h < H; ++h)
+                            tma_load_3d(dst + h * (kTreeKeys * 128), is_k ? &tmKt : &tmVt, full, h * 64, g, b * kMaxNodes);
+                    } else {
+                        mbar_arrive_expect_tx(full, kTileKeys * D * 2);
+                        const int row = (int)(cur.s.kv0 + (long long)t * kTileKeys);
+                        for (int h = 0; h < H; ++h)
+                            tma_load_3d(dst + h * (kTileKeys * 128), is_k ? &tmKc : &tmVc, full, h * 64, g, row);
+                    }
+                };
+                // same order as the MMA warp consumes: the first K tile(s), then V(i), K(i + lookahead)
+                const int la = two ? 1 : 2;
+                for (int i = 0; i < la && i < n; ++i) load_tile(cur.t0 + i, true);
+                for (int i = 0; i < n; ++i) {
+                    load_tile(cur.t0 + i, false);
+                    if (i + la < n) load_tile(cur.t0 + i + la, true);
+                }
             }
+            P.cut[blockIdx.x] = cu;
         }
         __syncwarp();
-    } else if (warp == 9) {
+    } else if (warp == kMmaWarp) {
         // =================================== MMA issuer ===================================
         constexpr uint32_t idesc_s128 = idesc_bf16_f32(128, kTileKeys, false, false);
         constexpr uint32_t idesc_s64 = idesc_bf16_f32(128, kTreeKeys, false, false);
         constexpr uint32_t idesc_pv = idesc_bf16_f32(128, D, false, true);
-        bool ok = mbar_wait(&bar_q, 0, ab);
-        auto issue_s = [&](int t) {
-            const int slot = t % kRing, grp = t & 1;
-            if (!mbar_wait(&bar_kfull[slot], (t / kRing) & 1, ab)) return false;
-            tc_fence_after_sync();
-            if (lane == 0) {
-                const bool tree = tile_is_tree(t);
-                const int nk = tree ? kTreeKeys : kTileKeys;
-                const uint32_t kbase = smem_u32(sK + slot * SM::kTileBytes);
+        uint32_t kc = 0, vc = 0;                 // tiles taken from the rings
+        uint32_t sc[2] = {0, 0};                 // P tiles awaited per group
+        bool ok = true;
+        for (uint32_t seg = 0; cur.valid(); cur.next(P, pp), ++seg) {
+            const int n = cur.t1 - cur.t0;
+            const bool two = TWO && cur.two_rb();
+            const int M = cur.s.M, Pb = cur.s.Pb, nt_unit = cur.s.nt;
+            ok = ok && mbar_wait(&bar_qfull, seg & 1, ab);
+            uint32_t k_slot = 0;                  // ring slot of the K tile in use (two row blocks share it)
+            // S for local tile i into group grp's buffer; fresh_k: take the next K tile from the ring
+            auto issue_s = [&](int i, int grp, bool fresh_k, bool release_k) {
+                if (fresh_k) {
+                    k_slot = kc % RK;
+                    ok = ok && mbar_wait(&bar_kfull[k_slot], (kc / RK) & 1, ab);
+                    ++kc;
+                }
+                tc_fence_after_sync();
+                if (lane == 0 && ok) {
+                    const bool tree = cur.t0 + i == nt_unit - 1;
+                    const int nk = tree ? kTreeKeys : kTileKeys;
+                    const uint32_t kbase = smem_u32(sK + k_slot * SM::kTileBytes);
+                    const uint32_t qbase = smem_u32(sQ) + (two ? grp : 0) * SM::kQBlock;
 #pragma unroll
-                for (int kk = 0; kk < D / 16; ++kk) {
-                    const int h = kk >> 2, ko = (kk & 3) * 32;
-                    const uint64_t ad = smem_desc_sw128(smem_u32(sQ) + h * (128 * 128) + ko, 16, 1024);
-                    const uint64_t bd = smem_desc_sw128(kbase + h * (nk * 128) + ko, 16, 1024);
-                    mma_ss(tmem + grp * 128, ad, bd, tree ? idesc_s64 : idesc_s128, kk > 0);
+                    for (int kk = 0; kk < D / 16; ++kk) {
+                        const int h = kk >> 2, ko = (kk & 3) * 32;
+                        const uint64_t ad = smem_desc_sw128(qbase + h * (128 * 128) + ko, 16, 1024);
+                        const uint64_t bd = smem_desc_sw128(kbase + h * (nk * 128) + ko, 16, 1024);
+                        mma_ss(tmem + grp * 128, ad, bd, tree ? idesc_s64 : idesc_s128, kk > 0);
+                    }
+                    if (release_k) mma_commit(&bar_kempty[k_slot]);
+                    mma_commit(&bar_sfull[grp]);
                 }
-                mma_commit(&bar_kempty[slot]);
-                mma_commit(&bar_sfull[grp]);
-            }
-            __syncwarp();
-            return true;
-        };
-        if (ok) ok = issue_s(0);
-        if (ok && nt > 1) ok = issue_s(1);
-        for (int t = 0; ok && t < nt; ++t) {
-            const int slot = t % kRing, grp = t & 1, j = t >> 1;
-            if (!mbar_wait(&bar_pready[grp], j & 1, ab)) { ok = false; break; }
-            if (!mbar_wait(&bar_vfull[slot], (t / kRing) & 1, ab)) { ok = false; break; }
-            tc_fence_after_sync();
-            const bool tree = tile_is_tree(t);
-            const int nk = tree ? kTreeKeys : kTileKeys;
-            const int valid = tree ? M : min(kTileKeys, Pb - (tile0 + t) * kTileKeys);
-            const int ksteps = (valid + 15) >> 4;
-            unsigned char* vtile = sV + slot * SM::kTileBytes;
-            if (valid < ksteps * 16) {
-                // rows past the last live key are multiplied by P = 0; they must not hold NaN/Inf bit patterns
-                const int nrows = ksteps * 16 - valid;
-                for (int e = lane; e < nrows * 8 * H; e += 32) {
-                    const int h = e / (nrows * 8), rem = e % (nrows * 8);
-                    const int r = valid + rem / 8, c = rem % 8;
-                    *reinterpret_cast<uint4*>(vtile + h * (nk * 128) + r * 128 + c * 16) = make_uint4(0, 0, 0, 0);
-                }
-                fence_proxy_async_smem();
                 __syncwarp();
-            }
-            if (lane == 0) {
-                const uint32_t vbase = smem_u32(vtile);
-                for (int kk = 0; kk < ksteps; ++kk) {
-                    const uint64_t bd = smem_desc_sw128(vbase + kk * 2048, nk * 128, 1024);
-                    mma_ts(tmem + 256 + grp * 128, tmem + grp * 128 + kk * 8, bd, idesc_pv, (j > 0) || (kk > 0));
+            };
+            uint32_t v_slot = 0;
+            // O[grp] (+)= P V for local tile i; fresh_v: take the next V tile; wait_free: first PV of the segment;
+            // fresh_acc: first PV of this group in the segment (overwrites the accumulator)
+            auto issue_pv = [&](int i, int grp, bool fresh_v, bool release_v, bool wait_free, bool fresh_acc, bool last) {
+                ok = ok && mbar_wait(&bar_pready[grp], sc[grp] & 1, ab);
+                ++sc[grp];
+                const bool tree = cur.t0 + i == nt_unit - 1;
+                const int nk = tree ? kTreeKeys : kTileKeys;
+                const int valid = tree ? M : min(kTileKeys, Pb - (cur.t0 + i) * kTileKeys);
+                const int ksteps = (valid + 15) >> 4;
+                if (fresh_v) {
+                    v_slot = vc % RV;
+                    ok = ok && mbar_wait(&bar_vfull[v_slot], (vc / RV) & 1, ab);
+                    ++vc;
+                    if (ok && valid < ksteps * 16) {
+                        // rows past the last live key meet P = 0; they must not hold NaN/Inf bit patterns
+                        unsigned char* vtile = sV + v_slot * SM::kTileBytes;
+                        const int nrows = ksteps * 16 - valid;
+                        for (int e = lane; e < nrows * 8 * H; e += 32) {
+                            const int h = e / (nrows * 8), rem = e % (nrows * 8);
+                            const int r = valid + rem / 8, c = rem % 8;
+                            *reinterpret_cast<uint4*>(vtile + h * (nk * 128) + r * 128 + c * 16) = make_uint4(0, 0, 0, 0);
+                        }
+                        fence_proxy_async_smem();
+                        __syncwarp();
+                    }
                 }
-                mma_commit(&bar_vempty[slot]);
-                if (t + 2 >= nt) mma_commit(&bar_odone[grp]);       // this group's last tile
+                if (wait_free) {                  // the previous segment's epilogue has read both accumulators
+                    ok = ok && mbar_wait(&bar_ofree[0], (seg & 1) ^ 1, ab);
+                    ok = ok && mbar_wait(&bar_ofree[1], (seg & 1) ^ 1, ab);
+                }
+                tc_fence_after_sync();
+                if (lane == 0 && ok) {
+                    const uint32_t vbase = smem_u32(sV + v_slot * SM::kTileBytes);
+                    for (int kk = 0; kk < ksteps; ++kk) {
+                        const uint64_t bd = smem_desc_sw128(vbase + kk * 2048, nk * 128, 1024);
+                        mma_ts(tmem + 256 + grp * 128, tmem + grp * 128 + kk * 8, bd, idesc_pv, !fresh_acc || kk > 0);
+                    }
+                    if (release_v) mma_commit(&bar_vempty[v_slot]);
+                    if (last) mma_commit(&bar_odone[grp]);
+                }
+                __syncwarp();
+            };
+            if (two) {
+                // both groups see every tile: S0(i) S1(i) share K(i), PV0(i) PV1(i) share V(i)
+                issue_s(0, 0, true, false);
+                issue_s(0, 1, false, true);
+                for (int i = 0; i < n; ++i) {
+                    issue_pv(i, 0, true, false, i == 0, i == 0, i == n - 1);
+                    if (i + 1 < n) issue_s(i + 1, 0, true, false);
+                    issue_pv(i, 1, false, true, false, i == 0, i == n - 1);
+                    if (i + 1 < n) issue_s(i + 1, 1, false, true);
+                }
+            } else {
+                // one live row block: the groups take alternate tiles
+                issue_s(0, 0, true, true);
+                if (n > 1) issue_s(1, 1, true, true);
+                for (int i = 0; i < n; ++i) {
+                    issue_pv(i, i & 1, true, true, i == 0, i < 2, i + 2 >= n);
+                    if (i + 2 < n) issue_s(i + 2, i & 1, true, true);
+                }
             }
+            if (lane == 0 && ok) mma_commit(&bar_qempty);     // every S of this segment has read Q
             __syncwarp();
-            if (t + 2 < nt) ok = issue_s(t + 2);
         }
     } else {
         // =================================== softmax groups ===================================
@@ -237,182 +433,199 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
         const uint32_t tS = tmem + grp * 128 + lane_addr;
         const uint32_t tO = tmem + 256 + grp * 128 + lane_addr;
-        const int r_glob = rb * 128 + row;
-        const int node = r_glob / G;
-        const int hq = g * G + r_glob % G;
-        const bool row_live = r_glob < R;
-        const unsigned long long live_bits = M >= 64 ? ~0ull : ((1ull << M) - 1ull);
-        const unsigned long long mask_bits = row_live ? (a.mask[(int64_t)b * kMaxNodes + node] & live_bits) : 0ull;
-        const int n_my = (nt - grp + 1) >> 1;
-        float m_run = -CUDART_INF_F, l_run = 0.f;
+        const uint32_t tO_other = tmem + 256 + (grp ^ 1) * 128 + lane_addr;
+        uint32_t sc = 0, oc = 0;                 // S tiles and accumulators this group has waited for
         bool ok = true;
+        for (uint32_t seg = 0; cur.valid(); cur.next(P, pp), ++seg) {
+            const int b = cur.b, g = cur.g, n = cur.t1 - cur.t0;
+            const bool two = TWO && cur.two_rb();
+            const int M = cur.s.M, Pb = cur.s.Pb, nt_unit = cur.s.nt;
+            const int prow = (two ? grp * 128 : 0) + row;        // row within the unit
+            const int r_glob = pp * P.pair_rows + prow;
+            const int node = r_glob / G;
+            const int hq = g * G + r_glob % G;
+            const bool row_live = prow < cur.s.rows;
+            const unsigned long long live_bits = M >= 64 ? ~0ull : ((1ull << M) - 1ull);
+            const unsigned long long mask_bits = row_live ? (a.mask[(int64_t)b * kMaxNodes + node] & live_bits) : 0ull;
+            const int n_my = two ? n : (n - grp + 1) >> 1;
+            float m_run = -CUDART_INF_F, l_run = 0.f;
 
-        for (int j = 0; j < n_my && ok; ++j) {
-            const int t = 2 * j + grp;
-            if (!mbar_wait(&bar_sfull[grp], j & 1, ab)) { ok = false; break; }
-            tc_fence_after_sync();
-            const bool tree = tile_is_tree(t);
-            const int nchunks = tree ? kTreeKeys / 32 : kTileKeys / 32;
-            uint32_t sv[4][32];
-#pragma unroll
-            for (int c = 0; c < 4; ++c)
-                if (c < nchunks) tmem_ld32(tS + c * 32, sv[c]);
-            tmem_wait_ld();
-            // ---- masking ----
-            if (tree) {
-#pragma unroll
-                for (int c = 0; c < 2; ++c)
-#pragma unroll
-                    for (int i = 0; i < 32; ++i)
-                        if (!((mask_bits >> (c * 32 + i)) & 1ull)) sv[c][i] = 0xff800000u;     // -inf
-            } else {
-                const int valid = min(kTileKeys, Pb - (tile0 + t) * kTileKeys);
-                if (valid < kTileKeys) {
+            for (int j = 0; j < n_my; ++j) {
+                const int i = two ? j : 2 * j + grp;             // local tile index
+                const int t = cur.t0 + i;
+                ok = __all_sync(kFull, ok && mbar_wait(&bar_sfull[grp], sc & 1, ab));    // warp-uniform: guards .aligned ops
+                ++sc;
+                tc_fence_after_sync();
+                if (ok) {
+                    const bool tree = t == nt_unit - 1;
+                    const int nchunks = tree ? kTreeKeys / 32 : kTileKeys / 32;
+                    uint32_t sv[4][32];
 #pragma unroll
                     for (int c = 0; c < 4; ++c)
+                        if (c < nchunks) tmem_ld32(tS + c * 32, sv[c]);
+                    tmem_wait_ld();
+                    // ---- masking ----
+                    if (tree) {
 #pragma unroll
-                        for (int i = 0; i < 32; ++i)
-                            if (c * 32 + i >= valid) sv[c][i] = 0xff800000u;
-                }
-            }
-            // ---- running max (log2 units), lazy rescale decision ----
-            float mx = -CUDART_INF_F;
+                        for (int c = 0; c < 2; ++c)
 #pragma unroll
-            for (int c = 0; c < 4; ++c)
-                if (c < nchunks)
+                            for (int e = 0; e < 32; ++e)
+                                if (!((mask_bits >> (c * 32 + e)) & 1ull)) sv[c][e] = 0xff800000u;     // -inf
+                    } else {
+                        const int valid = min(kTileKeys, Pb - t * kTileKeys);
+                        if (valid < kTileKeys) {
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) mx = fmaxf(mx, __uint_as_float(sv[c][i]));
-            const float m_tile = mx * P.scale_log2;
-            float factor = 1.f;
-            if (j == 0) {
-                m_run = m_tile;
-            } else if (m_tile > m_run + kRescaleThreshold) {
-                factor = ex2(m_run - m_tile);               // m_run may be -inf: factor 0 clears O and l
-                m_run = m_tile;
-            }
-            const float m_use = m_run == -CUDART_INF_F ? 0.f : m_run;
-            // ---- P = exp2(s * scale - m), row sum, bf16 pairs back to tensor memory (over S) ----
-            float lsum = 0.f;
+                            for (int c = 0; c < 4; ++c)
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                if (c < nchunks) {
-                    uint32_t pk[16];
-#pragma unroll
-                    for (int i = 0; i < 16; ++i) {
-                        const float p0 = ex2(fmaf(__uint_as_float(sv[c][2 * i]), P.scale_log2, -m_use));
-                        const float p1 = ex2(fmaf(__uint_as_float(sv[c][2 * i + 1]), P.scale_log2, -m_use));
-                        lsum += p0 + p1;
-                        const __nv_bfloat162 v = __floats2bfloat162_rn(p0, p1);
-                        pk[i] = *reinterpret_cast<const uint32_t*>(&v);
+                                for (int e = 0; e < 32; ++e)
+                                    if (c * 32 + e >= valid) sv[c][e] = 0xff800000u;
+                        }
                     }
-                    tmem_st16(tS + c * 16, pk);
-                }
-            }
-            l_run = l_run * factor + lsum;
-            // ---- rescale the accumulator when some row of this warp moved its reference max ----
-            if (j > 0 && __any_sync(kFull, factor != 1.f)) {
+                    // ---- running max (log2 units), lazy rescale decision ----
+                    float mxa[4] = {-CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F};   // short dependency chains
 #pragma unroll
-                for (int c = 0; c < D / 32; ++c) {
-                    uint32_t o[32];
-                    tmem_ld32(tO + c * 32, o);
-                    tmem_wait_ld();
+                    for (int c = 0; c < 4; ++c)
+                        if (c < nchunks)
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * factor);
-                    tmem_st32(tO + c * 32, o);
+                            for (int e = 0; e < 32; ++e) mxa[e & 3] = fmaxf(mxa[e & 3], __uint_as_float(sv[c][e]));
+                    const float mx = fmaxf(fmaxf(mxa[0], mxa[1]), fmaxf(mxa[2], mxa[3]));
+                    const float m_tile = mx * P.scale_log2;
+                    float factor = 1.f;
+                    if (j == 0) {
+                        m_run = m_tile;
+                    } else if (m_tile > m_run + kRescaleThreshold) {
+                        factor = ex2(m_run - m_tile);           // m_run may be -inf: factor 0 clears O and l
+                        m_run = m_tile;
+                    }
+                    const float m_use = m_run == -CUDART_INF_F ? 0.f : m_run;
+                    // ---- P = exp2(s * scale - m), row sum, bf16 pairs back to tensor memory (over S) ----
+                    float ls[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        if (c < nchunks) {
+                            uint32_t pk[16];
+#pragma unroll
+                            for (int e = 0; e < 16; ++e) {
+                                const float p0 = ex2(fmaf(__uint_as_float(sv[c][2 * e]), P.scale_log2, -m_use));
+                                const float p1 = ex2(fmaf(__uint_as_float(sv[c][2 * e + 1]), P.scale_log2, -m_use));
+                                ls[e & 3] += p0 + p1;
+                                const __nv_bfloat162 v = __floats2bfloat162_rn(p0, p1);
+                                pk[e] = *reinterpret_cast<const uint32_t*>(&v);
+                            }
+                            tmem_st16(tS + c * 16, pk);
+                        }
+                    }
+                    l_run = l_run * factor + ((ls[0] + ls[1]) + (ls[2] + ls[3]));
+                    // ---- rescale the accumulator when some row of this warp moved its reference max ----
+                    if (j > 0 && __any_sync(kFull, factor != 1.f)) {
+#pragma unroll
+                        for (int c = 0; c < D / 32; ++c) {
+                            uint32_t o[32];
+                            tmem_ld32(tO + c * 32, o);
+                            tmem_wait_ld();
+#pragma unroll
+                            for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * factor);
+                            tmem_st32(tO + c * 32, o);
+                        }
+                    }
+                    tmem_wait_st();
                 }
+                tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&bar_pready[grp]);
             }
-            tmem_wait_st();
-            tc_fence_before_sync();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&bar_pready[grp]);
-        }
 
-        // ---- epilogue: merge the two groups, then write the final rows or the split's partial ----
-        if (ok && n_my > 0) ok = mbar_wait(&bar_odone[grp], 0, ab);
-        tc_fence_after_sync();
-        float* xo = reinterpret_cast<float*>(sK);            // [D][128] exchange buffer (rings are idle by now)
-        if (grp == 1) {
-            if (ok && n_my > 0) {
+            // ---- epilogue of the segment ----
+            if (n_my > 0) {
+                ok = __all_sync(kFull, ok && mbar_wait(&bar_odone[grp], oc & 1, ab));
+                ++oc;
+            }
+            tc_fence_after_sync();
+            const bool final_rows = cur.complete();
+            const int slot = seg == 0 ? 0 : 1;                   // a CTA has at most a cut first and a cut last segment
+            const int64_t rec = ((int64_t)blockIdx.x * 2 + slot) * kPairRows + prow;
+            float m_out = m_run, l_out = l_run, w0 = 1.f, w1 = 0.f;
+            bool writer = true, merge_any = false;
+            if (!two) {
+                // group 0 merges group 1's accumulator, which sits in the same tensor-memory lanes
+                if (grp == 1) { s_xm[row] = n_my > 0 ? m_run : -CUDART_INF_F; s_xl[row] = l_run; }
+                asm volatile("bar.sync 1, 256;" ::: "memory");
+                writer = grp == 0;
+                if (writer) {
+                    const float m1 = s_xm[row], l1 = s_xl[row];
+                    const bool merge = m1 != -CUDART_INF_F;
+                    m_out = fmaxf(m_run, m1);
+                    const float ms = m_out == -CUDART_INF_F ? 0.f : m_out;
+                    w0 = ex2(m_run - ms);                        // exp2(-inf) = 0
+                    w1 = ex2(m1 - ms);
+                    l_out = l_run * w0 + l1 * w1;
+                    merge_any = __any_sync(kFull, merge);        // rows that do not merge carry w1 = 0
+                }
+            }
+            if (writer && ok) {
+                const float m_safe = m_out == -CUDART_INF_F ? 0.f : m_out;
+                const float inv = final_rows ? 1.f / l_out : 1.f;
+                const int64_t out_row = ((int64_t)b * kMaxNodes + node) * a.Hq + hq;
 #pragma unroll
                 for (int c = 0; c < D / 32; ++c) {
                     uint32_t o[32];
                     tmem_ld32(tO + c * 32, o);
                     tmem_wait_ld();
+                    float v[32];
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) xo[(c * 32 + i) * 128 + row] = __uint_as_float(o[i]);
-                }
-                s_xm[row] = m_run;
-                s_xl[row] = l_run;
-            } else {
-                s_xm[row] = -CUDART_INF_F;
-                s_xl[row] = 0.f;
-            }
-        }
-        asm volatile("bar.sync 1, 256;" ::: "memory");
-        if (grp == 0 && ok) {
-            const float m1 = s_xm[row], l1 = s_xl[row];
-            const float m = fmaxf(m_run, m1);
-            const float m_safe = m == -CUDART_INF_F ? 0.f : m;
-            const float w0 = ex2(m_run - m_safe), w1 = ex2(m1 - m_safe);      // exp2(-inf) = 0
-            const float l = l_run * w0 + l1 * w1;
-            const bool merge = m1 != -CUDART_INF_F;
-            const bool final_rows = n_splits == 1;
-            const float inv = final_rows ? 1.f / l : 1.f;
-            const int64_t out_row = ((int64_t)b * kMaxNodes + node) * a.Hq + hq;
-            const int64_t rec = (((int64_t)b * a.Hq + hq) * kMaxNodes + node) * P.n_splits_max + split;
+                    for (int e = 0; e < 32; ++e) v[e] = __uint_as_float(o[e]) * w0;
+                    if (merge_any) {
+                        tmem_ld32(tO_other + c * 32, o);
+                        tmem_wait_ld();
 #pragma unroll
-            for (int c = 0; c < D / 32; ++c) {
-                uint32_t o[32];
-                tmem_ld32(tO + c * 32, o);
-                tmem_wait_ld();
-                float v[32];
+                        for (int e = 0; e < 32; ++e) v[e] = fmaf(__uint_as_float(o[e]), w1, v[e]);
+                    }
+                    if (row_live) {
+                        if (final_rows) {
+                            __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(a.O) + out_row * D + c * 32;
 #pragma unroll
-                for (int i = 0; i < 32; ++i) {
-                    v[i] = __uint_as_float(o[i]) * w0;
-                    if (merge) v[i] = fmaf(xo[(c * 32 + i) * 128 + row], w1, v[i]);
-                    v[i] *= inv;
+                            for (int q = 0; q < 4; ++q) {
+                                uint32_t w[4];
+#pragma unroll
+                                for (int e = 0; e < 4; ++e) {
+                                    const __nv_bfloat162 t2 = __floats2bfloat162_rn(v[q * 8 + 2 * e] * inv, v[q * 8 + 2 * e + 1] * inv);
+                                    w[e] = *reinterpret_cast<const uint32_t*>(&t2);
+                                }
+                                *reinterpret_cast<uint4*>(dst + q * 8) = make_uint4(w[0], w[1], w[2], w[3]);
+                            }
+                        } else {
+                            float* dst = P.part_o + rec * D + c * 32;
+#pragma unroll
+                            for (int q = 0; q < 8; ++q)
+                                *reinterpret_cast<float4*>(dst + q * 4) = make_float4(v[q * 4], v[q * 4 + 1], v[q * 4 + 2], v[q * 4 + 3]);
+                        }
+                    }
                 }
                 if (row_live) {
+                    const float m_nat = m_safe * 0.6931471805599453f;
                     if (final_rows) {
-                        __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(a.O) + out_row * D + c * 32;
-#pragma unroll
-                        for (int q = 0; q < 4; ++q) {
-                            uint32_t w[4];
-#pragma unroll
-                            for (int i = 0; i < 4; ++i) {
-                                const __nv_bfloat162 t2 = __floats2bfloat162_rn(v[q * 8 + 2 * i], v[q * 8 + 2 * i + 1]);
-                                w[i] = *reinterpret_cast<const uint32_t*>(&t2);
-                            }
-                            *reinterpret_cast<uint4*>(dst + q * 8) = make_uint4(w[0], w[1], w[2], w[3]);
-                        }
+                        if (a.lse != nullptr) a.lse[((int64_t)b * a.Hq + hq) * kMaxNodes + node] = m_nat + logf(l_out);
                     } else {
-                        float* dst = P.part_o + rec * D + c * 32;
-#pragma unroll
-                        for (int q = 0; q < 8; ++q)
-                            *reinterpret_cast<float4*>(dst + q * 4) = make_float4(v[q * 4], v[q * 4 + 1], v[q * 4 + 2], v[q * 4 + 3]);
+                        P.part_ml[rec] = make_float2(m_out == -CUDART_INF_F ? -CUDART_INF_F : m_nat, l_out);
                     }
                 }
             }
-            if (row_live) {
-                const float m_nat = m_safe * 0.6931471805599453f;
-                if (final_rows) {
-                    if (a.lse != nullptr) a.lse[((int64_t)b * a.Hq + hq) * kMaxNodes + node] = m_nat + logf(l);
-                } else {
-                    P.part_ml[rec] = make_float2(m == -CUDART_INF_F ? -CUDART_INF_F : m_nat, l);
-                }
-            }
+            if (!two) asm volatile("bar.sync 2, 256;" ::: "memory");   // group 1's accumulator and (m, l) have been read
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&bar_ofree[grp]);
         }
     }
 
     // ---- teardown ----
     tc_fence_before_sync();
     __syncthreads();
-    if (warp == 8) {
+    if (warp == kProducerWarp) {
         if (s_abort) {
             // let loads that are still in flight land before the CTA's shared memory is released
             if (lane == 0) {
                 int dummy = 0;
-                for (int i = 0; i < kRing; ++i) {
+                for (int i = 0; i < 3; ++i) {
                     mbar_wait(&bar_kfull[i], 0, &dummy, 1u << 12);
                     mbar_wait(&bar_vfull[i], 0, &dummy, 1u << 12);
                 }
@@ -424,42 +637,61 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     }
 }
 
-// one warp per (sequence, query head, tree row) of a sequence that was split: merge the partials
+// Merges the pieces of the units that were cut across CTAs.  Block (c, y): CTA c of the attention
+// kernel holds the first piece of a cut unit (or the block exits); the following CTAs of the same
+// class hold the rest, each as its first segment.  One warp per query row, 32 rows per block.
 template <int D>
-__global__ void __launch_bounds__(128) tree_attn_tc_combine_kernel(const TcParams P) {
+__global__ void __launch_bounds__(256) tree_attn_tc_combine_kernel(const TcParams P) {
     const radar_attn_args& a = P.a;
-    const int lane = threadIdx.x & 31;
-    const int64_t item = (int64_t)blockIdx.x * 4 + (threadIdx.x >> 5);
-    const int node = (int)(item % kMaxNodes);
-    const int hq = (int)((item / kMaxNodes) % a.Hq);
-    const int b = (int)(item / ((int64_t)kMaxNodes * a.Hq));
-    if (b >= a.B) return;
-    const int M = min(max(a.n_nodes[b], 0), kMaxNodes);
-    const int Pb = a.prefix_len[b];
-    if (node >= M || Pb < 0 || Pb > a.max_prefix_len) return;
-    const int ntp_all = (Pb + kTileKeys - 1) / kTileKeys;
-    const int n_splits = max(1, (ntp_all + P.tiles_per_split - 1) / P.tiles_per_split);
-    if (n_splits == 1) return;                              // written directly by the attention kernel
-    const int64_t rec0 = (((int64_t)b * a.Hq + hq) * kMaxNodes + node) * P.n_splits_max;
-    float mx = -CUDART_INF_F;
-    for (int s = 0; s < n_splits; ++s) mx = fmaxf(mx, P.part_ml[rec0 + s].x);
-    float den = 0.f, o[D / 32];
+    const CutUnit cu = P.cut[blockIdx.x];
+    if (!cu.valid) return;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int pp = blockIdx.x % P.n_cls, c0 = blockIdx.x / P.n_cls;
+    const long long u1 = cu.u0 + (long long)cu.nt * cu.w;
+    // pieces: class-local CTAs c0, c0 + 1, ... while their range starts before the unit's end
+    int n_pieces = 1;
+    while (c0 + n_pieces < P.ncc && cu.tot * (c0 + n_pieces) / P.ncc < u1) ++n_pieces;
+    const int G = P.G;
+    for (int r = 0; r < 4; ++r) {
+        const int prow = blockIdx.y * 32 + warp * 4 + r;
+        if (prow >= cu.rows) break;                          // rows of a unit are live from 0 up
+        auto rec_of = [&](int j) {
+            const int slot = j == 0 ? cu.slot : 0;
+            return ((int64_t)((c0 + j) * P.n_cls + pp) * 2 + slot) * kPairRows + prow;
+        };
+        auto live = [&](int j) {                             // a CTA whose range holds no tile start has no piece
+            return tiles_before(cu.tot * (c0 + j + 1) / P.ncc, cu.u0, cu.nt, cu.w) >
+                   tiles_before(cu.tot * (c0 + j) / P.ncc, cu.u0, cu.nt, cu.w);
+        };
+        float mx = -CUDART_INF_F;
+        for (int j0 = 0; j0 < n_pieces; j0 += 32) {
+            const int j = j0 + lane;
+            float m = -CUDART_INF_F;
+            if (j < n_pieces && live(j)) m = P.part_ml[rec_of(j)].x;
+            mx = fmaxf(mx, warp_max(m));
+        }
+        float den = 0.f, o[D / 32];
 #pragma unroll
-    for (int c = 0; c < D / 32; ++c) o[c] = 0.f;
-    for (int s = 0; s < n_splits; ++s) {
-        const float2 ml = P.part_ml[rec0 + s];
-        if (ml.x == -CUDART_INF_F) continue;
-        const float w = __expf(ml.x - mx);
-        den += ml.y * w;
-        const float* src = P.part_o + (rec0 + s) * D + lane * (D / 32);
+        for (int q = 0; q < D / 32; ++q) o[q] = 0.f;
+        for (int j = 0; j < n_pieces; ++j) {
+            if (!live(j)) continue;
+            const int64_t rec = rec_of(j);
+            const float2 ml = P.part_ml[rec];
+            if (ml.x == -CUDART_INF_F) continue;
+            const float w = __expf(ml.x - mx);
+            den += ml.y * w;
+            const float* src = P.part_o + rec * D + lane * (D / 32);
 #pragma unroll
-        for (int c = 0; c < D / 32; ++c) o[c] = fmaf(src[c], w, o[c]);
+            for (int q = 0; q < D / 32; ++q) o[q] = fmaf(src[q], w, o[q]);
+        }
+        const float inv = 1.f / den;
+        const int r_glob = pp * P.pair_rows + prow;
+        const int node = r_glob / G, hq = cu.g * G + r_glob % G;
+        __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(a.O) + (((int64_t)cu.b * kMaxNodes + node) * a.Hq + hq) * D + lane * (D / 32);
+#pragma unroll
+        for (int q = 0; q < D / 32; ++q) dst[q] = __float2bfloat16(o[q] * inv);
+        if (a.lse != nullptr && lane == 0) a.lse[((int64_t)cu.b * a.Hq + hq) * kMaxNodes + node] = mx + logf(den);
     }
-    const float inv = 1.f / den;
-    __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(a.O) + (((int64_t)b * kMaxNodes + node) * a.Hq + hq) * D + lane * (D / 32);
-#pragma unroll
-    for (int c = 0; c < D / 32; ++c) dst[c] = __float2bfloat16(o[c] * inv);
-    if (a.lse != nullptr && lane == 0) a.lse[((int64_t)b * a.Hq + hq) * kMaxNodes + node] = mx + logf(den);
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -489,6 +721,27 @@ bool make_map(CUtensorMap* tm, const void* base, int d, int heads, long long row
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Grid shape.  A class is one row-block pair (256 query rows: both row blocks share every K/V tile in
+// shared memory) or, when such fused units would leave most SMs without work, one row block (128 rows).
+// CTAs per class: the grid is one CTA per SM, but at least four tiles per CTA when every sequence
+// has the longest prefix.
+void plan_grid(const radar_ctx* ctx, int B, int Hq, int Hkv, int max_prefix_len, int* pair_rows, int* n_cls, int* ncc) {
+    const int G = Hq / Hkv;
+    const int rows_max = kMaxNodes * G;
+    const long long unit_tiles = (long long)B * Hkv * ((max_prefix_len + kTileKeys - 1) / kTileKeys + 1);
+    int pr = kPairRows;
+    if (rows_max > 128 && unit_tiles * ((rows_max + 255) / 256) < 4LL * ctx->sm_count) pr = 128;
+    const int cls = (rows_max + pr - 1) / pr;
+    long long per = ctx->sm_count / cls;
+    if (per < 1) per = 1;
+    const long long cap = (unit_tiles + 3) / 4;
+    if (per > cap) per = cap;
+    if (per < 1) per = 1;
+    *pair_rows = pr;
+    *n_cls = cls;
+    *ncc = (int)per;
+}
+
 }  // namespace
 
 bool tree_attn_tc_supported(const radar_attn_args* a) {
@@ -502,31 +755,15 @@ bool tree_attn_tc_supported(const radar_attn_args* a) {
     return (al & 15) == 0 && encode_fn() != nullptr;
 }
 
-void tree_attn_tc_plan(const radar_ctx* ctx, int B, int Hq, int Hkv, int max_prefix_len, int* tiles_per_split,
-                       int* n_splits_max) {
-    const int G = Hq / Hkv;
-    const int nrb = (kMaxNodes * G + 127) / 128;
-    const int nt = (max_prefix_len + kTileKeys - 1) / kTileKeys;
-    const long long units = (long long)B * Hkv * nrb;
-    // enough CTAs to cover the machine about twice, but at least 4 tiles (512 keys) per CTA
-    int want = (int)((2LL * ctx->sm_count + units - 1) / units);
-    if (want < 1) want = 1;
-    int tps = (nt + want - 1) / want;
-    if (tps < 4) tps = 4;
-    if (tps > nt && nt > 0) tps = nt;
-    *tiles_per_split = tps;
-    *n_splits_max = nt > 0 ? (nt + tps - 1) / tps : 1;
-}
-
 size_t tree_attn_tc_workspace_bytes(const radar_ctx* ctx, int B, int Hq, int Hkv, int d, int max_prefix_len) {
-    int tps, ns;
-    tree_attn_tc_plan(ctx, B, Hq, Hkv, max_prefix_len, &tps, &ns);
-    if (ns == 1) return 256;
-    const size_t rec = (size_t)B * Hq * kMaxNodes * ns;
-    return align_up(rec * sizeof(float2), 256) + align_up(rec * d * sizeof(float), 256);
+    int pair_rows, n_cls, ncc;
+    plan_grid(ctx, B, Hq, Hkv, max_prefix_len, &pair_rows, &n_cls, &ncc);
+    const size_t rec = (size_t)n_cls * ncc * 2 * kPairRows;
+    return align_up(rec * sizeof(float2), 256) + align_up(rec * d * sizeof(float), 256) +
+           align_up((size_t)n_cls * ncc * sizeof(CutUnit), 256);
 }
 
-template <int D>
+template <int D, bool TWO>
 static int launch_tc(radar_ctx* ctx, TcParams& P, cudaStream_t stream) {
     const radar_attn_args& a = P.a;
     CUtensorMap tmQ, tmKc, tmVc, tmKt, tmVt;
@@ -538,22 +775,21 @@ static int launch_tc(radar_ctx* ctx, TcParams& P, cudaStream_t stream) {
         !make_map(&tmKc, have_prefix ? a.Kc : a.Kt, D, a.Hkv, have_prefix ? a.cache_rows : tree_rows, 1, kTileKeys) ||
         !make_map(&tmVc, have_prefix ? a.Vc : a.Vt, D, a.Hkv, have_prefix ? a.cache_rows : tree_rows, 1, kTileKeys))
         return RADAR_ERR_CUDA;
-    static bool attr_done = false;                  // once per process: not a stream operation
+    static bool attr_done = false;                  // once per process and instantiation: not a stream operation
     if (!attr_done) {
-        RADAR_CUDA_CHECK(cudaFuncSetAttribute(tree_attn_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                              Smem<D>::kDynamic));
+        RADAR_CUDA_CHECK(cudaFuncSetAttribute(tree_attn_tc_kernel<D, TWO>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                              Smem<D, TWO>::kDynamic));
         attr_done = true;
     }
-    dim3 grid((unsigned)(P.nrb_max * P.n_splits_max), (unsigned)a.Hkv, (unsigned)a.B);
     {
         radar_launch_scope scope(ctx, RADAR_K_ATTN, stream);
-        tree_attn_tc_kernel<D><<<grid, kTcThreads, Smem<D>::kDynamic, stream>>>(tmQ, tmKc, tmVc, tmKt, tmVt, P);
+        tree_attn_tc_kernel<D, TWO><<<(unsigned)(P.n_cls * P.ncc), kTcThreads, Smem<D, TWO>::kDynamic, stream>>>(
+            tmQ, tmKc, tmVc, tmKt, tmVt, P);
     }
     RADAR_CUDA_CHECK(cudaGetLastError());
-    if (P.n_splits_max > 1) {
-        const int64_t items = (int64_t)a.B * a.Hq * kMaxNodes;
+    {
         radar_launch_scope scope(ctx, RADAR_K_ATTN_COMBINE, stream);
-        tree_attn_tc_combine_kernel<D><<<(unsigned)((items + 3) / 4), 128, 0, stream>>>(P);
+        tree_attn_tc_combine_kernel<D><<<dim3((unsigned)(P.n_cls * P.ncc), kPairRows / 32), 256, 0, stream>>>(P);
     }
     RADAR_CUDA_CHECK(cudaGetLastError());
     return RADAR_OK;
@@ -564,18 +800,20 @@ int tree_attn_tc_launch(radar_ctx* ctx, const radar_attn_args* a, cudaStream_t s
     P.a = *a;
     P.G = a->Hq / a->Hkv;
     P.nodes_per_rb = 128 / P.G;
-    P.nrb_max = (kMaxNodes * P.G + 127) / 128;
     const float scale = a->scale > 0.f ? a->scale : 1.f / sqrtf((float)a->d);
     P.scale_log2 = scale * 1.4426950408889634f;
     P.cache_rows = a->cache_rows;
     P.status = ctx->d_status;
-    tree_attn_tc_plan(ctx, a->B, a->Hq, a->Hkv, a->max_prefix_len, &P.tiles_per_split, &P.n_splits_max);
+    plan_grid(ctx, a->B, a->Hq, a->Hkv, a->max_prefix_len, &P.pair_rows, &P.n_cls, &P.ncc);
     if (tree_attn_tc_workspace_bytes(ctx, a->B, a->Hq, a->Hkv, a->d, a->max_prefix_len) > a->workspace_bytes)
         return RADAR_ERR_WORKSPACE;
-    const size_t rec = (size_t)a->B * a->Hq * kMaxNodes * P.n_splits_max;
+    const size_t rec = (size_t)P.n_cls * P.ncc * 2 * kPairRows;
     P.part_ml = reinterpret_cast<float2*>(a->workspace);
     P.part_o = reinterpret_cast<float*>(reinterpret_cast<char*>(a->workspace) + align_up(rec * sizeof(float2), 256));
-    return a->d == 128 ? launch_tc<128>(ctx, P, stream) : launch_tc<64>(ctx, P, stream);
+    P.cut = reinterpret_cast<CutUnit*>(reinterpret_cast<char*>(P.part_o) + align_up(rec * a->d * sizeof(float), 256));
+    const bool two = P.pair_rows > 128 && P.G * kMaxNodes > 128;      // some unit can have two live row blocks
+    if (a->d == 128) return two ? launch_tc<128, true>(ctx, P, stream) : launch_tc<128, false>(ctx, P, stream);
+    return two ? launch_tc<64, true>(ctx, P, stream) : launch_tc<64, false>(ctx, P, stream);
 }
 
 }  // namespace radar
