@@ -262,10 +262,15 @@ def run_ours(args):
         ctx.check_device_status(stream)
 
         # ---- per-kernel durations (CUDA events around every kernel, eager launches, same rotation) ----
+        # The host must stay ahead of the GPU, otherwise an event pair also spans the host's launch latency:
+        # each batch of steps is enqueued behind a spinning kernel that holds the stream for a few ms.
         prof_steps = min(args.steps, 50)
         ctx.profile_begin(prof_steps * (2 * t_max + 8))
-        for i in range(prof_steps):
-            one_step(copies[i % n_copies])
+        for i0 in range(0, prof_steps, 5):
+            torch.cuda._sleep(8_000_000)
+            for i in range(i0, min(i0 + 5, prof_steps)):
+                one_step(copies[i % n_copies])
+            stream.synchronize()
         ctx.profile_end()
         kstats = ctx.kernel_stats()
 

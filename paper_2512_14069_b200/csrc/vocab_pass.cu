@@ -4,8 +4,8 @@
 // The pass is HBM-bound, so each logit is read exactly once, with 16-byte streaming loads, and a
 // block keeps its whole chunk (16 or 32 values per thread) in registers: every load of the chunk is
 // in flight at once, and nothing is re-read from memory for the selection.  Selection is a filter,
-// not a running list: the k-th best of each warp's 32 per-thread maxima is a lower bound of the
-// chunk's k-th best value; the best such bound over the warps becomes the threshold, the few
+// not a running list: with j = ceil(k / 8), the j-th best of each warp's 32 per-thread maxima, taken
+// at its lowest over the 8 warps, is a lower bound of the chunk's k-th best value; the few
 // register values that reach it go to a shared-memory candidate list, and their exact ranks by
 // (logit desc, token asc) are counted there.  If an adversarial chunk overflows the list, k rounds
 // of a block-wide arg-best over the registers give the same result.
@@ -44,6 +44,12 @@ template <> struct Vec<__nv_bfloat16> {
 __device__ __forceinline__ float fast_exp2(float x) {
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+__device__ __forceinline__ float max_nan(float a, float b) {
+    float y;
+    asm("max.NaN.f32 %0, %1, %2;" : "=f"(y) : "f"(a), "f"(b));
     return y;
 }
 
@@ -105,22 +111,27 @@ __global__ void __launch_bounds__(kThreads, WANT_LSE ? (EPT == 32 ? 3 : 4) : 5) 
     else if (tid >= N && tid - N < ntail) xs_idx = tail0 + tid - N;
     if (xs_idx >= 0) xs = to_float(base[xs_idx]);
 
-    // ---- per-thread best and (max, sum exp) ----
-    float bv = xs;
-    int bi = xs_idx >= 0 ? xs_idx : kEmptyIdx + tid;
-    bool nan = xs != xs;
+    // ---- per-thread best: NaN-propagating max first, then the lowest index that holds it ----
+    // (index order within a thread: head scalar < vector elements in (u, e) order < tail scalar)
+    float mxa[4] = {xs, -CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F};
 #pragma unroll
-    for (int u = 0; u < NV; ++u) {
+    for (int u = 0; u < NV; ++u)
+#pragma unroll
+        for (int e = 0; e < N; ++e) mxa[e & 3] = max_nan(mxa[e & 3], x[u][e]);
+    const float bv = max_nan(max_nan(mxa[0], mxa[1]), max_nan(mxa[2], mxa[3]));
+    const bool nan = bv != bv;
+    int bi = kEmptyIdx + tid;
+    if (xs_idx >= 0 && tid >= N && xs == bv) bi = xs_idx;
+#pragma unroll
+    for (int u = NV - 1; u >= 0; --u) {
         const int idx0 = body0 + (tid + u * kThreads) * N;
+        if (tid + u * kThreads < nvec) {
 #pragma unroll
-        for (int e = 0; e < N; ++e) {
-            const float v = x[u][e];
-            nan |= (v != v);
-            // a later element only wins when strictly larger: the lowest index of the maximum is kept,
-            // except against the scalar slot, whose index may be higher (tail) - handled by precedes
-            if (v > bv || (v == bv && idx0 + e < bi)) { bv = v; bi = idx0 + e; }
+            for (int e = N - 1; e >= 0; --e)
+                if (x[u][e] == bv) bi = idx0 + e;
         }
     }
+    if (xs_idx >= 0 && tid < N && xs == bv) bi = xs_idx;
     float ssum = 0.f;
     if (WANT_LSE) {
         if (bv > -CUDART_INF_F) {
@@ -167,16 +178,19 @@ __global__ void __launch_bounds__(kThreads, WANT_LSE ? (EPT == 32 ? 3 : 4) : 5) 
             }
         }
     } else {
-        // ---- threshold: k-th best of this warp's per-thread bests (k <= 32), best over the warps ----
+        // ---- threshold: the j-th best per-thread best of every warp, j = ceil(k / warps); the last of these
+        //      in (value desc, index asc) order has at least k elements of the chunk not after it ----
         {
-            int rank = 0;
-#pragma unroll
-            for (int l = 0; l < 32; ++l) {
-                const float ov = __shfl_sync(kFull, bv, l);
-                const int oi = __shfl_sync(kFull, bi, l);
-                rank += precedes(ov, oi, bv, bi) ? 1 : 0;
+            const int jth = (k + kWarps - 1) / kWarps;
+            float cv = bv, wv = bv;
+            int ci = bi, wi = bi;
+            for (int r = 0; r < jth; ++r) {
+                wv = cv;
+                wi = ci;
+                warp_best(wv, wi);
+                if (ci == wi) { cv = -CUDART_INF_F; ci = 0x7fffffff; }       // this lane's entry was taken
             }
-            if (rank == k - 1) { sh_tv[warp] = bv; sh_ti[warp] = bi; }
+            if (lane == 0) { sh_tv[warp] = wv; sh_ti[warp] = wi; }
         }
         __syncthreads();
         if (nan) atomicOr(&sh_nan, 1);
@@ -184,7 +198,7 @@ __global__ void __launch_bounds__(kThreads, WANT_LSE ? (EPT == 32 ? 3 : 4) : 5) 
         int ti = sh_ti[0];
 #pragma unroll
         for (int w = 1; w < kWarps; ++w)
-            if (precedes(sh_tv[w], sh_ti[w], tv, ti)) { tv = sh_tv[w]; ti = sh_ti[w]; }
+            if (precedes(tv, ti, sh_tv[w], sh_ti[w])) { tv = sh_tv[w]; ti = sh_ti[w]; }
         // ---- candidates: everything that is not after the threshold pair ----
         auto push = [&](float v, int idx) {
             if (v > tv || (v == tv && idx <= ti)) {

@@ -71,7 +71,9 @@ def oracle_attention(cfg: W.Config, inp, trees, pairs=None):
     n_nodes = np.array([t["n_nodes"] for t in trees])
     mask = np.stack([t["mask"] for t in trees])
     w = lambda x: W.widen(cfg, x)
-    return O.tree_attention(w(inp["Q"]), [w(x) for x in inp["Kc"]], [w(x) for x in inp["Vc"]], w(inp["Kt"]),
+    need = set(range(cfg.B)) if pairs is None else {b for b, _ in pairs}     # widen only what will be read
+    wide = lambda xs: [w(x) if b in need else x[:0] for b, x in enumerate(xs)]
+    return O.tree_attention(w(inp["Q"]), wide(inp["Kc"]), wide(inp["Vc"]), w(inp["Kt"]),
                             w(inp["Vt"]), mask, n_nodes, inp["prefix_len"], pairs=pairs)
 
 
