@@ -44,6 +44,7 @@ def parse():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-graph", action="store_true", help="launch eagerly instead of replaying CUDA graphs")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-scale-probe", action="store_true", help="skip the roofline probe at the 70B shapes")
     return ap.parse_args()
 
 
@@ -131,12 +132,91 @@ class ClockSampler:
         return out
 
 
-def measured_peak_gbs():
+def measured_peaks():
+    """HBM GB/s and dense bf16 TFLOP/s (burst: a kernel timed alone) measured on this machine, else the stated fallback."""
     try:
         with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
-            return float(json.load(f)["hbm_gbs"]), "measured"
+            d = json.load(f)
+        return {"hbm_gbs": float(d["hbm_gbs"]), "bf16_tflops": float(d["bf16_tflops"]), "kind": "of measured"}
     except Exception:
-        return 6650.0, "fallback"
+        return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "kind": "of fallback"}
+
+
+def roofline_entry(name, k, peaks, traffic):
+    """Roofline object of one kernel from its event-timed duration: the binding roof is the one that
+    needs more time (bytes / HBM peak against flops / bf16 peak)."""
+    us = k["avg_us"]
+    t_hbm = k["alg_bytes_per_launch"] / (peaks["hbm_gbs"] * 1e9)
+    t_tensor = (k["tflops"] * us * 1e-6 * 1e12) / (peaks["bf16_tflops"] * 1e12) if "tflops" in k else 0.0
+    if t_tensor > t_hbm:
+        return {"kernel": name, "bound": "tensor", "achieved": k["tflops"], "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                "frac": k["tflops"] / peaks["bf16_tflops"], "peak_kind": peaks["kind"], "traffic": traffic,
+                "alg_bytes_per_launch": k["alg_bytes_per_launch"], "hbm_gbs": k["gbs"], "avg_us": us}
+    return {"kernel": name, "bound": "hbm", "achieved": k["gbs"], "peak": peaks["hbm_gbs"], "unit": "GB/s",
+            "frac": k["gbs"] / peaks["hbm_gbs"], "peak_kind": peaks["kind"], "traffic": traffic,
+            "alg_bytes_per_launch": k["alg_bytes_per_launch"], "avg_us": us}
+
+
+def scale_probe(ctx, dev, peaks, reps=20):
+    """Roofline fractions of the three bandwidth / tensor kernels at the LLaMA-3.3-70B shapes (B = 8, 64 / 8 heads,
+    prefix 8192, V = 128256, k = 10, 61 tree rows), where a launch is long enough for a roofline to mean
+    something.  Timing only: operands are random device tensors (every buffer read is larger than L2, or
+    rotates over buffers that together are), each launch bracketed by CUDA events."""
+    import torch
+    from paper_2512_14069_b200 import binding as rb
+    from paper_2512_14069_b200.pipeline import SpecStep
+    cfg = W.CONFIGS[4]
+    B, V, k, t_max, Hq, Hkv, d, P = cfg.B, cfg.V, cfg.k, cfg.t_max, cfg.Hq, cfg.Hkv, cfg.d, cfg.P[1]
+    g = torch.Generator(device=dev)
+    g.manual_seed(4)
+    step = SpecStep(ctx, B=B, V=V, k=k, t_max=t_max, N=cfg.N, Hq=Hq, Hkv=Hkv, d=d, kv_dtype=torch.bfloat16,
+                    max_prefix_len=P, mode=rb.RADAR_GREEDY, device=dev)
+    gate = {n: torch.from_numpy(v).to(dev) for n, v in W.gate_weights(cfg).items()}
+    draft = torch.randn(B, step.R, V, device=dev, generator=g)
+    force = torch.full((B,), t_max, dtype=torch.int32, device=dev)
+    root = torch.zeros(B, dtype=torch.int32, device=dev)
+    plen = torch.full((B,), P, dtype=torch.int32, device=dev)
+    kv_start = (torch.arange(B, device=dev, dtype=torch.int64) * P)
+    step.run_expansion(draft, gate, force)
+    step.build_tree(root, plen, None)
+    n_nodes = step.n_nodes.cpu().numpy().astype(np.int64)
+    Q = torch.randn(B, 64, Hq, d, device=dev, generator=g).bfloat16()
+    Kt, Vt = (torch.randn(B, 64, Hkv, d, device=dev, generator=g).bfloat16() for _ in range(2))
+    Kc, Vc = (torch.randn(B * P, Hkv, d, device=dev, generator=g).bfloat16() for _ in range(2))
+    target = torch.randn(B, 64, V, device=dev, generator=g)
+
+    def timed(fn):
+        for i in range(3):
+            fn(i)
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(reps)]
+        for i, (e0, e1) in enumerate(ev):
+            e0.record(); fn(i); e1.record()
+        torch.cuda.synchronize()
+        return float(np.median([e0.elapsed_time(e1) for e0, e1 in ev])) * 1000.0        # us
+
+    ctx.reset_launch_counts()
+    us_attn = timed(lambda i: step.attention(Q, Kc, Vc, kv_start, plen, Kt, Vt))          # attention + combine
+    us_acc = timed(lambda i: step.accept(target))                                          # row arg-best + walk
+    us_exp = timed(lambda i: step.expand(2 + i % (t_max - 1), draft, gate, force))         # calls 2..t_max rotate 287 MB
+    ctx.check_device_status()
+    kv_bytes = float(((P + n_nodes) * Hkv * d * 2 * 2).sum() + 2 * n_nodes.sum() * Hq * d * 2)
+    flops = float((4 * n_nodes * Hq * (P + n_nodes) * d).sum())
+    shapes = "LLaMA-3.3-70B shapes: B=8, Hq/Hkv/d=64/8/128, prefix 8192, V=128256, k=10, %d..%d tree rows" % (n_nodes.min(), n_nodes.max())
+    out = []
+    ka = {"avg_us": us_attn, "alg_bytes_per_launch": kv_bytes, "gbs": kv_bytes / us_attn / 1e3, "tflops": flops / us_attn / 1e6}
+    out.append(roofline_entry("tree_attention (+combine)", ka, peaks, NCU_TRAFFIC.get(("tree_attention", 4))))
+    b_acc = float(n_nodes.sum()) * V * 4
+    out.append(roofline_entry("vocab_pass(accept) (+greedy_walk)", {"avg_us": us_acc, "alg_bytes_per_launch": b_acc,
+                                                                    "gbs": b_acc / us_acc / 1e3}, peaks,
+                              NCU_TRAFFIC.get(("vocab_pass(accept)", 4))))
+    b_exp = float(B * k * V * 4)
+    out.append(roofline_entry("vocab_pass(expand) (+select_gate)", {"avg_us": us_exp, "alg_bytes_per_launch": b_exp,
+                                                                    "gbs": b_exp / us_exp / 1e3}, peaks,
+                              NCU_TRAFFIC.get(("vocab_pass(expand)", 4))))
+    for o in out:
+        o["workload"] = shapes
+        o["timing"] = "median of %d eager launches, each API call (all its kernels) between two CUDA events" % reps
+    return out
 
 
 # ------------------------------------------------------------------------------------------------
@@ -316,19 +396,19 @@ def run_ours(args):
     kv_b = 2 if cfg.kv_dtype == "bf16" else 4
     plen = inp["prefix_len"].astype(np.int64)
     rows_expand = int(sum(1 + (c - 1) * k for c in calls))
-    alg = {   # algorithmic bytes per STEP of each HBM-bound kernel
+    alg = {   # algorithmic bytes per STEP of each kernel that has a bandwidth model
         "vocab_pass(expand)": rows_expand * V * s,
         "vocab_pass(accept)": int(n_nodes.sum()) * V * s,
         "tree_attention": int(((plen + n_nodes) * cfg.Hkv * cfg.d * 2 * kv_b).sum()
                               + 2 * n_nodes.sum() * cfg.Hq * cfg.d * kv_b),
     }
+    attn_flops = float((4 * n_nodes * cfg.Hq * (plen + n_nodes) * cfg.d).sum())     # un-padded rows, QK^T + PV
     if mode == rb.RADAR_STOCHASTIC:
         alen = step.accept_len.cpu().numpy()
         alg["stochastic_walk"] = int(((alen + 1) * 2 * V * s).sum())      # target + draft row of each visited node, once
     timed = {n: v for n, v in kstats.items() if v[2] > 0}
-    dom = max(timed, key=lambda n: timed[n][1]) if timed else None
-    peak, peak_kind = measured_peak_gbs()
-    roofline = None
+    peaks = measured_peaks()
+    peak = peaks["hbm_gbs"]
     kernels = {n: {"launches_per_step": v[2] / prof_steps, "avg_us": 1000.0 * v[1] / v[2],
                    "share": v[1] / sum(x[1] for x in timed.values())} for n, v in timed.items()}
     for n in kernels:
@@ -336,16 +416,20 @@ def run_ours(args):
             per_launch = alg[n] / kernels[n]["launches_per_step"]
             kernels[n]["alg_bytes_per_launch"] = per_launch
             kernels[n]["gbs"] = per_launch / (kernels[n]["avg_us"] * 1e-6) / 1e9
+    if "tree_attention" in kernels and cfg.kv_dtype == "bf16":
+        kernels["tree_attention"]["tflops"] = attn_flops / (kernels["tree_attention"]["avg_us"] * 1e-6) / 1e12
+    # The dominant kernel among those that move data (the per-sequence select / tree / walk blocks touch
+    # kilobytes and have no bandwidth or tensor model: they are listed in `kernels` with their share).
+    modelled = [n for n in kernels if n in alg]
+    dom = max(modelled, key=lambda n: timed[n][1]) if modelled else None
+    dom_overall = max(timed, key=lambda n: timed[n][1]) if timed else None
+    roofline = None
     if dom is not None:
-        if dom in alg:
-            ach = kernels[dom]["gbs"]
-            roofline = {"kernel": dom, "bound": "hbm", "achieved": ach, "peak": peak, "unit": "GB/s",
-                        "frac": ach / peak, "peak_kind": "of " + peak_kind,
-                        "traffic": NCU_TRAFFIC.get((dom, cfg.cid)),
-                        "alg_bytes_per_launch": kernels[dom]["alg_bytes_per_launch"], "avg_us": kernels[dom]["avg_us"]}
-        else:
-            roofline = {"kernel": dom, "bound": "latency", "achieved": None, "peak": peak, "unit": "GB/s",
-                        "frac": None, "traffic": None, "avg_us": kernels[dom]["avg_us"]}
+        roofline = roofline_entry(dom, kernels[dom], peaks, NCU_TRAFFIC.get((dom, cfg.cid)))
+        roofline["dominant_overall"] = dom_overall
+        if dom_overall != dom:
+            roofline["note"] = ("%s has the largest share of device time (%.0f %%) but is a latency-bound per-sequence "
+                                "block with no bandwidth model" % (dom_overall, 100 * kernels[dom_overall]["share"]))
 
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
@@ -365,6 +449,10 @@ def run_ours(args):
         "roofline": roofline,
         "kernels": kernels,
     }
+    if rank == 0 and world == 1 and not args.no_scale_probe:
+        del copies, graphs
+        torch.cuda.empty_cache()
+        out["rooflines_at_scale"] = scale_probe(ctx, dev, peaks)
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         out["cpu_baseline"] = cpu_baseline(cfg, budget_s=15.0)
     if rank == 0:

@@ -4,9 +4,9 @@
 // The pass is HBM-bound, so each logit is read exactly once, with 16-byte streaming loads, and a
 // block keeps its whole chunk (16 or 32 values per thread) in registers: every load of the chunk is
 // in flight at once, and nothing is re-read from memory for the selection.  Selection is a filter,
-// not a running list: with j = ceil(k / 8), the j-th best of each warp's 32 per-thread maxima, taken
+// not a running list: with j = ceil(k / 8), the j-th largest of each warp's 32 per-thread maxima, taken
 // at its lowest over the 8 warps, is a lower bound of the chunk's k-th best value; the few
-// register values that reach it go to a shared-memory candidate list, and their exact ranks by
+// values that reach it go to a shared-memory candidate list, and their exact ranks by
 // (logit desc, token asc) are counted there.  If an adversarial chunk overflows the list, k rounds
 // of a block-wide arg-best over the registers give the same result.
 #include "common.cuh"
@@ -111,8 +111,7 @@ __global__ void __launch_bounds__(kThreads, WANT_LSE ? (EPT == 32 ? 3 : 4) : 5) 
     else if (tid >= N && tid - N < ntail) xs_idx = tail0 + tid - N;
     if (xs_idx >= 0) xs = to_float(base[xs_idx]);
 
-    // ---- per-thread best: NaN-propagating max first, then the lowest index that holds it ----
-    // (index order within a thread: head scalar < vector elements in (u, e) order < tail scalar)
+    // ---- per-thread max (NaN-propagating) ----
     float mxa[4] = {xs, -CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F};
 #pragma unroll
     for (int u = 0; u < NV; ++u)
@@ -120,18 +119,6 @@ __global__ void __launch_bounds__(kThreads, WANT_LSE ? (EPT == 32 ? 3 : 4) : 5) 
         for (int e = 0; e < N; ++e) mxa[e & 3] = max_nan(mxa[e & 3], x[u][e]);
     const float bv = max_nan(max_nan(mxa[0], mxa[1]), max_nan(mxa[2], mxa[3]));
     const bool nan = bv != bv;
-    int bi = kEmptyIdx + tid;
-    if (xs_idx >= 0 && tid >= N && xs == bv) bi = xs_idx;
-#pragma unroll
-    for (int u = NV - 1; u >= 0; --u) {
-        const int idx0 = body0 + (tid + u * kThreads) * N;
-        if (tid + u * kThreads < nvec) {
-#pragma unroll
-            for (int e = N - 1; e >= 0; --e)
-                if (x[u][e] == bv) bi = idx0 + e;
-        }
-    }
-    if (xs_idx >= 0 && tid < N && xs == bv) bi = xs_idx;
     float ssum = 0.f;
     if (WANT_LSE) {
         if (bv > -CUDART_INF_F) {
@@ -161,6 +148,19 @@ __global__ void __launch_bounds__(kThreads, WANT_LSE ? (EPT == 32 ? 3 : 4) : 5) 
 
     if (!WANT_LSE || k == 1) {
         // ---- arg-best only (the pass without the normaliser is always run with k = 1) ----
+        // lowest index that holds the thread's max (index order: head scalar < vector elements < tail scalar)
+        int bi = kEmptyIdx + tid;
+        if (xs_idx >= 0 && tid >= N && xs == bv) bi = xs_idx;
+#pragma unroll
+        for (int u = NV - 1; u >= 0; --u) {
+            const int idx0 = body0 + (tid + u * kThreads) * N;
+            if (tid + u * kThreads < nvec) {
+#pragma unroll
+                for (int e = N - 1; e >= 0; --e)
+                    if (x[u][e] == bv) bi = idx0 + e;
+            }
+        }
+        if (xs_idx >= 0 && tid < N && xs == bv) bi = xs_idx;
         float wv = bv;
         int wi = bi;
         warp_best(wv, wi);
@@ -178,44 +178,44 @@ __global__ void __launch_bounds__(kThreads, WANT_LSE ? (EPT == 32 ? 3 : 4) : 5) 
             }
         }
     } else {
-        // ---- threshold: the j-th best per-thread best of every warp, j = ceil(k / warps); the last of these
-        //      in (value desc, index asc) order has at least k elements of the chunk not after it ----
+        // ---- threshold: the j-th largest per-thread max of every warp (with multiplicity), j = ceil(k / warps);
+        //      the smallest of these over the warps has at least k elements of the chunk at or above it ----
         {
             const int jth = (k + kWarps - 1) / kWarps;
             float cv = bv, wv = bv;
-            int ci = bi, wi = bi;
             for (int r = 0; r < jth; ++r) {
-                wv = cv;
-                wi = ci;
-                warp_best(wv, wi);
-                if (ci == wi) { cv = -CUDART_INF_F; ci = 0x7fffffff; }       // this lane's entry was taken
+                wv = warp_max(cv);
+                const unsigned who = __ballot_sync(kFull, cv == wv);
+                if (lane == __ffs(who) - 1) cv = -CUDART_INF_F;                // one holder of the max leaves
             }
-            if (lane == 0) { sh_tv[warp] = wv; sh_ti[warp] = wi; }
+            if (lane == 0) sh_tv[warp] = wv;
         }
         __syncthreads();
         if (nan) atomicOr(&sh_nan, 1);
         float tv = sh_tv[0];
-        int ti = sh_ti[0];
 #pragma unroll
-        for (int w = 1; w < kWarps; ++w)
-            if (precedes(tv, ti, sh_tv[w], sh_ti[w])) { tv = sh_tv[w]; ti = sh_ti[w]; }
-        // ---- candidates: everything that is not after the threshold pair ----
-        auto push = [&](float v, int idx) {
-            if (v > tv || (v == tv && idx <= ti)) {
+        for (int w = 1; w < kWarps; ++w) tv = fminf(tv, sh_tv[w]);
+        // ---- candidates: every element at or above the threshold value.  One bit per register value; the few
+        //      that qualify are re-read from memory by position, so no register is indexed dynamically ----
+        unsigned mask = 0;
+#pragma unroll
+        for (int u = 0; u < NV; ++u)
+#pragma unroll
+            for (int e = 0; e < N; ++e) mask |= (x[u][e] >= tv ? 1u : 0u) << (u * N + e);
+        if (xs_idx >= 0 && xs >= tv) {
+            const int slot = atomicAdd(&sh_cnt, 1);
+            if (slot < kCandCap) { sh_cv[slot] = xs; sh_ci[slot] = xs_idx; }
+        }
+        while (mask) {
+            const int bit = __ffs(mask) - 1;
+            mask &= mask - 1;
+            const int j = tid + (bit / N) * kThreads;
+            if (j < nvec) {                                                     // padding of a short chunk is not an element
+                const int idx = body0 + j * N + bit % N;
                 const int slot = atomicAdd(&sh_cnt, 1);
-                if (slot < kCandCap) { sh_cv[slot] = v; sh_ci[slot] = idx; }
-            }
-        };
-#pragma unroll
-        for (int u = 0; u < NV; ++u) {
-            const int idx0 = body0 + (tid + u * kThreads) * N;
-            if (tid + u * kThreads < nvec) {
-#pragma unroll
-                for (int e = 0; e < N; ++e)
-                    if (x[u][e] >= tv) push(x[u][e], idx0 + e);
+                if (slot < kCandCap) { sh_cv[slot] = to_float(base[idx]); sh_ci[slot] = idx; }
             }
         }
-        if (xs_idx >= 0 && xs >= tv) push(xs, xs_idx);
         __syncthreads();
         const int C = sh_cnt;
         float* out_v = p.part_v + rec * k;
