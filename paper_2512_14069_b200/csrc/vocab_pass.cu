@@ -65,7 +65,7 @@ __device__ __forceinline__ void warp_best(float& v, int& i) {
 
 // EPT = values per thread kept in registers (a multiple of the vector width), chunk = kThreads * EPT
 template <typename T, int EPT, bool WANT_LSE>
-__global__ void __launch_bounds__(kThreads, WANT_LSE ? (EPT == 32 ? 3 : 4) : 5) vocab_pass_kernel(const VocabPassParams p) {
+__global__ void __launch_bounds__(kThreads, WANT_LSE ? (EPT == 32 ? 5 : 6) : 5) vocab_pass_kernel(const VocabPassParams p) {
     using VT = Vec<T>;
     constexpr int N = VT::N;
     constexpr int NV = EPT / N;
@@ -284,11 +284,11 @@ void launch_ept(const VocabPassParams& p, unsigned grid, cudaStream_t stream) {
 
 }  // namespace
 
-// chunk is 8192 values (32 per thread, three blocks per SM), or 4096 (16 per thread, four blocks) when
+// chunk is 8192 values (32 per thread, five blocks per SM), or 4096 (16 per thread, six blocks) when
 // the larger one would leave SMs without work
 int vocab_pass_plan_chunks(int sm_count, int rows, int V, int* chunk_out) {
     int chunk = 8192;
-    if ((long long)rows * ((V + chunk - 1) / chunk) < 3LL * sm_count) chunk = 4096;
+    if ((long long)rows * ((V + chunk - 1) / chunk) < 5LL * sm_count) chunk = 4096;
     *chunk_out = chunk;
     return (V + chunk - 1) / chunk;
 }
