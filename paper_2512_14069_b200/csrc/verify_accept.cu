@@ -1,9 +1,10 @@
 // radar_verify_accept: acceptance of the verified tree.
 //   greedy     - vocabulary pass with k = 1 (row argmax, no exponentials) over the target logits of
 //                the live tree rows, then one warp per sequence walks the tree with ballots.
-//   stochastic - one block per sequence walks the tree lazily: only rows on the accepted path are
-//                read.  Probabilities are fp64.  p and q of the current node are cached (normalised)
-//                in the workspace; after j rejections the residual pair is, for every token v that has
+//   stochastic - one thread-block cluster per sequence walks the tree lazily: only rows on the accepted
+//                path are read, and each CTA of the cluster owns a slice of the vocabulary in every pass.
+//                Probabilities are fp64.  exp((z - max) / T) of the current node's target and draft rows
+//                is cached in the workspace (p, q = cached value / row sum); after j rejections the residual pair is, for every token v that has
 //                not been proposed yet,  p_j(v) = max(0, p(v) - a_j q(v)) / W_j,  q_j(v) = c_j q(v),
 //                and for the token proposed at trial i <= j,  p_j(x_i) = max(0, p(x_i) - a_i q(x_i)) / W_j,
 //                q_j(x_i) = 0, with a_{j+1} = a_j + c_j W_j,  c_{j+1} = c_j / (1 - q_j(x_{j+1})) and
@@ -78,70 +79,115 @@ __global__ void __launch_bounds__(64) greedy_walk_kernel(const GreedyParams P) {
 // stochastic walk
 // ------------------------------------------------------------------------------------------
 constexpr int kSThreads = 1024;
+constexpr int kMaxCluster = 8;           // portable cluster size limit
 
 struct StochParams {
     radar_accept_args a;
-    double* p_cache;     // [B][V]
-    double* q_cache;     // [B][V]
+    double* p_cache;     // [B][V] unnormalised exp((z_target - max) / T)
+    double* q_cache;     // [B][V] same for the draft row
     int* status;
 };
 
-struct BlockRed {
-    double* scratch;     // [32] shared
-    __device__ double sum(double v) {
+// The walk of one sequence is shared by the CTAs of a thread-block cluster: CTA r owns the vocabulary
+// slice [V r / n, V (r + 1) / n) of every full-vocabulary pass.  Every scalar that steers the walk is
+// reduced over the cluster into every CTA in a fixed order, so all CTAs take identical decisions and
+// meet at the same cluster barriers.
+struct ClusterRed {
+    double* block_scratch;   // [32] shared
+    double* slots;           // [2][kMaxCluster] shared; the same array exists in every CTA of the cluster
+    unsigned rank, n;
+    unsigned phase;
+
+    __device__ double block_sum(double v) {
         v = warp_sum(v);
         __syncthreads();
-        if ((threadIdx.x & 31) == 0) scratch[threadIdx.x >> 5] = v;
+        if ((threadIdx.x & 31) == 0) block_scratch[threadIdx.x >> 5] = v;
         __syncthreads();
         double t = 0.0;
-        for (int w = 0; w < kSThreads / 32; ++w) t += scratch[w];     // same order in every thread
+        for (int w = 0; w < kSThreads / 32; ++w) t += block_scratch[w];     // same order in every thread
         return t;
     }
-    __device__ double max(double v) {
+    __device__ double block_max(double v) {
         v = warp_max(v);
         __syncthreads();
-        if ((threadIdx.x & 31) == 0) scratch[threadIdx.x >> 5] = v;
+        if ((threadIdx.x & 31) == 0) block_scratch[threadIdx.x >> 5] = v;
         __syncthreads();
-        double t = scratch[0];
-        for (int w = 1; w < kSThreads / 32; ++w) t = fmax(t, scratch[w]);
+        double t = block_scratch[0];
+        for (int w = 1; w < kSThreads / 32; ++w) t = fmax(t, block_scratch[w]);
+        return t;
+    }
+    // every CTA's value lands in out[0..n) of every CTA (rank order)
+    __device__ void all_gather(double mine, double* out) {
+        double* my = slots + (phase & 1) * kMaxCluster;
+        if (threadIdx.x < n) {
+            asm volatile(
+                "{\n\t.reg .u32 ra;\n\t"
+                "mapa.shared::cluster.u32 ra, %0, %1;\n\t"
+                "st.shared::cluster.f64 [ra], %2;\n\t}"
+                ::"r"((uint32_t)__cvta_generic_to_shared(my + rank)), "r"(threadIdx.x), "d"(mine)
+                : "memory");
+        }
+        cluster_sync();
+        for (unsigned r = 0; r < n; ++r) out[r] = my[r];
+        ++phase;                         // the other half is written next: no second barrier is needed
+    }
+    __device__ static void cluster_sync() {
+        asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+    }
+    __device__ double sum(double local) {
+        double all[kMaxCluster];
+        all_gather(block_sum(local), all);
+        double t = 0.0;
+        for (unsigned r = 0; r < n; ++r) t += all[r];
+        return t;
+    }
+    __device__ double max(double local) {
+        double all[kMaxCluster];
+        all_gather(block_max(local), all);
+        double t = all[0];
+        for (unsigned r = 1; r < n; ++r) t = fmax(t, all[r]);
         return t;
     }
 };
 
-// cache[v] = softmax(z / T)[v] in fp64; every thread returns after the cache is complete
+// cache[v] = exp(z[v] / T - max) over this CTA's slice; returns 1 / sum over the whole row
 template <typename T>
-__device__ void softmax_to_cache(const T* z, int V, double invT, double* cache, BlockRed& red, bool* nan_seen) {
+__device__ double softmax_to_cache(const T* z, int v0, int v1, double invT, double* cache, ClusterRed& red, bool* nan_seen) {
     double m = -CUDART_INF;
-    for (int v = threadIdx.x; v < V; v += kSThreads) {
+    for (int v = v0 + threadIdx.x; v < v1; v += kSThreads) {
         const float zf = to_float(z[v]);
         if (zf != zf) *nan_seen = true;
         m = fmax(m, (double)zf * invT);
     }
     m = red.max(m);
     double s = 0.0;
-    for (int v = threadIdx.x; v < V; v += kSThreads) {
+    for (int v = v0 + threadIdx.x; v < v1; v += kSThreads) {
         const double e = exp((double)to_float(z[v]) * invT - m);
         cache[v] = e;
         s += e;
     }
-    s = red.sum(s);
-    const double inv = 1.0 / s;
-    for (int v = threadIdx.x; v < V; v += kSThreads) cache[v] *= inv;
-    __syncthreads();
+    s = red.sum(s);                      // its cluster barrier also publishes every slice of the cache
+    return 1.0 / s;
 }
 
 template <typename T>
 __global__ void __launch_bounds__(kSThreads) stochastic_walk_kernel(const StochParams P) {
     const radar_accept_args& a = P.a;
-    const int b = blockIdx.x, tid = threadIdx.x;
+    unsigned crank, csize;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(crank));
+    asm volatile("mov.u32 %0, %%cluster_nctarank;" : "=r"(csize));
+    const int b = blockIdx.x / csize, tid = threadIdx.x;
     const int V = a.V, W = a.t_max + 1;
     __shared__ double s_red[32];
+    __shared__ double s_slots[2 * kMaxCluster];
     __shared__ int s_tok[kMaxNodes], s_par[kMaxNodes], s_drow[kMaxNodes], s_child[kMaxNodes];
     __shared__ int s_nchild;
     __shared__ int s_rx[RADAR_MAX_NODES];        // tokens proposed and rejected at the current node
     __shared__ double s_ra[RADAR_MAX_NODES];     // their frozen coefficients a_i
     __shared__ int s_pick, s_last_pos;
-    BlockRed red{s_red};
+    ClusterRed red{s_red, s_slots, crank, csize, 0};
+    const int v0 = (int)((long long)V * crank / csize), v1 = (int)((long long)V * (crank + 1) / csize);
+    const bool lead = crank == 0;                 // writes the per-sequence outputs
 
     const int M = min(max(a.n_nodes[b], 1), kMaxNodes);
     if (tid < kMaxNodes) {
@@ -150,6 +196,7 @@ __global__ void __launch_bounds__(kSThreads) stochastic_walk_kernel(const StochP
         s_drow[tid] = tid < M ? a.tree_draft_row[(size_t)b * kMaxNodes + tid] : -1;
     }
     __syncthreads();
+    ClusterRed::cluster_sync();                   // every CTA's shared memory is live before the first remote store
 
     const T* target = reinterpret_cast<const T*>(a.target_logits) + (size_t)b * kMaxNodes * V;
     const T* draft = reinterpret_cast<const T*>(a.draft_logits) + (size_t)b * a.R * V;
@@ -162,13 +209,14 @@ __global__ void __launch_bounds__(kSThreads) stochastic_walk_kernel(const StochP
     int32_t* pn = a.path_nodes + (size_t)b * W;
     int32_t* pt = a.path_tokens + (size_t)b * W;
     int cur = 0, len = 0;
-    if (tid == 0) { pn[0] = 0; pt[0] = s_tok[0]; }
+    if (lead && tid == 0) { pn[0] = 0; pt[0] = s_tok[0]; }
 
     int n_rej = 0;           // rejections at the final node (0 => weights are p itself)
-    double a_coef = 0.0;
+    double a_coef = 0.0;     // p_j(v) = max(0, p(v) - a q(v)) / W_j for tokens not yet proposed
+    double ip = 1.0, iq = 1.0;   // 1 / sum of the cached exponentials: p(v) = pc[v] * ip, q(v) = qc[v] * iq
     bool bad_tree = false;
     for (;;) {
-        softmax_to_cache<T>(target + (size_t)cur * V, V, invT, pc, red, &nan_seen);
+        ip = softmax_to_cache<T>(target + (size_t)cur * V, v0, v1, invT, pc, red, &nan_seen);
         if (tid == 0) {
             int n = 0;
             for (int j = cur + 1; j < M; ++j)
@@ -182,7 +230,7 @@ __global__ void __launch_bounds__(kSThreads) stochastic_walk_kernel(const StochP
         if (nchild == 0 || len >= a.t_max) break;
         const int drow = s_drow[cur];
         if (drow < 0 || drow >= a.R) { bad_tree = true; break; }
-        softmax_to_cache<T>(draft + (size_t)drow * V, V, invT, qc, red, &nan_seen);
+        iq = softmax_to_cache<T>(draft + (size_t)drow * V, v0, v1, invT, qc, red, &nan_seen);
 
         double Wn = 1.0, cq = 1.0;
         int accepted = -1;
@@ -190,7 +238,7 @@ __global__ void __launch_bounds__(kSThreads) stochastic_walk_kernel(const StochP
             const int j = s_child[ci];
             const int x = s_tok[j];
             if (x < 0 || x >= V) { bad_tree = true; break; }
-            const double px = pc[x], qx = qc[x];
+            const double px = pc[x] * ip, qx = qc[x] * iq;
             const double pj = fmax(0.0, px - a_coef * qx) / Wn;      // x has not been proposed before
             const double qj = cq * qx;
             bool acc;
@@ -203,12 +251,13 @@ __global__ void __launch_bounds__(kSThreads) stochastic_walk_kernel(const StochP
             // reject: one pass for the new residual mass
             const double a_new = a_coef + cq * Wn;
             double g = 0.0;
-            for (int v = tid; v < V; v += kSThreads) g += fmax(0.0, pc[v] - a_new * qc[v]);
+            for (int v = v0 + tid; v < v1; v += kSThreads) g += fmax(0.0, pc[v] * ip - a_new * (qc[v] * iq));
             g = red.sum(g);
             // tokens rejected earlier keep their own coefficient: swap their terms
             for (int r = 0; r < n_rej; ++r) {
                 const int xr = s_rx[r];
-                g += fmax(0.0, pc[xr] - s_ra[r] * qc[xr]) - fmax(0.0, pc[xr] - a_new * qc[xr]);
+                const double pr = pc[xr] * ip, qr = qc[xr] * iq;
+                g += fmax(0.0, pr - s_ra[r] * qr) - fmax(0.0, pr - a_new * qr);
             }
             double frozen = a_coef;
             if (g > 0.0) { a_coef = a_new; Wn = g; frozen = a_new; }   // else: residual empty, p stays as it is
@@ -223,29 +272,30 @@ __global__ void __launch_bounds__(kSThreads) stochastic_walk_kernel(const StochP
         if (bad_tree || accepted < 0) break;
         cur = accepted;
         ++len;
-        if (tid == 0) { pn[len] = cur; pt[len] = s_tok[cur]; }
+        if (lead && tid == 0) { pn[len] = cur; pt[len] = s_tok[cur]; }
     }
 
     // ---- final draw: inverse CDF over w(v) = max(0, p(v) - a(v) q(v)) (or p(v) when nothing was rejected) ----
-    const int per = (V + kSThreads - 1) / kSThreads;
-    const int v0 = min(tid * per, V), v1 = min(v0 + per, V);
+    const int nv = v1 - v0;
+    const int per = (nv + kSThreads - 1) / kSThreads;
+    const int t0 = v0 + min(tid * per, nv), t1 = v0 + min(tid * per + per, nv);
     auto weight = [&](int v) -> double {
-        if (n_rej == 0) return pc[v];
+        if (n_rej == 0) return pc[v] * ip;
         double av = a_coef;
         for (int r = 0; r < n_rej; ++r)
             if (s_rx[r] == v) av = s_ra[r];
-        return fmax(0.0, pc[v] - av * qc[v]);
+        return fmax(0.0, pc[v] * ip - av * (qc[v] * iq));
     };
     if (tid == 0) { s_pick = 0x7fffffff; s_last_pos = -1; }
     double seg = 0.0;
     int last_pos = -1;
-    for (int v = v0; v < v1; ++v) {
+    for (int v = t0; v < t1; ++v) {
         const double w = weight(v);
         seg += w;
         if (w > 0.0) last_pos = v;
     }
-    // scan of seg over threads (fp64).  A thread's end and its successor's start are the same
-    // expression, so exactly one thread owns the point u * total.
+    // scan of seg over the threads of this CTA (fp64).  A thread's end and its successor's start are the
+    // same expression, so at most one thread owns a point.
     double incl = seg;
     const int lane = tid & 31, warp = tid >> 5;
 #pragma unroll
@@ -258,41 +308,66 @@ __global__ void __launch_bounds__(kSThreads) stochastic_walk_kernel(const StochP
     __syncthreads();
     if (lane == 31) s_red[warp] = incl;
     __syncthreads();
-    double woff = 0.0, total = 0.0;
+    double woff = 0.0, slice_total = 0.0;
     for (int w = 0; w < kSThreads / 32; ++w) {
-        if (w == warp) woff = total;
-        total += s_red[w];
-    }
-    const double start = woff + excl, end = woff + incl;
-    const double tgt = (double)a.u_sample[b] * total;
-    if (last_pos >= 0) atomicMax(&s_last_pos, last_pos);
-    if (start <= tgt && tgt < end) {
-        double run = start;
-        int pick = last_pos;                                            // rounding guard: the crossing is in here
-        for (int v = v0; v < v1; ++v) {
-            run += weight(v);
-            if (run > tgt) { pick = v; break; }
-        }
-        atomicMin(&s_pick, pick);
+        if (w == warp) woff = slice_total;
+        slice_total += s_red[w];
     }
     __syncthreads();
-    if (tid == 0) {
-        int nt = s_pick != 0x7fffffff ? s_pick : s_last_pos;
-        a.next_token[b] = nt;
+    // slice totals of every CTA, in rank order: the running sum gives each slice's start, and the same
+    // expression is the previous slice's end
+    double tots[kMaxCluster];
+    red.all_gather(slice_total, tots);
+    double total = 0.0, my_start = 0.0;
+    for (unsigned r = 0; r < csize; ++r) {
+        if (r == crank) my_start = total;
+        total += tots[r];
+    }
+    const double tgt = (double)a.u_sample[b] * total;
+    // owner: the first slice whose end exceeds the point; if rounding leaves none, the last slice with mass
+    int owner = -1, last_live = 0;
+    {
+        double run = 0.0;
+        for (unsigned r = 0; r < csize; ++r) {
+            run += tots[r];
+            if (tots[r] > 0.0) last_live = (int)r;
+            if (owner < 0 && tgt < run) owner = (int)r;
+        }
+        if (owner < 0) owner = last_live;
+    }
+    if ((int)crank == owner) {
+        const double start = my_start + (woff + excl), end = my_start + (woff + incl);
+        if (last_pos >= 0) atomicMax(&s_last_pos, last_pos);
+        if (start <= tgt && tgt < end) {
+            double run = start;
+            int pick = last_pos;                                            // rounding guard: the crossing is in here
+            for (int v = t0; v < t1; ++v) {
+                run += weight(v);
+                if (run > tgt) { pick = v; break; }
+            }
+            if (pick >= 0) atomicMin(&s_pick, pick);
+        }
+        __syncthreads();
+        if (tid == 0) a.next_token[b] = s_pick != 0x7fffffff ? s_pick : s_last_pos;
+    }
+    if (lead && tid == 0) {
         a.accept_len[b] = len;
         if (bad_tree) set_status(P.status, RADAR_ERR_TREE);
     }
     if (nan_seen) set_status(P.status, RADAR_ERR_NUMERIC);
-    for (int dd = len + 1 + tid; dd < W; dd += kSThreads) { pn[dd] = -1; pt[dd] = -1; }
-    if (tid < 32) {
-        int best = 0x7fffffff;
-        const int nl = a.n_leaves[b];
-        for (int r = tid; r < nl; r += 32)
-            if (a.retrieve[((size_t)b * a.N + r) * W + len] == cur) best = min(best, r);
+    if (lead) {
+        for (int dd = len + 1 + tid; dd < W; dd += kSThreads) { pn[dd] = -1; pt[dd] = -1; }
+        if (tid < 32) {
+            int best = 0x7fffffff;
+            const int nl = a.n_leaves[b];
+            for (int r = tid; r < nl; r += 32)
+                if (a.retrieve[((size_t)b * a.N + r) * W + len] == cur) best = min(best, r);
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) best = min(best, __shfl_xor_sync(kFull, best, o));
-        if (tid == 0) a.best_retrieve_row[b] = best == 0x7fffffff ? -1 : best;
+            for (int o = 16; o > 0; o >>= 1) best = min(best, __shfl_xor_sync(kFull, best, o));
+            if (tid == 0) a.best_retrieve_row[b] = best == 0x7fffffff ? -1 : best;
+        }
     }
+    ClusterRed::cluster_sync();                   // no CTA leaves while another may still store into its shared memory
 }
 
 }  // namespace
@@ -357,10 +432,25 @@ extern "C" int radar_verify_accept(radar_ctx* ctx, const radar_accept_args* a, v
     sp.q_cache = reinterpret_cast<double*>(reinterpret_cast<char*>(a->workspace) +
                                            align_up((size_t)a->B * a->V * sizeof(double), 256));
     sp.status = ctx->d_status;
+    // cluster size: as many CTAs per sequence as keep the whole batch resident at once (at most 8)
+    int cs = 1;
+    while (cs < kMaxCluster && (long long)a->B * cs * 2 <= ctx->sm_count) cs *= 2;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(a->B * cs));
+    cfg.blockDim = dim3(kSThreads);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeClusterDimension;
+    attr.val.clusterDim.x = (unsigned)cs;
+    attr.val.clusterDim.y = 1;
+    attr.val.clusterDim.z = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
     {
         radar_launch_scope scope(ctx, RADAR_K_STOCH_WALK, stream);
-        if (a->logits_dtype == RADAR_F32) stochastic_walk_kernel<float><<<a->B, kSThreads, 0, stream>>>(sp);
-        else stochastic_walk_kernel<__nv_bfloat16><<<a->B, kSThreads, 0, stream>>>(sp);
+        if (a->logits_dtype == RADAR_F32) RADAR_CUDA_CHECK(cudaLaunchKernelEx(&cfg, stochastic_walk_kernel<float>, sp));
+        else RADAR_CUDA_CHECK(cudaLaunchKernelEx(&cfg, stochastic_walk_kernel<__nv_bfloat16>, sp));
     }
     RADAR_CUDA_CHECK(cudaGetLastError());
     return RADAR_OK;
