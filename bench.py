@@ -30,9 +30,15 @@ from paper_2512_14069_b200 import workloads as W  # noqa: E402
 
 METRIC, UNIT = "tree_verify_steps_per_s", "steps/s"
 L2_BYTES = 126 * 1024 * 1024
-# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under profiles/
-# (kernel name, config id) -> bytes; absent = not captured.
-NCU_TRAFFIC = {}
+# (dram__bytes_read.sum + dram__bytes_write.sum) / algorithmic bytes of the captured launch, from the ncu
+# captures summarised under profiles/ (kernel name, config id); traffic of a launch at the same shapes =
+# ratio x its algorithmic bytes (both grow with the rows processed).  Absent = not captured.
+NCU_TRAFFIC_RATIO = {
+    ("tree_attention", 4): 450.52 / 284.58,
+    ("tree_attention", 3): 352.84 / 343.57,
+    ("vocab_pass(expand)", 4): 35.947 / 35.912,
+    ("vocab_pass(accept)", 4): 228.65 / 224.70,
+}
 
 
 def parse():
@@ -146,6 +152,8 @@ def roofline_entry(name, k, peaks, traffic):
     """Roofline object of one kernel from its event-timed duration: the binding roof is the one that
     needs more time (bytes / HBM peak against flops / bf16 peak)."""
     us = k["avg_us"]
+    if traffic is not None:
+        traffic = traffic * k["alg_bytes_per_launch"]
     t_hbm = k["alg_bytes_per_launch"] / (peaks["hbm_gbs"] * 1e9)
     t_tensor = (k["tflops"] * us * 1e-6 * 1e12) / (peaks["bf16_tflops"] * 1e12) if "tflops" in k else 0.0
     if t_tensor > t_hbm:
@@ -210,15 +218,15 @@ def scale_probe(ctx, dev, peaks, reps=20):
     shapes = "LLaMA-3.3-70B shapes: B=8, Hq/Hkv/d=64/8/128, prefix 8192, V=128256, k=10, %d..%d tree rows" % (n_nodes.min(), n_nodes.max())
     out = []
     ka = {"avg_us": us_attn, "alg_bytes_per_launch": kv_bytes, "gbs": kv_bytes / us_attn / 1e3, "tflops": flops / us_attn / 1e6}
-    out.append(roofline_entry("tree_attention", ka, peaks, NCU_TRAFFIC.get(("tree_attention", 4))))
+    out.append(roofline_entry("tree_attention", ka, peaks, NCU_TRAFFIC_RATIO.get(("tree_attention", 4))))
     b_acc = float(n_nodes.sum()) * V * 4
     out.append(roofline_entry("vocab_pass(accept)", {"avg_us": us_acc, "alg_bytes_per_launch": b_acc,
                                                      "gbs": b_acc / us_acc / 1e3}, peaks,
-                              NCU_TRAFFIC.get(("vocab_pass(accept)", 4))))
+                              NCU_TRAFFIC_RATIO.get(("vocab_pass(accept)", 4))))
     b_exp = float(B * k * V * 4)
     out.append(roofline_entry("vocab_pass(expand)", {"avg_us": us_exp, "alg_bytes_per_launch": b_exp,
                                                      "gbs": b_exp / us_exp / 1e3}, peaks,
-                              NCU_TRAFFIC.get(("vocab_pass(expand)", 4))))
+                              NCU_TRAFFIC_RATIO.get(("vocab_pass(expand)", 4))))
     other = {n: round(v, 2) for n, v in ks.items() if n not in ("tree_attention", "vocab_pass(accept)", "vocab_pass(expand)")}
     for o in out:
         o["workload"] = shapes
@@ -433,7 +441,7 @@ def run_ours(args):
     dom_overall = max(timed, key=lambda n: timed[n][1]) if timed else None
     roofline = None
     if dom is not None:
-        roofline = roofline_entry(dom, kernels[dom], peaks, NCU_TRAFFIC.get((dom, cfg.cid)))
+        roofline = roofline_entry(dom, kernels[dom], peaks, NCU_TRAFFIC_RATIO.get((dom, cfg.cid)))
         roofline["dominant_overall"] = dom_overall
         if dom_overall != dom:
             roofline["note"] = ("%s has the largest share of device time (%.0f %%) but is a latency-bound per-sequence "

@@ -246,6 +246,37 @@ size_t radar_accept_workspace_bytes(const radar_ctx* ctx, int B, int V, int mode
 int radar_verify_accept(radar_ctx* ctx, const radar_accept_args* args, void* stream);
 
 /* ------------------------------------------------------------------------------------------
+ * radar_accept_length_distribution - acceptance-length distribution of a verified tree.
+ * (Sec. 4.3, Eq. 11-13: for node v with children l_1..l_n tried in order, P_acc(l_j | v) is the
+ * probability that l_1..l_{j-1} are rejected and l_j accepted under the sibling-sequential scheme of
+ * radar_verify_accept; P_rej(l | v) = 1 - sum_j P_acc(l_j | v); P_acc(v) is the product along v's
+ * path; P_stop(v) = P_acc(v) P_rej(l | v); p_i = sum of P_stop over the rows of depth i.)
+ *
+ * Inputs as for stochastic radar_verify_accept (target / draft logits, temperature, tree arrays)
+ * plus tree_depth; no uniforms: every internal row is evaluated, not only one sampled path.
+ * Outputs, fp64: dist[b][0..t_max] = p_0..p_tmax (sums to 1); p_acc_node[b][row] = P_acc(row)
+ * (rows >= n_nodes[b]: 0).  Probabilities are evaluated in fp64.
+ * Workspace: radar_acclen_workspace_bytes (two fp64 vocabulary rows per resident block).
+ */
+typedef struct {
+    int B, V, t_max;
+    float temperature;                  /* > 0 */
+    const void* target_logits;          /* [B][64][V] */
+    int logits_dtype;                   /* RADAR_F32 or RADAR_BF16 (both logits tensors) */
+    const int32_t *tree_tok, *tree_parent, *tree_depth, *tree_draft_row;   /* [B][64] */
+    const int32_t* n_nodes;             /* [B] */
+    const void* draft_logits;           /* [B][R][V] */
+    int R;
+    double* dist;                       /* [B][t_max+1] out */
+    double* p_acc_node;                 /* [B][64] out */
+    void* workspace;
+    size_t workspace_bytes;
+} radar_acclen_args;
+
+size_t radar_acclen_workspace_bytes(const radar_ctx* ctx, int B, int V);
+int radar_accept_length_distribution(radar_ctx* ctx, const radar_acclen_args* args, void* stream);
+
+/* ------------------------------------------------------------------------------------------
  * radar_verify_accept_greedy_noalloc - greedy acceptance that needs no workspace from the caller.
  * (The paper has no counterpart: this is a deployment variant of radar_verify_accept in greedy
  * mode, with the same inputs, outputs and results.)

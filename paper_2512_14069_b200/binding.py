@@ -70,6 +70,16 @@ class AcceptArgs(ctypes.Structure):
     ]
 
 
+class AccLenArgs(ctypes.Structure):
+    _fields_ = [
+        ("B", _c_int), ("V", _c_int), ("t_max", _c_int), ("temperature", _c_f),
+        ("target_logits", _vp), ("logits_dtype", _c_int),
+        ("tree_tok", _vp), ("tree_parent", _vp), ("tree_depth", _vp), ("tree_draft_row", _vp), ("n_nodes", _vp),
+        ("draft_logits", _vp), ("R", _c_int), ("dist", _vp), ("p_acc_node", _vp),
+        ("workspace", _vp), ("workspace_bytes", _sz),
+    ]
+
+
 _lib = None
 
 
@@ -104,6 +114,10 @@ def lib() -> ctypes.CDLL:
         L.radar_accept_workspace_bytes.argtypes = [_vp, _c_int, _c_int, _c_int]
         L.radar_verify_accept.restype = _c_int
         L.radar_verify_accept.argtypes = [_vp, ctypes.POINTER(AcceptArgs), _vp]
+        L.radar_acclen_workspace_bytes.restype = _sz
+        L.radar_acclen_workspace_bytes.argtypes = [_vp, _c_int, _c_int]
+        L.radar_accept_length_distribution.restype = _c_int
+        L.radar_accept_length_distribution.argtypes = [_vp, ctypes.POINTER(AccLenArgs), _vp]
         L.radar_profile_begin.restype = _c_int
         L.radar_profile_begin.argtypes = [_vp, _c_int]
         L.radar_profile_end.restype = _c_int
@@ -296,6 +310,28 @@ def radar_verify_accept(ctx: Context, *, B, V, t_max, N, mode, target_logits, tr
     a.next_token, a.best_retrieve_row = _ptr(next_token, i32), _ptr(best_retrieve_row, i32)
     a.workspace, a.workspace_bytes = _ptr(workspace), workspace.numel() * workspace.element_size()
     _check("radar_verify_accept", lib().radar_verify_accept(ctx.handle, ctypes.byref(a), _stream(stream)))
+
+
+def radar_acclen_workspace_bytes(ctx: Context, B, V) -> int:
+    return int(lib().radar_acclen_workspace_bytes(ctx.handle, B, V))
+
+
+def radar_accept_length_distribution(ctx: Context, *, B, V, t_max, temperature, target_logits, tree_tok, tree_parent,
+                                     tree_depth, tree_draft_row, n_nodes, draft_logits, R, dist, p_acc_node, workspace,
+                                     stream=None):
+    i32, f64 = torch.int32, torch.float64
+    a = AccLenArgs()
+    a.B, a.V, a.t_max, a.temperature = B, V, t_max, temperature
+    if draft_logits.dtype != target_logits.dtype:
+        raise ValueError("target and draft logits must share one dtype")
+    a.target_logits, a.logits_dtype = _ptr(target_logits), dtype_code(target_logits)
+    a.tree_tok, a.tree_parent = _ptr(tree_tok, i32), _ptr(tree_parent, i32)
+    a.tree_depth, a.tree_draft_row, a.n_nodes = _ptr(tree_depth, i32), _ptr(tree_draft_row, i32), _ptr(n_nodes, i32)
+    a.draft_logits, a.R = _ptr(draft_logits), R
+    a.dist, a.p_acc_node = _ptr(dist, f64), _ptr(p_acc_node, f64)
+    a.workspace, a.workspace_bytes = _ptr(workspace), workspace.numel() * workspace.element_size()
+    _check("radar_accept_length_distribution",
+           lib().radar_accept_length_distribution(ctx.handle, ctypes.byref(a), _stream(stream)))
 
 
 def radar_noalloc_scratch_bytes() -> int:

@@ -86,6 +86,8 @@ extern "C" const char* radar_kernel_name(int id) {
         case RADAR_K_VOCAB_ACCEPT: return "vocab_pass(accept)";
         case RADAR_K_GREEDY_WALK: return "greedy_walk";
         case RADAR_K_STOCH_WALK: return "stochastic_walk";
+        case RADAR_K_ACCLEN_NODES: return "accept_length_nodes";
+        case RADAR_K_ACCLEN_DIST: return "accept_length_dist";
         default: return "?";
     }
 }

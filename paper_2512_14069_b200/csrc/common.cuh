@@ -17,6 +17,8 @@ enum radar_kernel_id {
     RADAR_K_VOCAB_ACCEPT,       // row-argmax pass of greedy acceptance
     RADAR_K_GREEDY_WALK,
     RADAR_K_STOCH_WALK,
+    RADAR_K_ACCLEN_NODES,       // per-row conditional acceptance probabilities (Eq. 13)
+    RADAR_K_ACCLEN_DIST,        // path products and the length distribution (Eq. 11-12)
     RADAR_K_COUNT
 };
 

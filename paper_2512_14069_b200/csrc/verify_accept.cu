@@ -10,6 +10,8 @@
 //                q_j(x_i) = 0, with a_{j+1} = a_j + c_j W_j,  c_{j+1} = c_j / (1 - q_j(x_{j+1})) and
 //                W_{j+1} = sum_v max(0, p(v) - a(v) q(v)).  This is the rectify / remove / renormalise
 //                recursion of Eq. 2 unrolled, so each rejection costs one read-only pass.
+#include <algorithm>
+
 #include "common.cuh"
 
 namespace radar {
@@ -370,6 +372,131 @@ __global__ void __launch_bounds__(kSThreads) stochastic_walk_kernel(const StochP
     ClusterRed::cluster_sync();                   // no CTA leaves while another may still store into its shared memory
 }
 
+// ------------------------------------------------------------------------------------------
+// acceptance-length distribution (Eq. 11-13)
+// ------------------------------------------------------------------------------------------
+struct AccLenParams {
+    radar_acclen_args a;
+    double* p_cache;     // [grid][V]
+    double* q_cache;     // [grid][V]
+    double* cond;        // [B][64]: P_acc(row | its parent), in the workspace
+    int* status;
+};
+
+// One item = one tree row of one sequence; rows without children have nothing to do.  A persistent
+// grid walks the items; each block evaluates its row's children in order with the same closed-form
+// residual recursion as the stochastic walk, but follows every rejection branch: child j gets
+// reach_j a_j with reach_j = prod_{i<j} (1 - a_i).
+template <typename T>
+__global__ void __launch_bounds__(kSThreads) accept_length_nodes_kernel(const AccLenParams P) {
+    const radar_acclen_args& a = P.a;
+    const int tid = threadIdx.x, V = a.V;
+    __shared__ double s_red[32];
+    __shared__ double s_slots[2 * kMaxCluster];
+    __shared__ int s_tok[kMaxNodes], s_par[kMaxNodes];
+    __shared__ int s_rx[RADAR_MAX_NODES];
+    __shared__ double s_ra[RADAR_MAX_NODES];
+    ClusterRed red{s_red, s_slots, 0u, 1u, 0};       // launched without clusters: every block is its own
+    double* pc = P.p_cache + (size_t)blockIdx.x * V;
+    double* qc = P.q_cache + (size_t)blockIdx.x * V;
+    const double invT = 1.0 / (double)a.temperature;
+    bool nan_seen = false, bad_tree = false;
+
+    for (int item = blockIdx.x; item < a.B * kMaxNodes; item += gridDim.x) {
+        const int b = item / kMaxNodes, c = item % kMaxNodes;
+        const int M = min(max(a.n_nodes[b], 1), kMaxNodes);
+        if (c >= M) {
+            if (tid == 0) P.cond[item] = 0.0;
+            continue;
+        }
+        __syncthreads();                                  // previous item's readers are done with s_tok / s_par
+        if (tid < kMaxNodes) {
+            s_tok[tid] = tid < M ? a.tree_tok[(size_t)b * kMaxNodes + tid] : -1;
+            s_par[tid] = tid < M ? a.tree_parent[(size_t)b * kMaxNodes + tid] : -2;
+        }
+        __syncthreads();
+        if (c == 0 && tid == 0) P.cond[item] = 1.0;       // the root is always "accepted"
+        int nchild = 0;
+        for (int j = c + 1; j < M; ++j) nchild += s_par[j] == c ? 1 : 0;
+        if (nchild == 0) continue;
+        const int drow = a.tree_draft_row[(size_t)b * kMaxNodes + c];
+        if (drow < 0 || drow >= a.R) { bad_tree = true; continue; }
+        const T* target = reinterpret_cast<const T*>(a.target_logits) + ((size_t)b * kMaxNodes + c) * V;
+        const T* draft = reinterpret_cast<const T*>(a.draft_logits) + ((size_t)b * a.R + drow) * V;
+        const double ip = softmax_to_cache<T>(target, 0, V, invT, pc, red, &nan_seen);
+        const double iq = softmax_to_cache<T>(draft, 0, V, invT, qc, red, &nan_seen);
+
+        double a_coef = 0.0, Wn = 1.0, cq = 1.0, reach = 1.0;
+        int n_rej = 0;
+        bool exhausted = false;
+        for (int j = c + 1; j < M; ++j) {
+            if (s_par[j] != c) continue;
+            if (exhausted) {
+                if (tid == 0) P.cond[(size_t)b * kMaxNodes + j] = 0.0;
+                continue;
+            }
+            const int x = s_tok[j];
+            if (x < 0 || x >= V) { bad_tree = true; break; }
+            const double px = pc[x] * ip, qx = qc[x] * iq;
+            const double pj = fmax(0.0, px - a_coef * qx) / Wn;
+            const double qj = cq * qx;
+            double acc;
+            if (qj <= 0.0) acc = pj > 0.0 ? 1.0 : 0.0;
+            else { acc = pj / qj; if (acc > 1.0) acc = 1.0; }
+            if (tid == 0) P.cond[(size_t)b * kMaxNodes + j] = reach * acc;
+            reach *= 1.0 - acc;
+            // the rejection branch: new residual, x leaves the draft distribution
+            const double a_new = a_coef + cq * Wn;
+            double g = 0.0;
+            for (int v = tid; v < V; v += kSThreads) g += fmax(0.0, pc[v] * ip - a_new * (qc[v] * iq));
+            g = red.sum(g);
+            for (int r = 0; r < n_rej; ++r) {
+                const int xr = s_rx[r];
+                const double pr = pc[xr] * ip, qr = qc[xr] * iq;
+                g += fmax(0.0, pr - s_ra[r] * qr) - fmax(0.0, pr - a_new * qr);
+            }
+            double frozen = a_coef;
+            if (g > 0.0) { a_coef = a_new; Wn = g; frozen = a_new; }
+            __syncthreads();
+            if (tid == 0) { s_rx[n_rej] = x; s_ra[n_rej] = frozen; }
+            __syncthreads();
+            ++n_rej;
+            const double rest = 1.0 - qj;
+            if (rest <= 0.0) exhausted = true;
+            else cq = cq / rest;
+        }
+    }
+    if (nan_seen) set_status(P.status, RADAR_ERR_NUMERIC);
+    if (bad_tree && tid == 0) set_status(P.status, RADAR_ERR_TREE);
+}
+
+// one warp per sequence: P_acc along the paths (parents precede children), P_stop, p_i
+__global__ void __launch_bounds__(32) accept_length_dist_kernel(const AccLenParams P) {
+    const radar_acclen_args& a = P.a;
+    const int b = blockIdx.x, lane = threadIdx.x;
+    const int M = min(max(a.n_nodes[b], 1), kMaxNodes);
+    __shared__ double s_pacc[kMaxNodes], s_sum[kMaxNodes], s_dist[64];
+    for (int i = lane; i < kMaxNodes; i += 32) { s_pacc[i] = 0.0; s_sum[i] = 0.0; }
+    for (int i = lane; i < 64; i += 32) s_dist[i] = 0.0;
+    __syncwarp();
+    if (lane == 0) {
+        s_pacc[0] = 1.0;
+        for (int j = 1; j < M; ++j) {
+            const int par = a.tree_parent[(size_t)b * kMaxNodes + j];
+            const double cj = (par >= 0 && par < j) ? P.cond[(size_t)b * kMaxNodes + j] : 0.0;
+            s_pacc[j] = (par >= 0 && par < j ? s_pacc[par] : 0.0) * cj;
+            if (par >= 0 && par < j) s_sum[par] += cj;
+        }
+        for (int c = 0; c < M; ++c) {
+            const int dep = a.tree_depth[(size_t)b * kMaxNodes + c];
+            if (dep >= 0 && dep <= a.t_max) s_dist[dep] += s_pacc[c] * (1.0 - s_sum[c]);
+        }
+    }
+    __syncwarp();
+    for (int i = lane; i < kMaxNodes; i += 32) a.p_acc_node[(size_t)b * kMaxNodes + i] = s_pacc[i];
+    for (int i = lane; i <= a.t_max; i += 32) a.dist[(size_t)b * (a.t_max + 1) + i] = s_dist[i];
+}
+
 }  // namespace
 }  // namespace radar
 
@@ -451,6 +578,47 @@ extern "C" int radar_verify_accept(radar_ctx* ctx, const radar_accept_args* a, v
         radar_launch_scope scope(ctx, RADAR_K_STOCH_WALK, stream);
         if (a->logits_dtype == RADAR_F32) RADAR_CUDA_CHECK(cudaLaunchKernelEx(&cfg, stochastic_walk_kernel<float>, sp));
         else RADAR_CUDA_CHECK(cudaLaunchKernelEx(&cfg, stochastic_walk_kernel<__nv_bfloat16>, sp));
+    }
+    RADAR_CUDA_CHECK(cudaGetLastError());
+    return RADAR_OK;
+}
+
+static int acclen_grid(const radar_ctx* ctx, int B) { return std::min(B * kMaxNodes, ctx->sm_count); }
+
+extern "C" size_t radar_acclen_workspace_bytes(const radar_ctx* ctx, int B, int V) {
+    if (!ctx || B <= 0 || V <= 0) return 0;
+    return 2 * align_up((size_t)acclen_grid(ctx, B) * V * sizeof(double), 256) + align_up((size_t)B * kMaxNodes * sizeof(double), 256);
+}
+
+extern "C" int radar_accept_length_distribution(radar_ctx* ctx, const radar_acclen_args* a, void* stream_) {
+    if (!ctx || !a) return RADAR_ERR_INVALID_ARG;
+    cudaStream_t stream = reinterpret_cast<cudaStream_t>(stream_);
+    if (a->B <= 0 || a->V <= 0 || a->t_max < 1 || a->R < 1 || !(a->temperature > 0.f)) return RADAR_ERR_INVALID_ARG;
+    if (a->t_max >= 64) return RADAR_ERR_UNSUPPORTED;
+    if (a->logits_dtype != RADAR_F32 && a->logits_dtype != RADAR_BF16) return RADAR_ERR_UNSUPPORTED;
+    if (!a->target_logits || !a->draft_logits || !a->tree_tok || !a->tree_parent || !a->tree_depth || !a->tree_draft_row ||
+        !a->n_nodes || !a->dist || !a->p_acc_node || !a->workspace)
+        return RADAR_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(a->workspace) & 255) != 0) return RADAR_ERR_WORKSPACE;
+    if (radar_acclen_workspace_bytes(ctx, a->B, a->V) > a->workspace_bytes) return RADAR_ERR_WORKSPACE;
+    const int grid = acclen_grid(ctx, a->B);
+    AccLenParams P;
+    P.a = *a;
+    char* w = reinterpret_cast<char*>(a->workspace);
+    const size_t cache = align_up((size_t)grid * a->V * sizeof(double), 256);
+    P.p_cache = reinterpret_cast<double*>(w);
+    P.q_cache = reinterpret_cast<double*>(w + cache);
+    P.cond = reinterpret_cast<double*>(w + 2 * cache);
+    P.status = ctx->d_status;
+    {
+        radar_launch_scope scope(ctx, RADAR_K_ACCLEN_NODES, stream);
+        if (a->logits_dtype == RADAR_F32) accept_length_nodes_kernel<float><<<grid, kSThreads, 0, stream>>>(P);
+        else accept_length_nodes_kernel<__nv_bfloat16><<<grid, kSThreads, 0, stream>>>(P);
+    }
+    RADAR_CUDA_CHECK(cudaGetLastError());
+    {
+        radar_launch_scope scope(ctx, RADAR_K_ACCLEN_DIST, stream);
+        accept_length_dist_kernel<<<a->B, 32, 0, stream>>>(P);
     }
     RADAR_CUDA_CHECK(cudaGetLastError());
     return RADAR_OK;

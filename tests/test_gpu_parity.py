@@ -54,6 +54,41 @@ def test_whole_step_matches_oracle(ctx, cid):
     H.compare_accept(cfg, g, accepts)
 
 
+@pytest.mark.parametrize("cid,temperature", [(1, 1.0), (3, 1.0), (5, 0.7), (2, 0.5)])
+def test_accept_length_distribution_matches_oracle(ctx, cid, temperature):
+    """Eq. 11-13 for every tree of the batch: p_0..p_tmax and P_acc of every row against the fp64 oracle.
+    Both sides work in fp64 and differ only in summation order: 1e-9 absolute is generous."""
+    import torch
+    from oracle import accept_oracle as A
+    from paper_2512_14069_b200 import binding as rb
+    cfg = small(cid) if cid != 2 else W.shrink(W.CONFIGS[2], V=30011)
+    inp = H.make_inputs(cfg, with_attention=False)
+    pools, traces, trees = H.oracle_expand_and_tree(cfg, inp)
+    target = H.make_target(cfg, inp, trees)
+    g = H.GpuRun(cfg, inp, ctx)
+    g.expand_and_tree()
+    H.compare_tree(cfg, g, trees)
+    s = g.step
+    dist = torch.full((cfg.B, cfg.t_max + 1), -1.0, dtype=torch.float64, device="cuda")
+    pacc = torch.full((cfg.B, 64), -1.0, dtype=torch.float64, device="cuda")
+    wb = rb.radar_acclen_workspace_bytes(ctx, cfg.B, cfg.V)
+    ws = torch.zeros(wb + 256, dtype=torch.uint8, device="cuda")
+    off = (-ws.data_ptr()) % 256
+    rb.radar_accept_length_distribution(
+        ctx, B=cfg.B, V=cfg.V, t_max=cfg.t_max, temperature=float(np.float32(temperature)), target_logits=H.to_dev(target),
+        tree_tok=s.tree_tok, tree_parent=s.tree_parent, tree_depth=s.tree_depth, tree_draft_row=s.tree_draft_row,
+        n_nodes=s.n_nodes, draft_logits=g.draft, R=s.R, dist=dist, p_acc_node=pacc, workspace=ws[off:off + wb])
+    ctx.check_device_status()
+    dist, pacc = dist.cpu().numpy(), pacc.cpu().numpy()
+    for b in range(cfg.B):
+        d_ref, p_ref = A.accept_length_distribution(target[b], inp["draft"][b], trees[b], float(np.float32(temperature)),
+                                                    cfg.t_max)
+        n = trees[b]["n_nodes"]
+        assert np.max(np.abs(dist[b] - d_ref)) < 1e-9, (b, dist[b], d_ref)
+        assert np.max(np.abs(pacc[b, :n] - p_ref)) < 1e-9 and not pacc[b, n:].any()
+        assert abs(dist[b].sum() - 1.0) < 1e-9
+
+
 @pytest.mark.parametrize("cid", [1, 3])
 def test_bf16_logits_with_many_ties(ctx, cid):
     """bf16 logits collide often: token order must still be (value desc, id asc) bit for bit."""
