@@ -60,24 +60,41 @@ def parse():
 def host_inputs(cfg, rank):
     B = cfg.B
     gb = lambda b: rank * B + b
-    plen_all = W.prefix_lens(W.shrink(cfg, B=B * (rank + 1)))[rank * B:]
+    big = W.shrink(cfg, B=B * (rank + 1))          # the generators index per-sequence scalars by global sequence
+    plen_all = W.prefix_lens(big)[rank * B:]
     inp = {
-        "draft": np.stack([W.draft_logits(cfg, gb(b)) for b in range(B)]),
+        "draft": np.stack([W.draft_logits(big, gb(b)) for b in range(B)]),
         "gate": W.gate_weights(cfg),
-        "force_calls": None if cfg.depth_plan == "gate" else W.forced_calls(W.shrink(cfg, B=B * (rank + 1)))[rank * B:],
-        "n_keep": np.minimum(W.keep_sizes(W.shrink(cfg, B=B * (rank + 1)))[rank * B:], cfg.N).astype(np.int32),
-        "root_tok": W.root_tokens(W.shrink(cfg, B=B * (rank + 1)))[rank * B:],
+        "force_calls": None if cfg.depth_plan == "gate" else W.forced_calls(big)[rank * B:],
+        "n_keep": np.minimum(W.keep_sizes(big)[rank * B:], cfg.N).astype(np.int32),
+        "root_tok": W.root_tokens(big)[rank * B:],
         "prefix_len": plen_all.astype(np.int32),
-        "Q": np.stack([W.attn_q(cfg, gb(b)) for b in range(B)]),
+        "Q": np.stack([W.attn_q(big, gb(b)) for b in range(B)]),
     }
-    kt, vt = zip(*[W.attn_tree_kv(cfg, gb(b)) for b in range(B)])
+    kt, vt = zip(*[W.attn_tree_kv(big, gb(b)) for b in range(B)])
     inp["Kt"], inp["Vt"] = np.stack(kt), np.stack(vt)
-    kc, vc = zip(*[W.attn_prefix_kv(cfg, gb(b), int(plen_all[b])) for b in range(B)])
+    kc, vc = zip(*[W.attn_prefix_kv(big, gb(b), int(plen_all[b])) for b in range(B)])
     inp["Kc"], inp["Vc"] = np.concatenate(kc, 0), np.concatenate(vc, 0)
     inp["kv_start"] = np.concatenate([[0], np.cumsum(plen_all)[:-1]]).astype(np.int64)
-    ua, us = W.accept_uniforms(W.shrink(cfg, B=B * (rank + 1)))
+    ua, us = W.accept_uniforms(big)
     inp["u_accept"], inp["u_sample"] = ua[rank * B:], us[rank * B:]
+    inp["big"] = big
     return inp
+
+
+def reduce_max(values, device):
+    """Max over the ranks of each value (the slowest rank defines a multi-GPU time)."""
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor(values, dtype=torch.float64, device=device)
+    if dist.is_available() and dist.is_initialized() and dist.get_world_size() > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(x) for x in t]
+
+
+def whole_job_value(world, steps, ms_total):
+    """Steps per second of the whole job: every rank runs `steps` steps of its own sequences in `ms_total`."""
+    return world * steps * 1000.0 / ms_total
 
 
 def torch_of(x):
@@ -276,7 +293,7 @@ def run_ours(args):
     n_nodes = step.n_nodes.cpu().numpy()
     drow = step.tree_draft_row.cpu().numpy()
     calls = np.array([int((step.pool_len[b].item() - k) // (k * k)) + 1 for b in range(B)])
-    inp["target"] = np.stack([W.target_logits(cfg, rank * B + b, inp["draft"][b], drow[b], int(n_nodes[b]))
+    inp["target"] = np.stack([W.target_logits(inp["big"], rank * B + b, inp["draft"][b], drow[b], int(n_nodes[b]))
                               for b in range(B)])
     del d0
 
@@ -399,12 +416,9 @@ def run_ours(args):
             e2e_step()
         e2e_s = time.perf_counter() - t0
 
-    t = torch.tensor([ms_total, e2e_s], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_total, e2e_s = float(t[0]), float(t[1])
+    ms_total, e2e_s = reduce_max([ms_total, e2e_s], dev)
     ms_per_step = ms_total / args.steps
-    value = world * 1000.0 / ms_per_step
+    value = whole_job_value(world, args.steps, ms_total)
     tree_rows = int(n_nodes.sum())
 
     # ---- roofline of the dominant kernel ----
