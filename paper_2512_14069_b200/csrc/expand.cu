@@ -86,9 +86,9 @@ __global__ void __launch_bounds__(kSelThreads, 1) expand_select_gate_kernel(cons
         }
         for (int f = warp; f < F; f += kMergeWarps) {
             const size_t row = row0 + f;
-            // log-sum-exp over the chunks in fp64 (loads first: they overlap the merge below)
-            float mloc = -CUDART_INF_F;
-            for (int c = lane; c < n_chunks; c += 32) mloc = fmaxf(mloc, P.vp.part_m[row * n_chunks + c]);
+            // log-sum-exp over the chunks in fp64: the first loads are issued here and consumed after the merge
+            const float pm0 = lane < n_chunks ? P.vp.part_m[row * n_chunks + lane] : -CUDART_INF_F;
+            const float ps0 = lane < n_chunks ? P.vp.part_s[row * n_chunks + lane] : 0.f;
             WarpTopList<float> top;
             top.reset();
             bool merged = false;
@@ -103,12 +103,26 @@ __global__ void __launch_bounds__(kSelThreads, 1) expand_select_gate_kernel(cons
                 s_rv[warp][lane] = -CUDART_INF_F;
                 s_ri[warp][lane] = 0x7fffffff;
                 __syncwarp();
-                for (int c = lane; c < n_chunks; c += 32) {
-                    const float hv = pv[c * k];
-                    const int hi = pi[c * k];
+                if (n_chunks <= 32) {
+                    // lane c holds the head of chunk c; its rank among the heads by 32 shuffles
+                    const float hv = lane < n_chunks ? pv[lane * k] : -CUDART_INF_F;
+                    const int hi = lane < n_chunks ? pi[lane * k] : 0x7fffffff;
                     int rank = 0;
-                    for (int o = 0; o < n_chunks; ++o) rank += precedes(pv[o * k], pi[o * k], hv, hi) ? 1 : 0;
-                    if (rank == k - 1) { s_tv[warp] = hv; s_ti[warp] = hi; }
+#pragma unroll
+                    for (int o = 0; o < 32; ++o) {
+                        const float ov = __shfl_sync(kFull, hv, o);
+                        const int oi = __shfl_sync(kFull, hi, o);
+                        rank += precedes(ov, oi, hv, hi) ? 1 : 0;
+                    }
+                    if (lane < n_chunks && rank == k - 1) { s_tv[warp] = hv; s_ti[warp] = hi; }
+                } else {
+                    for (int c = lane; c < n_chunks; c += 32) {
+                        const float hv = pv[c * k];
+                        const int hi = pi[c * k];
+                        int rank = 0;
+                        for (int o = 0; o < n_chunks; ++o) rank += precedes(pv[o * k], pi[o * k], hv, hi) ? 1 : 0;
+                        if (rank == k - 1) { s_tv[warp] = hv; s_ti[warp] = hi; }
+                    }
                 }
                 __syncwarp();
                 const float tv = s_tv[warp];
@@ -163,9 +177,11 @@ __global__ void __launch_bounds__(kSelThreads, 1) expand_select_gate_kernel(cons
                     }
                 }
             }
+            float mloc = pm0;
+            for (int c = lane + 32; c < n_chunks; c += 32) mloc = fmaxf(mloc, P.vp.part_m[row * n_chunks + c]);
             const float M = warp_max(mloc);
-            double sloc = 0.0;
-            for (int c = lane; c < n_chunks; c += 32) {
+            double sloc = pm0 > -CUDART_INF_F ? (double)ps0 * exp((double)pm0 - (double)M) : 0.0;
+            for (int c = lane + 32; c < n_chunks; c += 32) {
                 const float mc = P.vp.part_m[row * n_chunks + c];
                 if (mc > -CUDART_INF_F) sloc += (double)P.vp.part_s[row * n_chunks + c] * exp((double)mc - (double)M);
             }

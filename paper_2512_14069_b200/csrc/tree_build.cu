@@ -1,5 +1,6 @@
-// radar_rerank_build_tree: one block per sequence sorts the pool's (score desc, pool index asc) keys
-// with a shared-memory bitonic network, keeps the best n, compacts them in pool order with a block
+// radar_rerank_build_tree: one block per sequence finds the n best (score desc, pool index asc) keys of the
+// pool (threshold filter + rank count for pools of up to 1024 entries, a shared-memory bitonic network
+// beyond), keeps them, compacts them in pool order with a block
 // scan and derives parent rows, depths, position ids, ancestor masks, leaves and retrieve rows.
 #include "common.cuh"
 
@@ -25,13 +26,14 @@ __global__ void __launch_bounds__(kThreads) rerank_build_tree_kernel(const TreeP
     const radar_tree_args& a = P.a;
     extern __shared__ unsigned char smem_raw[];
     unsigned long long* s_key = reinterpret_cast<unsigned long long*>(smem_raw);        // [n2] sort keys
-    float* s_score = reinterpret_cast<float*>(smem_raw + (size_t)P.n2 * 8);              // [C]
-    short* s_node = reinterpret_cast<short*>(smem_raw + (size_t)P.n2 * 8 + (size_t)a.pool_capacity * 4);   // [C] tree row or 0
+    float* s_score = reinterpret_cast<float*>(smem_raw + (size_t)(P.n2 + 32) * 8);              // [C]
+    short* s_node = reinterpret_cast<short*>(smem_raw + (size_t)(P.n2 + 32) * 8 + (size_t)a.pool_capacity * 4);   // [C] tree row or 0
     __shared__ int s_warp_cnt[kThreads / 32];
     __shared__ int s_parent[kMaxNodes], s_depth[kMaxNodes], s_haschild[kMaxNodes], s_leaf_rank[kMaxNodes];
     __shared__ int s_nleaves;
 
     const int b = blockIdx.x;
+    const int n2_cap = P.n2 + 32;                                          // key array: n2 sort slots + 32 per-warp thresholds
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int C = a.pool_capacity;
     const size_t pb = (size_t)b * C;
@@ -45,26 +47,68 @@ __global__ void __launch_bounds__(kThreads) rerank_build_tree_kernel(const TreeP
     for (int i = tid; i < L; i += kThreads) s_score[i] = a.pool_score[pb + i];
     if (tid < kMaxNodes) { s_parent[tid] = -1; s_depth[tid] = 0; s_haschild[tid] = 0; }
     __syncthreads();
-    // smallest power of two that holds the live entries; the rest of the network is padding
-    int n2 = 2;
-    while (n2 < L) n2 <<= 1;
-    for (int i = tid; i < n2; i += kThreads) s_key[i] = i < L ? sort_key(s_score[i], i) : ~0ull;
     for (int i = tid; i < L; i += kThreads) s_node[i] = 0;
-    __syncthreads();
-    for (int size = 2; size <= n2; size <<= 1) {
-        for (int stride = size >> 1; stride > 0; stride >>= 1) {
-            for (int t = tid; t < (n2 >> 1); t += kThreads) {
-                const int lo = ((t & ~(stride - 1)) << 1) | (t & (stride - 1));
-                const int hi = lo | stride;
-                const bool up = (lo & size) == 0;
-                const unsigned long long x = s_key[lo], y = s_key[hi];
-                if ((x > y) == up) { s_key[lo] = y; s_key[hi] = x; }
+    if (L <= kThreads) {
+        // One key per thread, dealt out like cards (lane l of warp w holds pool entry 32 l + w) so that every warp
+        // sees all depths of the pool.  With j = ceil(n_eff / 32), the j-th best key of every warp, taken at its
+        // worst over the warps, has at least n_eff keys at or before it: those few are ranked by counting.
+        // If some warp holds fewer than j entries, every entry is a candidate.
+        const int mine = lane * 32 + warp;
+        const unsigned long long key = mine < L ? sort_key(s_score[mine], mine) : ~0ull;
+        const int jth = (n_eff + 31) / 32;
+        unsigned long long cur = key, best = ~0ull;
+        if (L / 32 >= jth) {
+            for (int r = 0; r < jth; ++r) {
+                best = cur;
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) best = min(best, __shfl_xor_sync(kFull, best, o));
+                if (cur == best) cur = ~0ull;                              // keys are distinct: one lane leaves
             }
-            __syncthreads();
         }
+        if (tid == 0) s_nleaves = 0;                                       // reused as the candidate counter
+        if (lane == 0) s_key[n2_cap - 32 + warp] = best;                   // tail of the key array: per-warp thresholds
+        __syncthreads();
+        unsigned long long thr = 0ull;
+        for (int w = 0; w < kThreads / 32; ++w) thr = max(thr, s_key[n2_cap - 32 + w]);
+        __syncthreads();
+        {   // one shared-memory atomic per warp, not per candidate
+            const bool cand = mine < L && key <= thr;
+            const unsigned m = __ballot_sync(kFull, cand);
+            int base = 0;
+            if (lane == 0 && m) base = atomicAdd(&s_nleaves, __popc(m));
+            base = __shfl_sync(kFull, base, 0);
+            if (cand) s_key[base + __popc(m & ((1u << lane) - 1u))] = key;
+        }
+        __syncthreads();
+        const int C = s_nleaves;                                           // <= L <= 1024 - 32 entries are free below the tail
+        for (int c = tid; c < C; c += kThreads) {
+            const unsigned long long kc = s_key[c];
+            int rank = 0;
+            for (int j = 0; j < C; ++j) rank += s_key[j] < kc ? 1 : 0;
+            if (rank < n_eff) s_node[(int)(kc & 0xffffffffu)] = 1;
+        }
+        __syncthreads();
+    } else {
+        // larger pools: bitonic network over the smallest power of two that holds the live entries
+        int n2 = 2;
+        while (n2 < L) n2 <<= 1;
+        for (int i = tid; i < n2; i += kThreads) s_key[i] = i < L ? sort_key(s_score[i], i) : ~0ull;
+        __syncthreads();
+        for (int size = 2; size <= n2; size <<= 1) {
+            for (int stride = size >> 1; stride > 0; stride >>= 1) {
+                for (int t = tid; t < (n2 >> 1); t += kThreads) {
+                    const int lo = ((t & ~(stride - 1)) << 1) | (t & (stride - 1));
+                    const int hi = lo | stride;
+                    const bool up = (lo & size) == 0;
+                    const unsigned long long x = s_key[lo], y = s_key[hi];
+                    if ((x > y) == up) { s_key[lo] = y; s_key[hi] = x; }
+                }
+                __syncthreads();
+            }
+        }
+        for (int p = tid; p < n_eff; p += kThreads) s_node[(int)(s_key[p] & 0xffffffffu)] = 1;
+        __syncthreads();
     }
-    for (int p = tid; p < n_eff; p += kThreads) s_node[(int)(s_key[p] & 0xffffffffu)] = 1;
-    __syncthreads();
 
     // each thread owns a contiguous run of pool entries so that the scan keeps pool order
     const int per = (L + kThreads - 1) / kThreads;
@@ -197,7 +241,7 @@ extern "C" int radar_rerank_build_tree(radar_ctx* ctx, const radar_tree_args* a,
     p.status = ctx->d_status;
     p.n2 = 2;
     while (p.n2 < a->pool_capacity) p.n2 <<= 1;
-    const size_t smem = (size_t)p.n2 * 8 + (size_t)a->pool_capacity * 6;
+    const size_t smem = (size_t)(p.n2 + 32) * 8 + (size_t)a->pool_capacity * 6;
     static size_t attr_smem = 48 * 1024;            // raised at most a few times per process
     if (smem > attr_smem) {
         RADAR_CUDA_CHECK(cudaFuncSetAttribute(rerank_build_tree_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
