@@ -433,9 +433,8 @@ def run_ours(args):
                               + 2 * n_nodes.sum() * cfg.Hq * cfg.d * kv_b),
     }
     attn_flops = float((4 * n_nodes * cfg.Hq * (plen + n_nodes) * cfg.d).sum())     # un-padded rows, QK^T + PV
-    if mode == rb.RADAR_STOCHASTIC:
-        alen = step.accept_len.cpu().numpy()
-        alg["stochastic_walk"] = int(((alen + 1) * 2 * V * s).sum())      # target + draft row of each visited node, once
+    # (the stochastic walk reads (accepted + 1) x 2 rows per sequence but is bound by fp64 exponentials and
+    # cluster barriers, not by bandwidth: it is listed in `kernels` without a roofline model)
     timed = {n: v for n, v in kstats.items() if v[2] > 0}
     peaks = measured_peaks()
     peak = peaks["hbm_gbs"]
