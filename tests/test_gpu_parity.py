@@ -130,6 +130,59 @@ def test_attention_with_oracle_masks_and_ragged_trees(ctx):
     H.compare_attention(cfg, O_gpu, lse_gpu, O_ref, lse_ref, trees)
 
 
+@pytest.mark.parametrize("Hq,Hkv,d", [(8, 8, 64), (8, 4, 64), (16, 1, 128), (6, 3, 128), (24, 8, 128)])
+def test_attention_bf16_head_layouts(ctx, Hq, Hkv, d):
+    """bf16 tensor-core path at head_dim 64 and 128, G = 1, 2 and 16 (eight row blocks), and G = 3, which the
+    tensor-core path does not take (falls to the FMA kernel): ragged prefixes incl. an empty one, ragged trees."""
+    cfg = W.shrink(W.CONFIGS[5], cid=80 + Hq + d, B=4, Hq=Hq, Hkv=Hkv, d=d, P=(0, 700), V=2000, k=4, t_max=5, N=50)
+    inp = H.make_inputs(cfg)
+    inp["prefix_len"][0] = 0
+    inp["Kc"][0], inp["Vc"][0] = inp["Kc"][0][:0], inp["Vc"][0][:0]
+    _, _, trees = H.oracle_expand_and_tree(cfg, inp)
+    trees[2] = dict(trees[2]); trees[2]["n_nodes"] = 1
+    g = H.GpuRun(cfg, inp, ctx)
+    g.upload_attention()
+    O_gpu, lse_gpu = g.attention(trees)
+    O_ref, lse_ref = H.oracle_attention(cfg, inp, trees)
+    H.compare_attention(cfg, O_gpu, lse_gpu, O_ref, lse_ref, trees)
+
+
+def test_attention_long_prefix_many_segments(ctx):
+    """One long and three short sequences: the long one's units are cut across many CTAs (partials + combine),
+    the short ones share CTAs with it."""
+    cfg = W.shrink(W.CONFIGS[5], cid=99, B=4, Hq=8, Hkv=2, P=(100, 100), V=2000, k=4, t_max=5, N=60)
+    inp = H.make_inputs(cfg)
+    long_len = 40000
+    inp["prefix_len"][1] = long_len
+    kc, vc = W.attn_prefix_kv(cfg, 1, long_len)
+    inp["Kc"][1], inp["Vc"][1] = kc, vc
+    _, _, trees = H.oracle_expand_and_tree(cfg, inp)
+    g = H.GpuRun(cfg, inp, ctx)
+    g.upload_attention()
+    O_gpu, lse_gpu = g.attention(trees)
+    O_ref, lse_ref = H.oracle_attention(cfg, inp, trees)
+    H.compare_attention(cfg, O_gpu, lse_gpu, O_ref, lse_ref, trees)
+
+
+def test_attention_reports_prefix_beyond_cache(ctx):
+    """A prefix that would read past the cache is refused on the device status word; nothing faults."""
+    import torch
+    from paper_2512_14069_b200 import binding as rb
+    cfg = W.shrink(W.CONFIGS[5], cid=98, B=2, Hq=8, Hkv=2, P=(300, 300), V=2000, k=4, t_max=4, N=30)
+    inp = H.make_inputs(cfg)
+    _, _, trees = H.oracle_expand_and_tree(cfg, inp)
+    g = H.GpuRun(cfg, inp, ctx, max_prefix_len=4096)
+    g.upload_attention()
+    g.prefix_len = H.to_dev(np.array([300, 4000], np.int32))          # sequence 1 claims more rows than the cache holds
+    s = g.step
+    mask = H.to_dev(np.stack([t["mask"] for t in trees]).view(np.int64))
+    n_nodes = H.to_dev(np.array([t["n_nodes"] for t in trees], np.int32))
+    s.attention(g.Q, g.Kc, g.Vc, g.kv_start, g.prefix_len, g.Kt, g.Vt, mask, n_nodes)
+    torch.cuda.synchronize()
+    assert ctx.read_device_status() == -1
+    assert ctx.read_device_status() == rb.RADAR_OK
+
+
 def test_attention_fp32_head_dim_64_and_128(ctx):
     for d in (64, 128):
         cfg = W.shrink(W.CONFIGS[1], cid=40 + d, B=2, Hq=4, Hkv=2, d=d, P=(257, 257))
