@@ -55,6 +55,30 @@ struct radar_launch_scope {
     }
 };
 
+// Every kernel of the library is launched with programmatic stream serialization and begins with
+// chain_wait(): the next kernel's launch and block scheduling overlap the tail of the previous one, and
+// nothing of a kernel touches memory before its predecessor (and, transitively, every earlier kernel of
+// the stream) has completed and flushed.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_chained(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                                  Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr.val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+__device__ __forceinline__ void chain_wait() {
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+
 #define RADAR_CUDA_CHECK(expr)                         \
     do {                                               \
         cudaError_t _e = (expr);                       \

@@ -40,6 +40,7 @@ __host__ __device__ inline size_t up16(size_t x) { return (x + 15) & ~(size_t)15
 // Phase 2 appends the candidates to the pool and selects the frontier; phase 3 finishes the LSTM cell
 // and the MLP head from shared memory only.
 __global__ void __launch_bounds__(kSelThreads, 1) expand_select_gate_kernel(const SelectParams P) {
+    chain_wait();
     const radar_expand_args& a = P.a;
     const int b = blockIdx.x;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -380,7 +381,7 @@ extern "C" int radar_expand_step(radar_ctx* ctx, const radar_expand_args* a, voi
     }
     {
         radar_launch_scope scope(ctx, RADAR_K_SELECT_GATE, stream);
-        expand_select_gate_kernel<<<a->B, kSelThreads, smem, stream>>>(sp);
+        RADAR_CUDA_CHECK(launch_chained(expand_select_gate_kernel, dim3(a->B), dim3(kSelThreads), smem, stream, sp));
     }
     RADAR_CUDA_CHECK(cudaGetLastError());
     return RADAR_OK;

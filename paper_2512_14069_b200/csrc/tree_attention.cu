@@ -51,6 +51,7 @@ template <> __device__ __forceinline__ void load16<__nv_bfloat16>(const __nv_bfl
 
 template <typename T, int D>
 __global__ void __launch_bounds__(kThreads) tree_attn_fp32_kernel(const AttnParams P) {
+    chain_wait();
     const radar_attn_args& a = P.a;
     constexpr int KS = D + 4;                       // padded K row: conflict-free 16-byte reads by 32 lanes
     extern __shared__ float smem[];
@@ -222,6 +223,7 @@ __global__ void __launch_bounds__(kThreads) tree_attn_fp32_kernel(const AttnPara
 // one warp per (sequence, query head, tree row): merge the KV splits
 template <typename T, int D>
 __global__ void __launch_bounds__(128) tree_attn_combine_kernel(const AttnParams P) {
+    chain_wait();
     const radar_attn_args& a = P.a;
     const int lane = threadIdx.x & 31;
     const int64_t item = (int64_t)blockIdx.x * 4 + (threadIdx.x >> 5);
@@ -286,13 +288,13 @@ int launch(radar_ctx* ctx, const AttnParams& P, cudaStream_t stream) {
     dim3 grid((unsigned)(rblocks * P.n_splits), (unsigned)a.Hkv, (unsigned)a.B);
     {
         radar_launch_scope scope(ctx, RADAR_K_ATTN, stream);
-        tree_attn_fp32_kernel<T, D><<<grid, kThreads, smem, stream>>>(P);
+        RADAR_CUDA_CHECK(launch_chained(tree_attn_fp32_kernel<T, D>, grid, dim3(kThreads), smem, stream, P));
     }
     RADAR_CUDA_CHECK(cudaGetLastError());
     const int64_t items = (int64_t)a.B * a.Hq * kMaxNodes;
     {
         radar_launch_scope scope(ctx, RADAR_K_ATTN_COMBINE, stream);
-        tree_attn_combine_kernel<T, D><<<(unsigned)((items + 3) / 4), 128, 0, stream>>>(P);
+        RADAR_CUDA_CHECK(launch_chained(tree_attn_combine_kernel<T, D>, dim3((unsigned)((items + 3) / 4)), dim3(128), 0, stream, P));
     }
     RADAR_CUDA_CHECK(cudaGetLastError());
     return RADAR_OK;

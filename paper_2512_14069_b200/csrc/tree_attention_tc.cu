@@ -154,6 +154,7 @@ __global__ void __launch_bounds__(kTcThreads, 1)
 tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmKc,
                     const __grid_constant__ CUtensorMap tmVc, const __grid_constant__ CUtensorMap tmKt,
                     const __grid_constant__ CUtensorMap tmVt, const TcParams P) {
+    chain_wait();
     using SM = Smem<D, TWO>;
     constexpr int H = SM::kHalves;
     constexpr int RK = SM::kRingK, RV = SM::kRingV;
@@ -642,6 +643,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
 // class hold the rest, each as its first segment.  One warp per query row, 8 rows per block.
 template <int D>
 __global__ void __launch_bounds__(256) tree_attn_tc_combine_kernel(const TcParams P) {
+    chain_wait();
     const radar_attn_args& a = P.a;
     const CutUnit cu = P.cut[blockIdx.x];
     if (!cu.valid) return;
@@ -793,13 +795,13 @@ static int launch_tc(radar_ctx* ctx, TcParams& P, cudaStream_t stream) {
     }
     {
         radar_launch_scope scope(ctx, RADAR_K_ATTN, stream);
-        tree_attn_tc_kernel<D, TWO><<<(unsigned)(P.n_cls * P.ncc), kTcThreads, Smem<D, TWO>::kDynamic, stream>>>(
-            tmQ, tmKc, tmVc, tmKt, tmVt, P);
+        RADAR_CUDA_CHECK(launch_chained(tree_attn_tc_kernel<D, TWO>, dim3((unsigned)(P.n_cls * P.ncc)), dim3(kTcThreads),
+                                        (size_t)Smem<D, TWO>::kDynamic, stream, tmQ, tmKc, tmVc, tmKt, tmVt, P));
     }
     RADAR_CUDA_CHECK(cudaGetLastError());
     {
         radar_launch_scope scope(ctx, RADAR_K_ATTN_COMBINE, stream);
-        tree_attn_tc_combine_kernel<D><<<dim3((unsigned)(P.n_cls * P.ncc), kPairRows / 8), 256, 0, stream>>>(P);
+        RADAR_CUDA_CHECK(launch_chained(tree_attn_tc_combine_kernel<D>, dim3((unsigned)(P.n_cls * P.ncc), kPairRows / 8), dim3(256), 0, stream, P));
     }
     RADAR_CUDA_CHECK(cudaGetLastError());
     return RADAR_OK;

@@ -23,6 +23,7 @@ __device__ __forceinline__ unsigned long long sort_key(float score, int idx) {
 }
 
 __global__ void __launch_bounds__(kThreads) rerank_build_tree_kernel(const TreeParams P) {
+    chain_wait();
     const radar_tree_args& a = P.a;
     extern __shared__ unsigned char smem_raw[];
     unsigned long long* s_key = reinterpret_cast<unsigned long long*>(smem_raw);        // [n2] sort keys
@@ -250,7 +251,7 @@ extern "C" int radar_rerank_build_tree(radar_ctx* ctx, const radar_tree_args* a,
     }
     {
         radar_launch_scope scope(ctx, RADAR_K_TREE_BUILD, stream);
-        rerank_build_tree_kernel<<<a->B, kThreads, smem, stream>>>(p);
+        RADAR_CUDA_CHECK(launch_chained(rerank_build_tree_kernel, dim3(a->B), dim3(kThreads), smem, stream, p));
     }
     RADAR_CUDA_CHECK(cudaGetLastError());
     return RADAR_OK;

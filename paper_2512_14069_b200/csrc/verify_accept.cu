@@ -26,6 +26,7 @@ struct GreedyParams {
 };
 
 __global__ void __launch_bounds__(64) greedy_walk_kernel(const GreedyParams P) {
+    chain_wait();
     const radar_accept_args& a = P.a;
     const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31;
     __shared__ int s_arg[kMaxNodes], s_tok[kMaxNodes], s_par[kMaxNodes];
@@ -174,6 +175,7 @@ __device__ double softmax_to_cache(const T* z, int v0, int v1, double invT, doub
 
 template <typename T>
 __global__ void __launch_bounds__(kSThreads) stochastic_walk_kernel(const StochParams P) {
+    chain_wait();
     const radar_accept_args& a = P.a;
     unsigned crank, csize;
     asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(crank));
@@ -389,6 +391,7 @@ struct AccLenParams {
 // reach_j a_j with reach_j = prod_{i<j} (1 - a_i).
 template <typename T>
 __global__ void __launch_bounds__(kSThreads) accept_length_nodes_kernel(const AccLenParams P) {
+    chain_wait();
     const radar_acclen_args& a = P.a;
     const int tid = threadIdx.x, V = a.V;
     __shared__ double s_red[32];
@@ -472,6 +475,7 @@ __global__ void __launch_bounds__(kSThreads) accept_length_nodes_kernel(const Ac
 
 // one warp per sequence: P_acc along the paths (parents precede children), P_stop, p_i
 __global__ void __launch_bounds__(32) accept_length_dist_kernel(const AccLenParams P) {
+    chain_wait();
     const radar_acclen_args& a = P.a;
     const int b = blockIdx.x, lane = threadIdx.x;
     const int M = min(max(a.n_nodes[b], 1), kMaxNodes);
@@ -546,7 +550,7 @@ extern "C" int radar_verify_accept(radar_ctx* ctx, const radar_accept_args* a, v
         RADAR_CUDA_CHECK(vocab_pass_launch(ctx, RADAR_K_VOCAB_ACCEPT, vp, stream));
         {
             radar_launch_scope scope(ctx, RADAR_K_GREEDY_WALK, stream);
-            greedy_walk_kernel<<<a->B, 64, 0, stream>>>(gp);
+            RADAR_CUDA_CHECK(launch_chained(greedy_walk_kernel, dim3(a->B), dim3(64), 0, stream, gp));
         }
         RADAR_CUDA_CHECK(cudaGetLastError());
         return RADAR_OK;
@@ -567,13 +571,15 @@ extern "C" int radar_verify_accept(radar_ctx* ctx, const radar_accept_args* a, v
     cfg.blockDim = dim3(kSThreads);
     cfg.dynamicSmemBytes = 0;
     cfg.stream = stream;
-    cudaLaunchAttribute attr;
-    attr.id = cudaLaunchAttributeClusterDimension;
-    attr.val.clusterDim.x = (unsigned)cs;
-    attr.val.clusterDim.y = 1;
-    attr.val.clusterDim.z = 1;
-    cfg.attrs = &attr;
-    cfg.numAttrs = 1;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = (unsigned)cs;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 2;
     {
         radar_launch_scope scope(ctx, RADAR_K_STOCH_WALK, stream);
         if (a->logits_dtype == RADAR_F32) RADAR_CUDA_CHECK(cudaLaunchKernelEx(&cfg, stochastic_walk_kernel<float>, sp));
@@ -612,13 +618,13 @@ extern "C" int radar_accept_length_distribution(radar_ctx* ctx, const radar_accl
     P.status = ctx->d_status;
     {
         radar_launch_scope scope(ctx, RADAR_K_ACCLEN_NODES, stream);
-        if (a->logits_dtype == RADAR_F32) accept_length_nodes_kernel<float><<<grid, kSThreads, 0, stream>>>(P);
-        else accept_length_nodes_kernel<__nv_bfloat16><<<grid, kSThreads, 0, stream>>>(P);
+        if (a->logits_dtype == RADAR_F32) RADAR_CUDA_CHECK(launch_chained(accept_length_nodes_kernel<float>, dim3(grid), dim3(kSThreads), 0, stream, P));
+        else RADAR_CUDA_CHECK(launch_chained(accept_length_nodes_kernel<__nv_bfloat16>, dim3(grid), dim3(kSThreads), 0, stream, P));
     }
     RADAR_CUDA_CHECK(cudaGetLastError());
     {
         radar_launch_scope scope(ctx, RADAR_K_ACCLEN_DIST, stream);
-        accept_length_dist_kernel<<<a->B, 32, 0, stream>>>(P);
+        RADAR_CUDA_CHECK(launch_chained(accept_length_dist_kernel, dim3(a->B), dim3(32), 0, stream, P));
     }
     RADAR_CUDA_CHECK(cudaGetLastError());
     return RADAR_OK;
@@ -712,7 +718,7 @@ extern "C" int radar_verify_accept_greedy_noalloc(radar_ctx* ctx, const radar_ac
     RADAR_CUDA_CHECK(vocab_pass_launch(ctx, RADAR_K_VOCAB_ACCEPT, vp, stream));
     {
         radar_launch_scope scope(ctx, RADAR_K_GREEDY_WALK, stream);
-        greedy_walk_kernel<<<a->B, 64, 0, stream>>>(gp);
+        RADAR_CUDA_CHECK(launch_chained(greedy_walk_kernel, dim3(a->B), dim3(64), 0, stream, gp));
     }
     RADAR_CUDA_CHECK(cudaGetLastError());
     return RADAR_OK;

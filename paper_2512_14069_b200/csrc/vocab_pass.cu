@@ -66,6 +66,7 @@ __device__ __forceinline__ void warp_best(float& v, int& i) {
 // EPT = values per thread kept in registers (a multiple of the vector width), chunk = kThreads * EPT
 template <typename T, int EPT, bool WANT_LSE>
 __global__ void __launch_bounds__(kThreads, WANT_LSE ? (EPT == 32 ? 5 : 6) : 5) vocab_pass_kernel(const VocabPassParams p) {
+    chain_wait();
     using VT = Vec<T>;
     constexpr int N = VT::N;
     constexpr int NV = EPT / N;
@@ -277,9 +278,9 @@ __global__ void __launch_bounds__(kThreads, WANT_LSE ? (EPT == 32 ? 5 : 6) : 5) 
 }
 
 template <typename T, bool WANT_LSE>
-void launch_ept(const VocabPassParams& p, unsigned grid, cudaStream_t stream) {
-    if (p.chunk / kThreads == 16) vocab_pass_kernel<T, 16, WANT_LSE><<<grid, kThreads, 0, stream>>>(p);
-    else vocab_pass_kernel<T, 32, WANT_LSE><<<grid, kThreads, 0, stream>>>(p);
+cudaError_t launch_ept(const VocabPassParams& p, unsigned grid, cudaStream_t stream) {
+    if (p.chunk / kThreads == 16) return launch_chained(vocab_pass_kernel<T, 16, WANT_LSE>, dim3(grid), dim3(kThreads), 0, stream, p);
+    return launch_chained(vocab_pass_kernel<T, 32, WANT_LSE>, dim3(grid), dim3(kThreads), 0, stream, p);
 }
 
 }  // namespace
@@ -313,14 +314,8 @@ cudaError_t vocab_pass_launch(radar_ctx* ctx, int kernel_id, const VocabPassPara
     if (grid == 0) return cudaSuccess;
     if (!p.want_lse && p.k != 1) return cudaErrorInvalidValue;
     radar_launch_scope scope(ctx, kernel_id, stream);
-    if (p.dtype == RADAR_F32) {
-        if (p.want_lse) launch_ept<float, true>(p, grid, stream);
-        else launch_ept<float, false>(p, grid, stream);
-    } else {
-        if (p.want_lse) launch_ept<__nv_bfloat16, true>(p, grid, stream);
-        else launch_ept<__nv_bfloat16, false>(p, grid, stream);
-    }
-    return cudaGetLastError();
+    if (p.dtype == RADAR_F32) return p.want_lse ? launch_ept<float, true>(p, grid, stream) : launch_ept<float, false>(p, grid, stream);
+    return p.want_lse ? launch_ept<__nv_bfloat16, true>(p, grid, stream) : launch_ept<__nv_bfloat16, false>(p, grid, stream);
 }
 
 }  // namespace radar
