@@ -78,6 +78,14 @@ __device__ __forceinline__ void chain_wait() {
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 }
+// The two halves, for kernels that do work that cannot depend on the predecessor before they wait for
+// it.  Rules that keep the chain sound: (1) every block runs chain_sync() in at least one thread
+// before it exits, so "kernel N complete" always implies "kernel N-1 complete"; (2) nothing written by
+// the immediate predecessor is read, and nothing it reads is written, before chain_sync() (or a block
+// barrier behind a thread that ran it).  Whatever kernels before the predecessor wrote is complete
+// when the block starts, because the predecessor's blocks trigger only after their own wait.
+__device__ __forceinline__ void chain_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void chain_sync() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
 #define RADAR_CUDA_CHECK(expr)                         \
     do {                                               \

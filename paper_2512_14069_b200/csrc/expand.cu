@@ -40,11 +40,15 @@ __host__ __device__ inline size_t up16(size_t x) { return (x + 15) & ~(size_t)15
 // Phase 2 appends the candidates to the pool and selects the frontier; phase 3 finishes the LSTM cell
 // and the MLP head from shared memory only.
 __global__ void __launch_bounds__(kSelThreads, 1) expand_select_gate_kernel(const SelectParams P) {
-    chain_wait();
+    // The predecessor is this call's vocabulary pass, whose blocks wait for everything before them:
+    // the previous call's state (active, h, c, pool_len) is complete when this block starts.  Only
+    // the chunk records need the pass itself, so the gate warps never wait for it.
+    chain_trigger();
     const radar_expand_args& a = P.a;
     const int b = blockIdx.x;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     if (a.t > 1 && a.active[b] == 0) {                 // call 1 always runs: it (re)starts every sequence
+        chain_sync();
         if (tid == 0) a.cont[b] = 0;
         return;
     }
@@ -80,6 +84,7 @@ __global__ void __launch_bounds__(kSelThreads, 1) expand_select_gate_kernel(cons
         const size_t row0 = (size_t)b * F;
         const float* gv = P.vp.part_v + row0 * per_row;
         const int* gi = P.vp.part_i + row0 * per_row;
+        chain_sync();
         if (P.staged) {
             for (int e = tid; e < F * per_row; e += kMergeWarps * 32) { cp_async4(st_v + e, gv + e); cp_async4(st_i + e, gi + e); }
             cp_async_wait_all();

@@ -38,9 +38,9 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 // time) or as soon as *abort is set by another thread.  Returns false on give-up and sets *abort.
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
                                           uint32_t limit = 4u << 20) {
-    if (*abort_flag) return false;
+    if (mbar_try_wait(bar, parity)) return !*abort_flag;
     for (uint32_t it = 0; it < limit; ++it) {
-        if (mbar_try_wait(bar, parity)) return true;
+        if (mbar_try_wait(bar, parity)) return !*abort_flag;
         if ((it & 63u) == 63u) {
             if (*abort_flag) return false;
             __nanosleep(64);
@@ -48,6 +48,13 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
     }
     *abort_flag = 1;
     return false;
+}
+// The same for a whole (converged) warp: one lane polls, the others learn the outcome from it, so that
+// the barrier word is not hit by 32 polls at a time.  `ok` chains earlier outcomes (false: do not wait).
+__device__ __forceinline__ bool mbar_wait_warp(bool ok, uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+    int r = 0;
+    if ((threadIdx.x & 31) == 0) r = ok && mbar_wait(bar, parity, abort_flag);
+    return __shfl_sync(0xffffffffu, r, 0) != 0;
 }
 
 // ---- proxies and fences -------------------------------------------------------------------------

@@ -154,7 +154,8 @@ __global__ void __launch_bounds__(kTcThreads, 1)
 tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmKc,
                     const __grid_constant__ CUtensorMap tmVc, const __grid_constant__ CUtensorMap tmKt,
                     const __grid_constant__ CUtensorMap tmVt, const TcParams P) {
-    chain_wait();
+    chain_trigger();                     // warp 0 waits for the predecessor below; the barrier, tensor-memory and
+                                         // descriptor set-up of the other warps needs nothing from global memory
     using SM = Smem<D, TWO>;
     constexpr int H = SM::kHalves;
     constexpr int RK = SM::kRingK, RV = SM::kRingV;
@@ -179,6 +180,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
 
     // ---- set-up: warp 0 finds this CTA's range while the barriers and tensor memory are prepared ----
     if (warp == 0) {
+        chain_sync();                    // every global access of the CTA comes after the block barrier below
         long long tot = 0;
         for (int b0 = 0; b0 < a.B; b0 += 32) {
             const int b = b0 + lane;
@@ -325,108 +327,118 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         __syncwarp();
     } else if (warp == kMmaWarp) {
         // =================================== MMA issuer ===================================
+        // One thread waits, issues and commits; a tcgen05.mma takes some 60 cycles to issue, about as long
+        // as a 128 x 128 x 16 product runs, so whatever else this thread executes between two of them
+        // costs tensor-pipe time: the issue sequences are straight-line with precomputed descriptor words.
+        // The other lanes follow the same control flow and only help to clear V rows (rare).
         constexpr uint32_t idesc_s128 = idesc_bf16_f32(128, kTileKeys, false, false);
         constexpr uint32_t idesc_s64 = idesc_bf16_f32(128, kTreeKeys, false, false);
         constexpr uint32_t idesc_pv = idesc_bf16_f32(128, D, false, true);
-        uint32_t kc = 0, vc = 0;                 // tiles taken from the rings
-        uint32_t sc[2] = {0, 0};                 // P tiles awaited per group
-        bool ok = true;
+        // high word of every shared-memory descriptor (stride between 8-row groups 1024 B, version, swizzle)
+        constexpr uint64_t kDescHi = (uint64_t)((1024u >> 4) | (1u << 14) | (2u << 29)) << 32;
+        const uint32_t q_lo = ((smem_u32(sQ) & 0x3ffff) >> 4) | (1u << 16);
+        const uint32_t k_lo = ((smem_u32(sK) & 0x3ffff) >> 4) | (1u << 16);
+        const uint32_t v_lo = (smem_u32(sV) & 0x3ffff) >> 4;
+        const bool lead = lane == 0;
+        uint32_t k_next = 0, k_par = 0, v_next = 0, v_par = 0;   // ring slot to take next and its phase parity
+        uint32_t pr0 = 0, pr1 = 0;               // P tiles awaited per group
+        bool ok = true;                          // meaningful in the leading lane only
         for (uint32_t seg = 0; cur.valid(); cur.next(P, pp), ++seg) {
             const int n = cur.t1 - cur.t0;
             const bool two = TWO && cur.two_rb();
             const int M = cur.s.M, Pb = cur.s.Pb, nt_unit = cur.s.nt;
-            ok = ok && mbar_wait(&bar_qfull, seg & 1, ab);
-            uint32_t k_slot = 0;                  // ring slot of the K tile in use (two row blocks share it)
-            // S for local tile i into group grp's buffer; fresh_k: take the next K tile from the ring
-            auto issue_s = [&](int i, int grp, bool fresh_k, bool release_k) {
-                if (fresh_k) {
-                    k_slot = kc % RK;
-                    ok = ok && mbar_wait(&bar_kfull[k_slot], (kc / RK) & 1, ab);
-                    ++kc;
-                }
-                tc_fence_after_sync();
-                if (lane == 0 && ok) {
-                    const bool tree = cur.t0 + i == nt_unit - 1;
-                    const int nk = tree ? kTreeKeys : kTileKeys;
-                    const uint32_t kbase = smem_u32(sK + k_slot * SM::kTileBytes);
-                    const uint32_t qbase = smem_u32(sQ) + (two ? grp : 0) * SM::kQBlock;
-#pragma unroll
-                    for (int kk = 0; kk < D / 16; ++kk) {
-                        const int h = kk >> 2, ko = (kk & 3) * 32;
-                        const uint64_t ad = smem_desc_sw128(qbase + h * (128 * 128) + ko, 16, 1024);
-                        const uint64_t bd = smem_desc_sw128(kbase + h * (nk * 128) + ko, 16, 1024);
-                        mma_ss(tmem + grp * 128, ad, bd, tree ? idesc_s64 : idesc_s128, kk > 0);
-                    }
-                    if (release_k) mma_commit(&bar_kempty[k_slot]);
-                    mma_commit(&bar_sfull[grp]);
-                }
-                __syncwarp();
-            };
-            uint32_t v_slot = 0;
-            // O[grp] (+)= P V for local tile i; fresh_v: take the next V tile; wait_free: first PV of the segment;
-            // fresh_acc: first PV of this group in the segment (overwrites the accumulator)
-            auto issue_pv = [&](int i, int grp, bool fresh_v, bool release_v, bool wait_free, bool fresh_acc, bool last) {
-                ok = ok && mbar_wait(&bar_pready[grp], sc[grp] & 1, ab);
-                ++sc[grp];
-                const bool tree = cur.t0 + i == nt_unit - 1;
-                const int nk = tree ? kTreeKeys : kTileKeys;
-                const int valid = tree ? M : min(kTileKeys, Pb - (cur.t0 + i) * kTileKeys);
-                const int ksteps = (valid + 15) >> 4;
-                if (fresh_v) {
-                    v_slot = vc % RV;
-                    ok = ok && mbar_wait(&bar_vfull[v_slot], (vc / RV) & 1, ab);
-                    ++vc;
-                    if (ok && valid < ksteps * 16) {
-                        // rows past the last live key meet P = 0; they must not hold NaN/Inf bit patterns
-                        unsigned char* vtile = sV + v_slot * SM::kTileBytes;
-                        const int nrows = ksteps * 16 - valid;
-                        for (int e = lane; e < nrows * 8 * H; e += 32) {
-                            const int h = e / (nrows * 8), rem = e % (nrows * 8);
-                            const int r = valid + rem / 8, c = rem % 8;
-                            *reinterpret_cast<uint4*>(vtile + h * (nk * 128) + r * 128 + c * 16) = make_uint4(0, 0, 0, 0);
+            if (lead) ok = ok && mbar_wait(&bar_qfull, seg & 1, ab);
+            uint32_t k_slot = 0, v_slot = 0;      // ring slots of the K and V tiles in use
+            bool acc0 = false, acc1 = false;      // accumulator holds a product of this segment
+            // Schedule.  Two live row blocks: group s owns row block s; per tile PV0(i) S0(i+1) PV1(i) S1(i+1),
+            // both groups sharing K(i+1) and V(i).  One live row block: the groups take alternate tiles,
+            // PV(i) S(i+2) for group i & 1.  S of the first tile(s) comes from the iterations with i < 0.
+            for (int i = two ? -1 : -2; i < n; ++i) {
+#pragma unroll 1
+                for (int qq = 0; qq < (two ? 2 : 1); ++qq) {
+                    const int q = two ? qq : (i & 1);
+                    if (i >= 0) {
+                        // ---- O[q] (+)= P V for tile i ----
+                        const bool tree = cur.t0 + i == nt_unit - 1;
+                        const int nk = tree ? kTreeKeys : kTileKeys;
+                        const int valid = tree ? M : min(kTileKeys, Pb - (cur.t0 + i) * kTileKeys);
+                        const int ksteps = (valid + 15) >> 4;
+                        if (lead) {
+                            ok = ok && mbar_wait(&bar_pready[q], (q ? pr1 : pr0) & 1, ab);
+                            if (q) ++pr1; else ++pr0;
                         }
-                        fence_proxy_async_smem();
-                        __syncwarp();
+                        if (!two || q == 0) {
+                            v_slot = v_next;
+                            if (lead) ok = ok && mbar_wait(&bar_vfull[v_slot], v_par, ab);
+                            if (++v_next == RV) { v_next = 0; v_par ^= 1; }
+                            if (valid < ksteps * 16) {
+                                // rows past the last live key meet P = 0; they must not hold NaN/Inf bit patterns
+                                __syncwarp();                                    // the tile has landed (leading lane waited)
+                                unsigned char* vtile = sV + v_slot * SM::kTileBytes;
+                                const int nrows = ksteps * 16 - valid;
+                                for (int e = lane; e < nrows * 8 * H; e += 32) {
+                                    const int h = e / (nrows * 8), rem = e % (nrows * 8);
+                                    const int r = valid + rem / 8, c = rem % 8;
+                                    *reinterpret_cast<uint4*>(vtile + h * (nk * 128) + r * 128 + c * 16) = make_uint4(0, 0, 0, 0);
+                                }
+                                fence_proxy_async_smem();
+                                __syncwarp();
+                            }
+                        }
+                        if (lead) {
+                            if (i == 0 && qq == 0) {      // the previous segment's epilogue has read both accumulators
+                                ok = ok && mbar_wait(&bar_ofree[0], (seg & 1) ^ 1, ab);
+                                ok = ok && mbar_wait(&bar_ofree[1], (seg & 1) ^ 1, ab);
+                            }
+                            tc_fence_after_sync();
+                            if (ok) {
+                                // V is consumed N-major: 16 keys are 2048 B; 64-column blocks are nk * 128 B apart
+                                const uint32_t b_lo = (v_lo + v_slot * (SM::kTileBytes >> 4)) | ((uint32_t)(nk * 128 >> 4) << 16);
+                                const uint32_t p_addr = tmem + q * 128;
+                                const uint32_t o_addr = tmem + 256 + q * 128;
+                                const bool acc = q ? acc1 : acc0;
+#pragma unroll
+                                for (int kk = 0; kk < kTileKeys / 16; ++kk)
+                                    if (kk < ksteps) mma_ts(o_addr, p_addr + kk * 8, kDescHi | (b_lo + kk * 128), idesc_pv, kk > 0 || acc);
+                                if (!two || q == 1) mma_commit(&bar_vempty[v_slot]);
+                                if (two ? i == n - 1 : i + 2 >= n) mma_commit(&bar_odone[q]);
+                            }
+                        }
+                        if (q) acc1 = true; else acc0 = true;
                     }
-                }
-                if (wait_free) {                  // the previous segment's epilogue has read both accumulators
-                    ok = ok && mbar_wait(&bar_ofree[0], (seg & 1) ^ 1, ab);
-                    ok = ok && mbar_wait(&bar_ofree[1], (seg & 1) ^ 1, ab);
-                }
-                tc_fence_after_sync();
-                if (lane == 0 && ok) {
-                    const uint32_t vbase = smem_u32(sV + v_slot * SM::kTileBytes);
-                    for (int kk = 0; kk < ksteps; ++kk) {
-                        const uint64_t bd = smem_desc_sw128(vbase + kk * 2048, nk * 128, 1024);
-                        mma_ts(tmem + 256 + grp * 128, tmem + grp * 128 + kk * 8, bd, idesc_pv, !fresh_acc || kk > 0);
+                    const int si = two ? i + 1 : i + 2;
+                    if (si >= 0 && si < n) {
+                        // ---- S = Q K^T for tile si into group q's buffer (one live row block: si & 1 == q) ----
+                        const bool fresh_k = !two || q == 0, release_k = !two || q == 1;
+                        if (fresh_k) {
+                            k_slot = k_next;
+                            if (lead) ok = ok && mbar_wait(&bar_kfull[k_slot], k_par, ab);
+                            if (++k_next == RK) { k_next = 0; k_par ^= 1; }
+                        }
+                        if (lead) {
+                            tc_fence_after_sync();
+                            if (ok) {
+                                const bool tree = cur.t0 + si == nt_unit - 1;
+                                const uint32_t a0 = q_lo + (two ? q : 0) * (SM::kQBlock >> 4);
+                                const uint32_t b0 = k_lo + k_slot * (SM::kTileBytes >> 4);
+                                const uint32_t b1 = b0 + ((uint32_t)((tree ? kTreeKeys : kTileKeys) * 128) >> 4);   // second 64-column block of K
+                                const uint32_t idesc = tree ? idesc_s64 : idesc_s128;
+                                const uint32_t d_addr = tmem + q * 128;
+#pragma unroll
+                                for (int kk = 0; kk < D / 16; ++kk) {
+                                    const uint32_t ko = (kk & 3) * 2;                 // 16 elements = 32 B within the 128-B row
+                                    mma_ss(d_addr, kDescHi | (a0 + (kk >> 2) * (128 * 128 >> 4) + ko), kDescHi | ((kk >> 2 ? b1 : b0) + ko), idesc, kk > 0);
+                                }
+                                if (release_k) mma_commit(&bar_kempty[k_slot]);
+                                mma_commit(&bar_sfull[q]);
+                            }
+                        }
                     }
-                    if (release_v) mma_commit(&bar_vempty[v_slot]);
-                    if (last) mma_commit(&bar_odone[grp]);
-                }
-                __syncwarp();
-            };
-            if (two) {
-                // both groups see every tile: S0(i) S1(i) share K(i), PV0(i) PV1(i) share V(i)
-                issue_s(0, 0, true, false);
-                issue_s(0, 1, false, true);
-                for (int i = 0; i < n; ++i) {
-                    issue_pv(i, 0, true, false, i == 0, i == 0, i == n - 1);
-                    if (i + 1 < n) issue_s(i + 1, 0, true, false);
-                    issue_pv(i, 1, false, true, false, i == 0, i == n - 1);
-                    if (i + 1 < n) issue_s(i + 1, 1, false, true);
-                }
-            } else {
-                // one live row block: the groups take alternate tiles
-                issue_s(0, 0, true, true);
-                if (n > 1) issue_s(1, 1, true, true);
-                for (int i = 0; i < n; ++i) {
-                    issue_pv(i, i & 1, true, true, i == 0, i < 2, i + 2 >= n);
-                    if (i + 2 < n) issue_s(i + 2, i & 1, true, true);
                 }
             }
-            if (lane == 0 && ok) mma_commit(&bar_qempty);     // every S of this segment has read Q
-            __syncwarp();
+            if (lead && ok) mma_commit(&bar_qempty);           // every S of this segment has read Q
         }
+        __syncwarp();
     } else {
         // =================================== softmax groups ===================================
         const int grp = warp >> 2;
