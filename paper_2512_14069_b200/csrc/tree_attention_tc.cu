@@ -652,7 +652,10 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
 
 // Merges the pieces of the units that were cut across CTAs.  Block (c, y): CTA c of the attention
 // kernel holds the first piece of a cut unit (or the block exits); the following CTAs of the same
-// class hold the rest, each as its first segment.  One warp per query row, 8 rows per block.
+// class hold the rest, each as its first segment.  A warp owns up to eight query rows
+// (y * 8 + warp + 32 r); it works out the unit's pieces once and fetches four rows at a time, every
+// piece of them in flight together.
+constexpr int kCombineY = 4;                 // blocks per cut unit: 4 * 8 warps * 8 rows = 256 rows
 template <int D>
 __global__ void __launch_bounds__(256) tree_attn_tc_combine_kernel(const TcParams P) {
     chain_wait();
@@ -662,60 +665,121 @@ __global__ void __launch_bounds__(256) tree_attn_tc_combine_kernel(const TcParam
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int pp = blockIdx.x % P.n_cls, c0 = blockIdx.x / P.n_cls;
     const long long u1 = cu.u0 + (long long)cu.nt * cu.w;
+    const int row0 = blockIdx.y * 8 + warp;
+    if (row0 >= cu.rows) return;                             // rows of a unit are live from 0 up
     // pieces: class-local CTAs c0, c0 + 1, ... while their range starts before the unit's end
     int n_pieces = 1;
     while (c0 + n_pieces < P.ncc && cu.tot * (c0 + n_pieces) / P.ncc < u1) ++n_pieces;
     const int G = P.G;
-    const int prow = blockIdx.y * 8 + warp;
-    if (prow >= cu.rows) return;                             // rows of a unit are live from 0 up
-    auto rec_of = [&](int j) {
+    constexpr int E = D / 32;                                // output elements per lane
+    auto rec_of = [&](int j) {                               // record of row 0 of piece j
         const int slot = j == 0 ? cu.slot : 0;
-        return ((int64_t)((c0 + j) * P.n_cls + pp) * 2 + slot) * kPairRows + prow;
+        return ((int64_t)((c0 + j) * P.n_cls + pp) * 2 + slot) * kPairRows;
     };
     auto live = [&](int j) {                                 // a CTA whose range holds no tile start has no piece
         return tiles_before(cu.tot * (c0 + j + 1) / P.ncc, cu.u0, cu.nt, cu.w) >
                tiles_before(cu.tot * (c0 + j) / P.ncc, cu.u0, cu.nt, cu.w);
     };
-    float den = 0.f, mx = -CUDART_INF_F, o[D / 32];
+    auto store_row = [&](int prow, const float (&o)[E], float mx, float den) {
+        const float inv = 1.f / den;
+        const int r_glob = pp * P.pair_rows + prow;
+        const int node = r_glob / G, hq = cu.g * G + r_glob % G;
+        __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(a.O) + (((int64_t)cu.b * kMaxNodes + node) * a.Hq + hq) * D + lane * E;
 #pragma unroll
-    for (int q = 0; q < D / 32; ++q) o[q] = 0.f;
-    // lane j holds piece j's (m, l); the accumulator rows of up to four pieces are fetched together
-    for (int j0 = 0; j0 < n_pieces; j0 += 32) {
-        const int jl = j0 + lane;
-        float2 ml = make_float2(-CUDART_INF_F, 0.f);
-        if (jl < n_pieces && live(jl)) ml = P.part_ml[rec_of(jl)];
-        const float mnew = fmaxf(mx, warp_max(ml.x));
-        if (mnew == -CUDART_INF_F) continue;
-        const float rescale = __expf(mx - mnew);             // 0 on the first live batch
-        den *= rescale;
+        for (int q = 0; q < E; q += 2) *reinterpret_cast<__nv_bfloat162*>(dst + q) = __floats2bfloat162_rn(o[q] * inv, o[q + 1] * inv);
+        if (a.lse != nullptr && lane == 0) a.lse[((int64_t)cu.b * a.Hq + hq) * kMaxNodes + node] = mx + logf(den);
+    };
+
+    if (n_pieces <= 4) {
+        // ---- the usual case: a unit spread over a few CTAs ----
+        int64_t rec[4];
+        bool on[4];
 #pragma unroll
-        for (int q = 0; q < D / 32; ++q) o[q] *= rescale;
-        mx = mnew;
-        const float wl = ml.x == -CUDART_INF_F ? 0.f : __expf(ml.x - mx);
-        den += warp_sum(ml.y * wl);
-        const int nb = min(32, n_pieces - j0);
-        for (int u0 = 0; u0 < nb; u0 += 4) {
-            float v[4][D / 32], w[4];
+        for (int j = 0; j < 4; ++j) { on[j] = j < n_pieces && live(j); rec[j] = rec_of(min(j, n_pieces - 1)); }
+        for (int rb = 0; rb < 8; rb += 4) {
+            if (row0 + 32 * rb >= cu.rows) break;
+            float2 ml[4][4];
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                w[u] = u0 + u < nb ? __shfl_sync(kFull, wl, u0 + u) : 0.f;
-                const float* src = P.part_o + rec_of(j0 + min(u0 + u, nb - 1)) * D + lane * (D / 32);
+            for (int r = 0; r < 4; ++r) {
+                const int prow = row0 + 32 * (rb + r);
 #pragma unroll
-                for (int q = 0; q < D / 32; ++q) v[u][q] = w[u] != 0.f ? src[q] : 0.f;
+                for (int j = 0; j < 4; ++j)
+                    ml[r][j] = on[j] && prow < cu.rows ? P.part_ml[rec[j] + prow] : make_float2(-CUDART_INF_F, 0.f);
+            }
+            float v[4][4][E];
+#pragma unroll
+            for (int r = 0; r < 4; ++r) {
+                const int prow = row0 + 32 * (rb + r);
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const bool take = on[j] && prow < cu.rows;
+                    const float* src = P.part_o + (rec[j] + (take ? prow : 0)) * D + lane * E;
+                    if (E == 4) {
+                        const float4 t = take ? *reinterpret_cast<const float4*>(src) : make_float4(0.f, 0.f, 0.f, 0.f);
+                        v[r][j][0] = t.x; v[r][j][1] = t.y; v[r][j][E - 2] = t.z; v[r][j][E - 1] = t.w;
+                    } else {
+                        const float2 t = take ? *reinterpret_cast<const float2*>(src) : make_float2(0.f, 0.f);
+                        v[r][j][0] = t.x; v[r][j][1] = t.y;
+                    }
+                }
             }
 #pragma unroll
-            for (int u = 0; u < 4; ++u)
+            for (int r = 0; r < 4; ++r) {
+                const int prow = row0 + 32 * (rb + r);
+                if (prow >= cu.rows) break;
+                const float mx = fmaxf(fmaxf(ml[r][0].x, ml[r][1].x), fmaxf(ml[r][2].x, ml[r][3].x));
+                float den = 0.f, o[E];
 #pragma unroll
-                for (int q = 0; q < D / 32; ++q) o[q] = fmaf(v[u][q], w[u], o[q]);
+                for (int q = 0; q < E; ++q) o[q] = 0.f;
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const float w = ml[r][j].x == -CUDART_INF_F ? 0.f : __expf(ml[r][j].x - mx);
+                    den = fmaf(ml[r][j].y, w, den);
+#pragma unroll
+                    for (int q = 0; q < E; ++q) o[q] = fmaf(v[r][j][q], w, o[q]);
+                }
+                store_row(prow, o, mx, den);
+            }
         }
+        return;
     }
-    const float inv = 1.f / den;
-    const int r_glob = pp * P.pair_rows + prow;
-    const int node = r_glob / G, hq = cu.g * G + r_glob % G;
-    __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(a.O) + (((int64_t)cu.b * kMaxNodes + node) * a.Hq + hq) * D + lane * (D / 32);
+
+    // ---- a unit spread over many CTAs (very long prefixes): one row at a time, lane j holds piece j's (m, l) ----
+    for (int prow = row0; prow < cu.rows; prow += 32) {
+        float den = 0.f, mx = -CUDART_INF_F, o[E];
 #pragma unroll
-    for (int q = 0; q < D / 32; ++q) dst[q] = __float2bfloat16(o[q] * inv);
-    if (a.lse != nullptr && lane == 0) a.lse[((int64_t)cu.b * a.Hq + hq) * kMaxNodes + node] = mx + logf(den);
+        for (int q = 0; q < E; ++q) o[q] = 0.f;
+        for (int j0 = 0; j0 < n_pieces; j0 += 32) {
+            const int jl = j0 + lane;
+            float2 ml = make_float2(-CUDART_INF_F, 0.f);
+            if (jl < n_pieces && live(jl)) ml = P.part_ml[rec_of(jl) + prow];
+            const float mnew = fmaxf(mx, warp_max(ml.x));
+            if (mnew == -CUDART_INF_F) continue;
+            const float rescale = __expf(mx - mnew);             // 0 on the first live batch
+            den *= rescale;
+#pragma unroll
+            for (int q = 0; q < E; ++q) o[q] *= rescale;
+            mx = mnew;
+            const float wl = ml.x == -CUDART_INF_F ? 0.f : __expf(ml.x - mx);
+            den += warp_sum(ml.y * wl);
+            const int nb = min(32, n_pieces - j0);
+            for (int u0 = 0; u0 < nb; u0 += 4) {
+                float v[4][E], w[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    w[u] = u0 + u < nb ? __shfl_sync(kFull, wl, u0 + u) : 0.f;
+                    const float* src = P.part_o + (rec_of(j0 + min(u0 + u, nb - 1)) + prow) * D + lane * E;
+#pragma unroll
+                    for (int q = 0; q < E; ++q) v[u][q] = w[u] != 0.f ? src[q] : 0.f;
+                }
+#pragma unroll
+                for (int u = 0; u < 4; ++u)
+#pragma unroll
+                    for (int q = 0; q < E; ++q) o[q] = fmaf(v[u][q], w[u], o[q]);
+            }
+        }
+        store_row(prow, o, mx, den);
+    }
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -813,7 +877,7 @@ static int launch_tc(radar_ctx* ctx, TcParams& P, cudaStream_t stream) {
     RADAR_CUDA_CHECK(cudaGetLastError());
     {
         radar_launch_scope scope(ctx, RADAR_K_ATTN_COMBINE, stream);
-        RADAR_CUDA_CHECK(launch_chained(tree_attn_tc_combine_kernel<D>, dim3((unsigned)(P.n_cls * P.ncc), kPairRows / 8), dim3(256), 0, stream, P));
+        RADAR_CUDA_CHECK(launch_chained(tree_attn_tc_combine_kernel<D>, dim3((unsigned)(P.n_cls * P.ncc), kCombineY), dim3(256), 0, stream, P));
     }
     RADAR_CUDA_CHECK(cudaGetLastError());
     return RADAR_OK;
