@@ -782,6 +782,74 @@ __global__ void __launch_bounds__(256) tree_attn_tc_combine_kernel(const TcParam
     }
 }
 
+// The same merge for launches with few cut units, where latency counts: block (c, y): CTA c of the attention
+// kernel holds the first piece of a cut unit (or the block exits); the following CTAs of the same
+// class hold the rest, each as its first segment.  One warp per query row, 8 rows per block.
+template <int D>
+__global__ void __launch_bounds__(256) tree_attn_tc_combine_wide_kernel(const TcParams P) {
+    chain_wait();
+    const radar_attn_args& a = P.a;
+    const CutUnit cu = P.cut[blockIdx.x];
+    if (!cu.valid) return;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int pp = blockIdx.x % P.n_cls, c0 = blockIdx.x / P.n_cls;
+    const long long u1 = cu.u0 + (long long)cu.nt * cu.w;
+    // pieces: class-local CTAs c0, c0 + 1, ... while their range starts before the unit's end
+    int n_pieces = 1;
+    while (c0 + n_pieces < P.ncc && cu.tot * (c0 + n_pieces) / P.ncc < u1) ++n_pieces;
+    const int G = P.G;
+    const int prow = blockIdx.y * 8 + warp;
+    if (prow >= cu.rows) return;                             // rows of a unit are live from 0 up
+    auto rec_of = [&](int j) {
+        const int slot = j == 0 ? cu.slot : 0;
+        return ((int64_t)((c0 + j) * P.n_cls + pp) * 2 + slot) * kPairRows + prow;
+    };
+    auto live = [&](int j) {                                 // a CTA whose range holds no tile start has no piece
+        return tiles_before(cu.tot * (c0 + j + 1) / P.ncc, cu.u0, cu.nt, cu.w) >
+               tiles_before(cu.tot * (c0 + j) / P.ncc, cu.u0, cu.nt, cu.w);
+    };
+    float den = 0.f, mx = -CUDART_INF_F, o[D / 32];
+#pragma unroll
+    for (int q = 0; q < D / 32; ++q) o[q] = 0.f;
+    // lane j holds piece j's (m, l); the accumulator rows of up to four pieces are fetched together
+    for (int j0 = 0; j0 < n_pieces; j0 += 32) {
+        const int jl = j0 + lane;
+        float2 ml = make_float2(-CUDART_INF_F, 0.f);
+        if (jl < n_pieces && live(jl)) ml = P.part_ml[rec_of(jl)];
+        const float mnew = fmaxf(mx, warp_max(ml.x));
+        if (mnew == -CUDART_INF_F) continue;
+        const float rescale = __expf(mx - mnew);             // 0 on the first live batch
+        den *= rescale;
+#pragma unroll
+        for (int q = 0; q < D / 32; ++q) o[q] *= rescale;
+        mx = mnew;
+        const float wl = ml.x == -CUDART_INF_F ? 0.f : __expf(ml.x - mx);
+        den += warp_sum(ml.y * wl);
+        const int nb = min(32, n_pieces - j0);
+        for (int u0 = 0; u0 < nb; u0 += 4) {
+            float v[4][D / 32], w[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                w[u] = u0 + u < nb ? __shfl_sync(kFull, wl, u0 + u) : 0.f;
+                const float* src = P.part_o + rec_of(j0 + min(u0 + u, nb - 1)) * D + lane * (D / 32);
+#pragma unroll
+                for (int q = 0; q < D / 32; ++q) v[u][q] = w[u] != 0.f ? src[q] : 0.f;
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+#pragma unroll
+                for (int q = 0; q < D / 32; ++q) o[q] = fmaf(v[u][q], w[u], o[q]);
+        }
+    }
+    const float inv = 1.f / den;
+    const int r_glob = pp * P.pair_rows + prow;
+    const int node = r_glob / G, hq = cu.g * G + r_glob % G;
+    __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(a.O) + (((int64_t)cu.b * kMaxNodes + node) * a.Hq + hq) * D + lane * (D / 32);
+#pragma unroll
+    for (int q = 0; q < D / 32; ++q) dst[q] = __float2bfloat16(o[q] * inv);
+    if (a.lse != nullptr && lane == 0) a.lse[((int64_t)cu.b * a.Hq + hq) * kMaxNodes + node] = mx + logf(den);
+}
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -877,7 +945,11 @@ static int launch_tc(radar_ctx* ctx, TcParams& P, cudaStream_t stream) {
     RADAR_CUDA_CHECK(cudaGetLastError());
     {
         radar_launch_scope scope(ctx, RADAR_K_ATTN_COMBINE, stream);
-        RADAR_CUDA_CHECK(launch_chained(tree_attn_tc_combine_kernel<D>, dim3((unsigned)(P.n_cls * P.ncc), kCombineY), dim3(256), 0, stream, P));
+        // few cut units: one row per warp and many small blocks; many: eight rows per warp, fewer waves of blocks
+        if ((long long)P.n_cls * P.ncc * (kPairRows / 8) <= 16ll * ctx->sm_count)
+            RADAR_CUDA_CHECK(launch_chained(tree_attn_tc_combine_wide_kernel<D>, dim3((unsigned)(P.n_cls * P.ncc), kPairRows / 8), dim3(256), 0, stream, P));
+        else
+            RADAR_CUDA_CHECK(launch_chained(tree_attn_tc_combine_kernel<D>, dim3((unsigned)(P.n_cls * P.ncc), kCombineY), dim3(256), 0, stream, P));
     }
     RADAR_CUDA_CHECK(cudaGetLastError());
     return RADAR_OK;
