@@ -182,6 +182,18 @@ def gate_step(x, h, c, w):
     return y, h_new, c_new
 
 
+def gate_step_mlp(x, w):
+    """The memoryless policy of the ablation (Table 3, "MLP / scores"; Sec. 4.2: it uses only the
+    confidence scores as its state).  The paper gives no layer sizes for it; the reading taken here is
+    the prediction model's own two-layer head without the LSTM in front: Linear(k -> H), ReLU,
+    Linear(H -> 2), with w["w1"] of shape [H, k].  Returns y[2]."""
+    x = np.asarray(x, np.float64)
+    W1, b1 = np.asarray(w["w1"], np.float64), np.asarray(w["b1"], np.float64)
+    W2, b2 = np.asarray(w["w2"], np.float64), np.asarray(w["b2"], np.float64)
+    assert W1.shape[1] == x.shape[0]
+    return W2 @ np.maximum(W1 @ x + b1, 0.0) + b2
+
+
 def gate_decision(y) -> bool:
     """Deterministic reading of the binary control signal: continue iff logit 1 wins."""
     return bool(y[1] > y[0]) if GATE_TIE_STOPS else bool(y[1] >= y[0])
@@ -190,7 +202,8 @@ def gate_decision(y) -> bool:
 # --------------------------------------------------------------------------
 # a4 loop: dynamic expansion for one sequence
 # --------------------------------------------------------------------------
-def run_expansion(draft_logits, k: int, t_max: int, gate_w, force_calls: int | None = None):
+def run_expansion(draft_logits, k: int, t_max: int, gate_w, force_calls: int | None = None,
+                  policy: str = "lstm_scores", features=None):
     """Draft-tree expansion for one sequence (Sec. 4.1; Eq. for T_pred).
 
     draft_logits [1+(t_max-1)k, V] float32: row 0 feeds call 1, rows
@@ -198,8 +211,14 @@ def run_expansion(draft_logits, k: int, t_max: int, gate_w, force_calls: int | N
     The gate runs after every call except call t_max (the paper drops that call
     because generation terminates anyway).  `force_calls` overrides the gate
     (used for workloads whose depth the harness fixes).
+    `policy` selects the ablation variants of Table 3: "lstm_scores" (the paper's model),
+    "mlp_scores" (gate_step_mlp; no recurrent state) and "lstm_hidden" (the same LSTM + head fed
+    with the draft model's hidden state of the call instead of the scores: `features`
+    [t_max-1, d_in] float32, row t-1 for call t; which hidden vector that is - the paper does not
+    say - is the caller's choice).
     Returns (pool, trace) where trace holds per-call outputs and margins.
     """
+    assert policy in ("lstm_scores", "mlp_scores", "lstm_hidden")
     H = GATE_HIDDEN
     pool = Pool(pool_capacity(k, t_max))
     h = np.zeros(H, np.float32)
@@ -216,8 +235,12 @@ def run_expansion(draft_logits, k: int, t_max: int, gate_w, force_calls: int | N
         if t < t_max:
             scores = out["frontier_score"] if GATE_INPUT_CUMULATIVE else out["frontier_local_logp"]
             x = np.exp(np.asarray(scores, np.float32).astype(np.float64))
-            y, h_new, c_new = gate_step(x, h, c, gate_w)
-            h, c = h_new.astype(np.float32), c_new.astype(np.float32)
+            if policy == "mlp_scores":
+                y = gate_step_mlp(x, gate_w)
+            else:
+                inp = x if policy == "lstm_scores" else np.asarray(features[t - 1], np.float32).astype(np.float64)
+                y, h_new, c_new = gate_step(inp, h, c, gate_w)
+                h, c = h_new.astype(np.float32), c_new.astype(np.float32)
             out["gate_logits"] = y
             out["gate_margin"] = float(abs(y[1] - y[0]))
             cont = gate_decision(y)

@@ -48,6 +48,94 @@ def test_gate_matches_torch_lstm_and_linear_over_a_sequence(k):
         assert np.allclose(c, th[1].view(-1).numpy(), atol=1e-12)
 
 
+def test_gate_with_a_wide_input_matches_torch_lstm():
+    """The hidden-state variant of Table 3 is the same network with another input size."""
+    d_in, H = 48, O.GATE_HIDDEN
+    g = np.random.default_rng(11)
+    u = lambda *shape: g.uniform(-0.5, 0.5, size=shape).astype(np.float32)
+    w = {"w_ih": u(4 * H, d_in), "w_hh": u(4 * H, H), "b_ih": u(4 * H), "b_hh": u(4 * H),
+         "w1": u(H, H + d_in), "b1": u(H), "w2": u(2, H), "b2": u(2)}
+    lstm, fc1, fc2 = _torch_gate(w, d_in)
+    h = np.zeros(H); c = np.zeros(H)
+    th = (torch.zeros(1, 1, H).double(), torch.zeros(1, 1, H).double())
+    for _ in range(4):
+        x = g.standard_normal(d_in)
+        y, h, c = O.gate_step(x, h, c, w)
+        with torch.no_grad():
+            out, th = lstm(torch.from_numpy(x).view(1, 1, d_in), th)
+            ty = fc2(torch.relu(fc1(torch.cat([out.view(-1), torch.from_numpy(x)]))))
+        assert np.allclose(y, ty.numpy(), atol=1e-12)
+        assert np.allclose(h, th[0].view(-1).numpy(), atol=1e-12)
+
+
+def _mlp_weights(k, seed=5, scale=2.0):
+    g = np.random.default_rng(seed)
+    H = O.GATE_HIDDEN
+    u = lambda *shape: g.uniform(-scale, scale, size=shape).astype(np.float32)
+    return {"w1": u(H, k), "b1": u(H), "w2": u(2, H), "b2": u(2)}
+
+
+@pytest.mark.parametrize("k", [4, 10])
+def test_mlp_gate_matches_torch_sequential(k):
+    w = _mlp_weights(k)
+    net = torch.nn.Sequential(torch.nn.Linear(k, O.GATE_HIDDEN), torch.nn.ReLU(), torch.nn.Linear(O.GATE_HIDDEN, 2)).double()
+    with torch.no_grad():
+        net[0].weight.copy_(torch.from_numpy(w["w1"]).double()); net[0].bias.copy_(torch.from_numpy(w["b1"]).double())
+        net[2].weight.copy_(torch.from_numpy(w["w2"]).double()); net[2].bias.copy_(torch.from_numpy(w["b2"]).double())
+    g = np.random.default_rng(9)
+    for _ in range(5):
+        x = g.random(k)
+        with torch.no_grad():
+            ty = net(torch.from_numpy(x))
+        assert np.allclose(O.gate_step_mlp(x, w), ty.numpy(), atol=1e-12)
+
+
+def test_mlp_gate_is_the_lstm_gate_with_the_recurrent_columns_cut():
+    """With the head's columns for the LSTM output zeroed, the paper's model no longer sees its state and
+    must equal the memoryless policy on the remaining columns; and zero weights give the output bias."""
+    cfg = W.shrink(W.CONFIGS[2], k=6)
+    w = {n: (v * 5).astype(np.float32) for n, v in W.gate_weights(cfg).items()}
+    H = O.GATE_HIDDEN
+    w["w1"][:, :H] = 0
+    wm = {"w1": w["w1"][:, H:].copy(), "b1": w["b1"], "w2": w["w2"], "b2": w["b2"]}
+    g = np.random.default_rng(2)
+    h = np.zeros(H); c = np.zeros(H)
+    for _ in range(4):
+        x = g.random(6)
+        y, h, c = O.gate_step(x, h, c, w)
+        assert np.allclose(y, O.gate_step_mlp(x, wm), atol=1e-12)
+    wz = {n: np.zeros_like(v) for n, v in wm.items()}
+    wz["b2"][:] = [0.5, -2.0]
+    assert O.gate_step_mlp(np.ones(6), wz).tolist() == [0.5, -2.0]
+
+
+def test_policy_variants_drive_the_expansion():
+    cfg = W.CONFIGS[1]
+    draft = W.draft_logits(cfg, 0)
+    k, t_max, H = cfg.k, cfg.t_max, O.GATE_HIDDEN
+    # memoryless policy: a bias that always continues runs to t_max, one that always stops makes one call
+    wm = {n: np.zeros_like(v) for n, v in _mlp_weights(k).items()}
+    wm["b2"][:] = [0.0, 1.0]
+    _, trace = O.run_expansion(draft, k, t_max, wm, policy="mlp_scores")
+    assert len(trace) == t_max and not any(tr["h"].any() for tr in trace)      # no recurrent state is kept
+    wm["b2"][:] = [1.0, 0.0]
+    _, trace = O.run_expansion(draft, k, t_max, wm, policy="mlp_scores")
+    assert len(trace) == 1
+    # hidden-state policy: the gate sees features[t-1] at call t and nothing of the scores
+    d_in = 24
+    g = np.random.default_rng(4)
+    u = lambda *shape: g.uniform(-0.3, 0.3, size=shape).astype(np.float32)
+    w = {"w_ih": u(4 * H, d_in), "w_hh": u(4 * H, H), "b_ih": u(4 * H), "b_hh": u(4 * H),
+         "w1": u(H, H + d_in), "b1": u(H), "w2": u(2, H), "b2": u(2)}
+    feats = g.standard_normal((t_max - 1, d_in)).astype(np.float32)
+    _, trace = O.run_expansion(draft, k, t_max, w, policy="lstm_hidden", features=feats, force_calls=3)
+    h = np.zeros(H); c = np.zeros(H)
+    for t, tr in enumerate(trace[:2], start=1):
+        y, h, c = O.gate_step(feats[t - 1].astype(np.float64), h, c, w)
+        h, c = h.astype(np.float32), c.astype(np.float32)
+        assert np.allclose(tr["gate_logits"], y, atol=1e-12)
+
+
 def test_gate_zero_weights_returns_output_bias():
     w = {n: np.zeros_like(v) for n, v in W.gate_weights(W.CONFIGS[1]).items()}
     w["b2"][:] = [0.25, -1.5]
