@@ -95,7 +95,19 @@ int radar_reset_launch_counts(radar_ctx* ctx);
  * A NaN logit records RADAR_ERR_NUMERIC (outputs of that sequence unspecified).
  * Limits: 1 <= k <= RADAR_MAX_K, 1 <= F <= 32, V >= k, pool_len[b] + F*k <= pool_capacity;
  * w_ih, w_hh and w1 16-byte aligned.
+ *
+ * `policy` selects the policy networks of the paper's ablation (Table 3):
+ *   RADAR_POLICY_LSTM_SCORES  the model above (the default, value 0);
+ *   RADAR_POLICY_MLP_SCORES   memoryless: Linear(k,H)-ReLU-Linear(H,2) on x; w1 is [H][k]; w_ih, w_hh,
+ *                             b_ih, b_hh may be NULL; h and c are neither read nor written;
+ *   RADAR_POLICY_LSTM_HIDDEN  the same LSTM + head fed with `features`[b] (the draft model's hidden
+ *                             state of this call, feat_dim floats) in place of x: w_ih is
+ *                             [4H][feat_dim], w1 is [H][H+feat_dim]; feat_dim a multiple of 4 in
+ *                             [4, 16384], features 16-byte aligned.
+ * Everything else of the call (candidates, pool, frontier) is the same for the three.
  */
+enum { RADAR_POLICY_LSTM_SCORES = 0, RADAR_POLICY_MLP_SCORES = 1, RADAR_POLICY_LSTM_HIDDEN = 2 };
+
 typedef struct {
     int B, F, V, k;
     int t, t_max;                       /* 1-based index of this draft call, and the maximum */
@@ -125,6 +137,9 @@ typedef struct {
     uint8_t* cont;                      /* [B] out */
     void* workspace;
     size_t workspace_bytes;
+    int policy;                         /* RADAR_POLICY_*                                    */
+    int feat_dim;                       /* RADAR_POLICY_LSTM_HIDDEN: length of a feature row */
+    const float* features;              /* RADAR_POLICY_LSTM_HIDDEN: [B][feat_dim], device   */
 } radar_expand_args;
 
 size_t radar_expand_workspace_bytes(const radar_ctx* ctx, int B, int F, int V, int k);

@@ -17,6 +17,7 @@ RADAR_MAX_NODES = 64
 RADAR_GATE_HIDDEN = 128
 RADAR_F32, RADAR_BF16 = 0, 1
 RADAR_GREEDY, RADAR_STOCHASTIC = 0, 1
+RADAR_POLICY_LSTM_SCORES, RADAR_POLICY_MLP_SCORES, RADAR_POLICY_LSTM_HIDDEN = 0, 1, 2
 RADAR_OK = 0
 
 _c_int, _c_i64, _c_f, _vp, _sz = ctypes.c_int, ctypes.c_int64, ctypes.c_float, ctypes.c_void_p, ctypes.c_size_t
@@ -36,6 +37,7 @@ class ExpandArgs(ctypes.Structure):
         ("frontier_tok", _vp), ("frontier_score", _vp), ("frontier_pool_idx", _vp), ("frontier_src_row", _vp),
         ("topk_tok", _vp), ("topk_logp", _vp), ("gate_logits", _vp), ("cont", _vp),
         ("workspace", _vp), ("workspace_bytes", _sz),
+        ("policy", _c_int), ("feat_dim", _c_int), ("features", _vp),
     ]
 
 
@@ -233,9 +235,11 @@ def radar_expand_step(ctx: Context, *, B, F, V, k, t, t_max, logits, logits_row_
                       logits_offset_elems=0, parent_score, parent_pool_idx, active, force_calls=None, gate,
                       h, c, pool_capacity, pool_tok, pool_parent, pool_depth, pool_draft_row, pool_score, pool_len,
                       frontier_tok, frontier_score, frontier_pool_idx, frontier_src_row, topk_tok, topk_logp,
-                      gate_logits, cont, workspace, stream=None):
+                      gate_logits, cont, workspace, stream=None, policy=RADAR_POLICY_LSTM_SCORES, features=None):
     """One draft call's expansion.  `logits` is a CUDA tensor; the rows of this call start
-    `logits_offset_elems` elements into it.  `gate` is a dict of the eight weight tensors."""
+    `logits_offset_elems` elements into it.  `gate` is a dict of the weight tensors (all eight for the
+    LSTM policies; w1, b1, w2, b2 for RADAR_POLICY_MLP_SCORES); `features` [B, feat_dim] float32 is the
+    input of RADAR_POLICY_LSTM_HIDDEN."""
     f32, i32, u8 = torch.float32, torch.int32, torch.uint8
     a = ExpandArgs()
     a.B, a.F, a.V, a.k, a.t, a.t_max = B, F, V, k, t, t_max
@@ -245,7 +249,10 @@ def radar_expand_step(ctx: Context, *, B, F, V, k, t, t_max, logits, logits_row_
     a.parent_score, a.parent_pool_idx = _ptr(parent_score, f32), _ptr(parent_pool_idx, i32)
     a.active, a.force_calls = _ptr(active, u8), _ptr(force_calls, i32)
     for n in ("w_ih", "w_hh", "b_ih", "b_hh", "w1", "b1", "w2", "b2"):
-        setattr(a, n, _ptr(gate[n], f32))
+        setattr(a, n, _ptr(gate.get(n), f32))
+    a.policy = policy
+    if features is not None:
+        a.features, a.feat_dim = _ptr(features, f32), features.shape[-1]
     a.h, a.c = _ptr(h, f32), _ptr(c, f32)
     a.pool_capacity = pool_capacity
     a.pool_tok, a.pool_parent, a.pool_depth = _ptr(pool_tok, i32), _ptr(pool_parent, i32), _ptr(pool_depth, i32)

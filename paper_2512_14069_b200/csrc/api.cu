@@ -88,6 +88,7 @@ extern "C" const char* radar_kernel_name(int id) {
         case RADAR_K_STOCH_WALK: return "stochastic_walk";
         case RADAR_K_ACCLEN_NODES: return "accept_length_nodes";
         case RADAR_K_ACCLEN_DIST: return "accept_length_dist";
+        case RADAR_K_GATE_FEATURES: return "gate_features";
         default: return "?";
     }
 }

@@ -19,6 +19,7 @@ enum radar_kernel_id {
     RADAR_K_STOCH_WALK,
     RADAR_K_ACCLEN_NODES,       // per-row conditional acceptance probabilities (Eq. 13)
     RADAR_K_ACCLEN_DIST,        // path products and the length distribution (Eq. 11-12)
+    RADAR_K_GATE_FEATURES,      // input-side products of the hidden-state policy (Table 3)
     RADAR_K_COUNT
 };
 

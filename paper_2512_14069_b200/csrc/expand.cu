@@ -20,7 +20,46 @@ struct SelectParams {
     VocabPassParams vp;
     int* status;
     int staged;                                      // 1: the block's chunk records fit the staging area
+    const float* feat_pre;                           // hidden-state policy: [B][4H] W_ih f and [B][H] W_1[:, H:] f,
+    const float* feat_hid;                           // written by gate_features_kernel
 };
+
+// Hidden-state policy (Table 3): the input-side products of the prediction model, W_ih f_b (4H rows) and the
+// head's columns for the input, W_1[:, H:] f_b (H rows), for every sequence.  One warp per output row; the
+// weights are read once, the feature rows come from L1/L2.  It needs nothing from the vocabulary pass and is
+// launched ahead of it.
+constexpr int kFeatRowsPerBlock = 8;
+__global__ void __launch_bounds__(kFeatRowsPerBlock * 32) gate_features_kernel(const radar_expand_args a, float* pre, float* hid) {
+    chain_wait();
+    const int H = kHidden, lane = threadIdx.x & 31;
+    const int r = blockIdx.x * kFeatRowsPerBlock + (threadIdx.x >> 5);          // 0 .. 5H-1
+    if (r >= 5 * H) return;
+    const int d = a.feat_dim;
+    const float* w = r < 4 * H ? a.w_ih + (size_t)r * d : a.w1 + (size_t)(r - 4 * H) * (H + d) + H;
+    for (int b0 = 0; b0 < a.B; b0 += 8) {
+        float acc[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) acc[i] = 0.f;
+        for (int c = lane * 4; c < d; c += 128) {
+            const float4 wv = __ldg(reinterpret_cast<const float4*>(w + c));
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                if (b0 + i < a.B) {
+                    const float4 f = __ldg(reinterpret_cast<const float4*>(a.features + (size_t)(b0 + i) * d + c));
+                    acc[i] = fmaf(wv.x, f.x, fmaf(wv.y, f.y, fmaf(wv.z, f.z, fmaf(wv.w, f.w, acc[i]))));
+                }
+            }
+        }
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const float v = warp_sum(acc[i]);
+            if (lane == 0 && b0 + i < a.B) {
+                if (r < 4 * H) pre[(size_t)(b0 + i) * 4 * H + r] = v;
+                else hid[(size_t)(b0 + i) * H + (r - 4 * H)] = v;
+            }
+        }
+    }
+}
 
 __device__ __forceinline__ float sigmoidf_(float x) { return 1.f / (1.f + expf(-x)); }
 
@@ -56,6 +95,8 @@ __global__ void __launch_bounds__(kSelThreads, 1) expand_select_gate_kernel(cons
     const int n_chunks = P.vp.n_chunks;
     const int per_row = n_chunks * k;
     const bool run_gate = a.t < a.t_max;
+    const int policy = a.policy;
+    const int kx = policy == RADAR_POLICY_LSTM_HIDDEN ? 0 : k;      // input columns the block itself multiplies
 
     extern __shared__ __align__(16) unsigned char sel_smem[];
     const size_t stage_elems = P.staged ? (size_t)F * per_row : 0;
@@ -206,13 +247,23 @@ __global__ void __launch_bounds__(kSelThreads, 1) expand_select_gate_kernel(cons
         // ---- 1b. the part of the prediction model that only needs the previous state ----
         const int gt = tid - kMergeWarps * 32;          // 0..511
         const int gw = warp - kMergeWarps;              // 0..15
-        for (int e = gt; e < H * k; e += 512) cp_async16(s_wih + 4 * e, a.w_ih + 4 * e);          // 4H*k floats
-        for (int e = gt; e < H * (H + k) / 4; e += 512) cp_async16(s_w1 + 4 * e, a.w1 + 4 * e);
-        if (gt < H) s_h[gt] = a.t > 1 ? a.h[(size_t)b * H + gt] : 0.f;
+        if (policy == RADAR_POLICY_MLP_SCORES) {
+            for (int e = gt; e < H * k / 4; e += 512) cp_async16(s_w1 + 4 * e, a.w1 + 4 * e);     // [H][k]
+        } else if (policy == RADAR_POLICY_LSTM_HIDDEN) {
+            // only the head's columns for the LSTM output; the input columns were applied by gate_features_kernel
+            for (int e = gt; e < H * H / 4; e += 512) {
+                const int r = e / (H / 4), c4 = e % (H / 4);
+                cp_async16(s_w1 + r * H + c4 * 4, a.w1 + (size_t)r * (H + a.feat_dim) + c4 * 4);
+            }
+        } else {
+            for (int e = gt; e < H * k; e += 512) cp_async16(s_wih + 4 * e, a.w_ih + 4 * e);          // 4H*k floats
+            for (int e = gt; e < H * (H + k) / 4; e += 512) cp_async16(s_w1 + 4 * e, a.w1 + 4 * e);
+        }
+        if (gt < H) s_h[gt] = a.t > 1 && policy != RADAR_POLICY_MLP_SCORES ? a.h[(size_t)b * H + gt] : 0.f;
         group_barrier(3);
         const float4 h4 = *reinterpret_cast<const float4*>(&s_h[lane * 4]);
         constexpr int kBatch = 8;
-        for (int r0 = gw * 32; r0 < gw * 32 + 32; r0 += kBatch) {
+        for (int r0 = gw * 32; policy != RADAR_POLICY_MLP_SCORES && r0 < gw * 32 + 32; r0 += kBatch) {
             float4 w[kBatch];
 #pragma unroll
             for (int i = 0; i < kBatch; ++i)
@@ -273,11 +324,33 @@ __global__ void __launch_bounds__(kSelThreads, 1) expand_select_gate_kernel(cons
 
     // ---- 4. prediction model, from shared memory ----
     bool cont = false;
-    if (run_gate) {
+    if (run_gate && policy == RADAR_POLICY_MLP_SCORES) {
+        if (tid < H) {
+            float acc = s_b1[tid];
+            const float* w = s_w1 + tid * k;
+            for (int j = 0; j < k; ++j) acc = fmaf(w[j], s_x[j], acc);
+            s_hid[tid] = fmaxf(acc, 0.f);
+        }
+        __syncthreads();
+        if (warp < 2) {
+            float acc = 0.f;
+            for (int c = lane; c < H; c += 32) acc = fmaf(s_w2[warp * H + c], s_hid[c], acc);
+            acc = warp_sum(acc);
+            if (lane == 0) s_y[warp] = acc + s_b2[warp];
+        }
+        __syncthreads();
+        cont = s_y[1] > s_y[0];
+        if (tid < 2) a.gate_logits[(size_t)b * 2 + tid] = s_y[tid];
+        if (a.force_calls != nullptr) cont = a.t < a.force_calls[b];
+    } else if (run_gate) {
         if (tid < 4 * H) {
             float acc = s_pre[tid];
-            const float* w = s_wih + tid * k;
-            for (int j = 0; j < k; ++j) acc = fmaf(w[j], s_x[j], acc);
+            if (policy == RADAR_POLICY_LSTM_HIDDEN) {
+                acc += P.feat_pre[(size_t)b * 4 * H + tid];
+            } else {
+                const float* w = s_wih + tid * k;
+                for (int j = 0; j < k; ++j) acc = fmaf(w[j], s_x[j], acc);
+            }
             s_pre[tid] = acc;
         }
         __syncthreads();
@@ -294,12 +367,12 @@ __global__ void __launch_bounds__(kSelThreads, 1) expand_select_gate_kernel(cons
         }
         __syncthreads();
         for (int r = warp; r < H; r += kSelWarps) {
-            const float* w = s_w1 + r * (H + k);
+            const float* w = s_w1 + r * (H + kx);
             float acc = 0.f;
             for (int c = lane; c < H; c += 32) acc = fmaf(w[c], s_hn[c], acc);
-            if (lane < k) acc = fmaf(w[H + lane], s_x[lane], acc);
+            if (lane < kx) acc = fmaf(w[H + lane], s_x[lane], acc);
             acc = warp_sum(acc);
-            if (lane == 0) s_hid[r] = fmaxf(acc + s_b1[r], 0.f);
+            if (lane == 0) s_hid[r] = fmaxf(acc + s_b1[r] + (policy == RADAR_POLICY_LSTM_HIDDEN ? P.feat_hid[(size_t)b * H + r] : 0.f), 0.f);
         }
         __syncthreads();
         if (warp < 2) {
@@ -330,7 +403,7 @@ extern "C" size_t radar_expand_workspace_bytes(const radar_ctx* ctx, int B, int 
     if (!ctx || B <= 0 || F <= 0 || V <= 0 || k <= 0) return 0;
     int chunk;
     const int n_chunks = vocab_pass_plan_chunks(ctx->sm_count, B * F, V, &chunk);
-    return vocab_pass_partial_bytes(B * F, n_chunks, k);
+    return align_up(vocab_pass_partial_bytes(B * F, n_chunks, k), 256) + (size_t)B * 5 * kHidden * sizeof(float);
 }
 
 extern "C" int radar_expand_step(radar_ctx* ctx, const radar_expand_args* a, void* stream_) {
@@ -345,10 +418,18 @@ extern "C" int radar_expand_step(radar_ctx* ctx, const radar_expand_args* a, voi
         !a->frontier_tok || !a->frontier_score || !a->frontier_pool_idx || !a->frontier_src_row || !a->topk_tok ||
         !a->topk_logp || !a->gate_logits || !a->cont || !a->workspace)
         return RADAR_ERR_INVALID_ARG;
-    if (a->t < a->t_max && (!a->w_ih || !a->w_hh || !a->b_ih || !a->b_hh || !a->w1 || !a->b1 || !a->w2 || !a->b2))
+    if (a->policy != RADAR_POLICY_LSTM_SCORES && a->policy != RADAR_POLICY_MLP_SCORES && a->policy != RADAR_POLICY_LSTM_HIDDEN)
         return RADAR_ERR_INVALID_ARG;
-    if (a->t < a->t_max && ((reinterpret_cast<uintptr_t>(a->w_hh) | reinterpret_cast<uintptr_t>(a->w_ih) |
-                             reinterpret_cast<uintptr_t>(a->w1)) & 15) != 0)
+    const bool gate_runs = a->t < a->t_max;
+    if (gate_runs && (!a->w1 || !a->b1 || !a->w2 || !a->b2 || (reinterpret_cast<uintptr_t>(a->w1) & 15) != 0))
+        return RADAR_ERR_INVALID_ARG;
+    if (gate_runs && a->policy != RADAR_POLICY_MLP_SCORES &&
+        (!a->w_ih || !a->w_hh || !a->b_ih || !a->b_hh ||
+         ((reinterpret_cast<uintptr_t>(a->w_hh) | reinterpret_cast<uintptr_t>(a->w_ih)) & 15) != 0))
+        return RADAR_ERR_INVALID_ARG;
+    if (gate_runs && a->policy == RADAR_POLICY_LSTM_HIDDEN &&
+        (!a->features || a->feat_dim < 4 || a->feat_dim > 16384 || (a->feat_dim & 3) != 0 ||
+         (reinterpret_cast<uintptr_t>(a->features) & 15) != 0))
         return RADAR_ERR_INVALID_ARG;
     if (a->pool_capacity < a->F * a->k) return RADAR_ERR_INVALID_ARG;
     if ((reinterpret_cast<uintptr_t>(a->workspace) & 255) != 0) return RADAR_ERR_WORKSPACE;
@@ -370,8 +451,17 @@ extern "C" int radar_expand_step(radar_ctx* ctx, const radar_expand_args* a, voi
     vp.seq_active = a->t > 1 ? a->active : nullptr;
     vp.seq_rows = nullptr;
     vp.status = ctx->d_status;
-    if (vocab_pass_partial_bytes(a->B * a->F, vp.n_chunks, a->k) > a->workspace_bytes) return RADAR_ERR_WORKSPACE;
+    const size_t part_bytes = align_up(vocab_pass_partial_bytes(a->B * a->F, vp.n_chunks, a->k), 256);
+    if (part_bytes + (size_t)a->B * 5 * kHidden * sizeof(float) > a->workspace_bytes) return RADAR_ERR_WORKSPACE;
     vocab_pass_carve(a->workspace, a->B * a->F, vp.n_chunks, a->k, &vp);
+    float* feat_pre = reinterpret_cast<float*>(reinterpret_cast<char*>(a->workspace) + part_bytes);
+    sp.feat_pre = feat_pre;
+    sp.feat_hid = feat_pre + (size_t)a->B * 4 * kHidden;
+    if (gate_runs && a->policy == RADAR_POLICY_LSTM_HIDDEN) {
+        radar_launch_scope scope(ctx, RADAR_K_GATE_FEATURES, stream);
+        RADAR_CUDA_CHECK(launch_chained(gate_features_kernel, dim3((5 * kHidden + kFeatRowsPerBlock - 1) / kFeatRowsPerBlock),
+                                        dim3(kFeatRowsPerBlock * 32), 0, stream, *a, feat_pre, feat_pre + (size_t)a->B * 4 * kHidden));
+    }
 
     RADAR_CUDA_CHECK(vocab_pass_launch(ctx, RADAR_K_VOCAB_EXPAND, vp, stream));
     const size_t stage_bytes = (size_t)a->F * vp.n_chunks * a->k * 8;

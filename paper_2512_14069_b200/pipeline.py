@@ -66,8 +66,9 @@ class SpecStep:
             setattr(self, n, t[off:off + t.numel() - 255])
 
     # ---- expansion -------------------------------------------------------------------
-    def expand(self, t, draft_logits, gate, force_calls=None):
-        """Draft call t (1-based) on draft_logits [B,R,V]: row 0 for t = 1, rows 1+(t-2)k.. for t >= 2."""
+    def expand(self, t, draft_logits, gate, force_calls=None, policy=rb.RADAR_POLICY_LSTM_SCORES, features=None):
+        """Draft call t (1-based) on draft_logits [B,R,V]: row 0 for t = 1, rows 1+(t-2)k.. for t >= 2.
+        `features` [t_max-1, B, feat_dim] feeds the hidden-state policy (row t-1 at call t)."""
         k, B, V = self.k, self.B, self.V
         F = 1 if t == 1 else k
         row0 = 0 if t == 1 else 1 + (t - 2) * k
@@ -84,11 +85,12 @@ class SpecStep:
             frontier_pool_idx=self.frontier_pool_idx[s], frontier_src_row=self.frontier_src_row[s],
             topk_tok=self.topk_tok1 if t == 1 else self.topk_tok[s],
             topk_logp=self.topk_logp1 if t == 1 else self.topk_logp[s],
-            gate_logits=self.gate_logits[s], cont=self.cont_hist[s], workspace=self.ws_expand)
+            gate_logits=self.gate_logits[s], cont=self.cont_hist[s], workspace=self.ws_expand, policy=policy,
+            features=None if features is None or t >= self.t_max else features[s])
 
-    def run_expansion(self, draft_logits, gate, force_calls=None):
+    def run_expansion(self, draft_logits, gate, force_calls=None, policy=rb.RADAR_POLICY_LSTM_SCORES, features=None):
         for t in range(1, self.t_max + 1):          # call 1 restarts the state on the device
-            self.expand(t, draft_logits, gate, force_calls)
+            self.expand(t, draft_logits, gate, force_calls, policy, features)
 
     # ---- tree, attention, acceptance ------------------------------------------------------
     def build_tree(self, root_tok, prefix_len, n_keep=None):

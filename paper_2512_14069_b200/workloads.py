@@ -21,7 +21,7 @@ GATE_HIDDEN = 128
 
 # tensor ids (second word of every stream key)
 T_DRAFT, T_TARGET_NOISE, T_GATE, T_Q, T_KC, T_VC, T_KT, T_VT, T_UACC, T_USAMP, T_PLEN, T_DEPTH, \
-    T_NKEEP, T_PEAK, T_TARGET_FRESH, T_ROOT = range(16)
+    T_NKEEP, T_PEAK, T_TARGET_FRESH, T_ROOT, T_POLICY, T_FEATURES = range(18)
 
 
 @dataclass(frozen=True)
@@ -43,7 +43,7 @@ class Config:
     draft_kind: str          # "normal2" | "zipf"
     zipf_a: tuple            # (lo, hi) per-sequence peakedness
     target_sigma: float
-    depth_plan: str          # "gate" | "uniform_1_tmax" | "uniform_2_tmax"
+    depth_plan: str          # "gate" | "uniform_1_tmax" | "uniform_2_tmax" | "fixed_tmax"
     nkeep_range: tuple | None  # per-sequence rerank size range, None = N everywhere
     # Random-init gate weights give an almost input-independent decision; this constant, added to
     # the "continue" bias, centres the decision inside the trajectory so that depth is input-decided.
@@ -107,6 +107,8 @@ def forced_calls(cfg: Config):
     """Per-sequence number of draft calls when the harness (not the gate) fixes it, else None."""
     if cfg.depth_plan == "gate":
         return None
+    if cfg.depth_plan == "fixed_tmax":             # EAGLE-3's fixed schedule: every sequence makes all t_max calls
+        return np.full(cfg.B, cfg.t_max, np.int32)
     lo = 1 if cfg.depth_plan == "uniform_1_tmax" else 2
     return stream(cfg, T_DEPTH).integers(lo, cfg.t_max + 1, size=cfg.B).astype(np.int32)
 
@@ -181,6 +183,27 @@ def gate_weights(cfg: Config) -> dict:
          "w1": u(H, H + k), "b1": u(H), "w2": u(2, H), "b2": u(2)}
     w["b2"][1] += np.float32(cfg.gate_b2_offset)
     return w
+
+
+def policy_weights(cfg: Config, policy: str, feat_dim: int = 0) -> dict:
+    """Random-init weights of the ablation's policy networks (Table 3), same distribution as
+    `gate_weights`: "mlp_scores" -> Linear(k, H), ReLU, Linear(H, 2); "lstm_hidden" -> LSTM(input
+    feat_dim, hidden H) and Linear(H + feat_dim, H), ReLU, Linear(H, 2).  The "continue" bias is
+    left at its draw: the variants are regression workloads, their depth is whatever comes out."""
+    H, k = GATE_HIDDEN, cfg.k
+    g = stream(cfg, T_POLICY, 0 if policy == "mlp_scores" else 1)
+    s = 1.0 / np.sqrt(H)
+    u = lambda *shape: g.uniform(-s, s, size=shape).astype(np.float32)
+    if policy == "mlp_scores":
+        return {"w1": u(H, k), "b1": u(H), "w2": u(2, H), "b2": u(2)}
+    assert policy == "lstm_hidden" and feat_dim > 0
+    return {"w_ih": u(4 * H, feat_dim), "w_hh": u(4 * H, H), "b_ih": u(4 * H), "b_hh": u(4 * H),
+            "w1": u(H, H + feat_dim), "b1": u(H), "w2": u(2, H), "b2": u(2)}
+
+
+def gate_features(cfg: Config, feat_dim: int) -> np.ndarray:
+    """[t_max-1, B, feat_dim] float32 N(0,1): stands in for the draft model's hidden state of each call."""
+    return stream(cfg, T_FEATURES).standard_normal((cfg.t_max - 1, cfg.B, feat_dim), dtype=np.float32)
 
 
 # ---- attention operands -------------------------------------------------------

@@ -54,6 +54,66 @@ def test_whole_step_matches_oracle(ctx, cid):
     H.compare_accept(cfg, g, accepts)
 
 
+@pytest.mark.parametrize("name", ["fixed_depth_greedy", "chain_greedy", "chain_stochastic"])
+def test_regression_workloads_match_oracle(ctx, name):
+    """The fixed schedule the paper compares with (gate off, every sequence makes all t_max calls) and
+    chain drafts (k = 1: the tree is a path, its mask is causal, and stochastic acceptance is the
+    single-draft rule of Eq. 1-2)."""
+    if name == "fixed_depth_greedy":
+        cfg = W.shrink(W.CONFIGS[2], B=3, V=9001, P=(700, 700), depth_plan="fixed_tmax")
+    elif name == "chain_greedy":
+        cfg = W.shrink(W.CONFIGS[2], B=3, V=9001, P=(700, 700), k=1, N=7, depth_plan="fixed_tmax")
+    else:
+        cfg = W.shrink(W.CONFIGS[3], B=3, Hq=8, Hkv=8, V=9001, P=(700, 700), k=1, t_max=6, N=5, depth_plan="fixed_tmax")
+    inp = H.make_inputs(cfg)
+    pools, traces, trees = H.oracle_expand_and_tree(cfg, inp)
+    assert all(len(t) == cfg.t_max for t in traces)
+    if cfg.k == 1:
+        for t in trees:                                   # a path: node i's ancestors are 0..i
+            assert all(int(t["mask"][i]) == (1 << (i + 1)) - 1 for i in range(t["n_nodes"]))
+    target = H.make_target(cfg, inp, trees)
+    accepts = H.oracle_accept(cfg, inp, trees, target)
+    H.check_margins(cfg, traces, trees, accepts)
+    g = H.GpuRun(cfg, inp, ctx)
+    g.expand_and_tree()
+    H.compare_expansion(cfg, g, pools, traces)
+    H.compare_tree(cfg, g, trees)
+    g.upload_attention()
+    O_gpu, lse_gpu = g.attention()
+    O_ref, lse_ref = H.oracle_attention(cfg, inp, trees)
+    H.compare_attention(cfg, O_gpu, lse_gpu, O_ref, lse_ref, trees)
+    g.accept(target)
+    H.compare_accept(cfg, g, accepts)
+
+
+@pytest.mark.parametrize("policy,feat_dim", [("mlp_scores", 0), ("lstm_hidden", 64), ("lstm_hidden", 4096)])
+def test_policy_variants_match_oracle(ctx, policy, feat_dim):
+    """The policy networks of the ablation (Table 3): memoryless MLP on the scores, and the LSTM fed with
+    a hidden-state vector (a small one and one of the draft model's width).  Same comparisons as the
+    paper's model: every call's outputs, gate logits within 1e-5, continue/stop bit-exact, final h and c."""
+    from oracle import radar_oracle as O
+    from paper_2512_14069_b200 import binding as rb
+    cfg = W.shrink(W.CONFIGS[2], B=5, V=9001, depth_plan="gate")
+    inp = H.make_inputs(cfg, with_attention=False)
+    w = W.policy_weights(cfg, policy, feat_dim)
+    feats = W.gate_features(cfg, feat_dim) if feat_dim else None
+    pools, traces = [], []
+    for b in range(cfg.B):
+        pool, trace = O.run_expansion(inp["draft"][b], cfg.k, cfg.t_max, w, policy=policy,
+                                      features=None if feats is None else feats[:, b])
+        pools.append(pool)
+        traces.append(trace)
+        for tr in trace:
+            assert tr["margin"] > H.TAU_SCORE and tr.get("gate_margin", 1.0) > H.TAU_SCORE
+    assert len({len(t) for t in traces}) > 1 or policy == "mlp_scores"      # the hidden-state gate stops at different depths
+    g = H.GpuRun(cfg, inp, ctx)
+    code = rb.RADAR_POLICY_MLP_SCORES if policy == "mlp_scores" else rb.RADAR_POLICY_LSTM_HIDDEN
+    g.step.run_expansion(g.draft, {n: H.to_dev(v) for n, v in w.items()}, None, policy=code,
+                         features=None if feats is None else H.to_dev(feats))
+    ctx.check_device_status()
+    H.compare_expansion(cfg, g, pools, traces)
+
+
 @pytest.mark.parametrize("cid,temperature", [(1, 1.0), (3, 1.0), (5, 0.7), (2, 0.5)])
 def test_accept_length_distribution_matches_oracle(ctx, cid, temperature):
     """Eq. 11-13 for every tree of the batch: p_0..p_tmax and P_acc of every row against the fp64 oracle.
