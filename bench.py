@@ -230,12 +230,28 @@ def scale_probe(ctx, dev, peaks, reps=20):
     ctx.check_device_status()
     ks = {n: 1000.0 * v[1] / v[2] for n, v in ctx.kernel_stats().items() if v[2] > 0}
     us_attn, us_acc, us_exp = ks["tree_attention"], ks["vocab_pass(accept)"], ks["vocab_pass(expand)"]
+    # the same attention launch reading the prefix through a block table of shuffled 16-token pages
+    page = 16
+    perm = torch.randperm(B * P // page, device=dev, generator=g).to(torch.int32).view(B, P // page).contiguous()
+    ctx.profile_begin(reps * 2)
+    for i0 in range(0, reps, 5):
+        torch.cuda._sleep(8_000_000)
+        for i in range(i0, min(i0 + 5, reps)):
+            step.attention(Q, Kc, Vc, None, plen, Kt, Vt, block_table=perm, page_size=page)
+        torch.cuda.synchronize()
+    ctx.profile_end()
+    ctx.check_device_status()
+    kp = ctx.kernel_stats()["tree_attention"]
+    us_attn_paged = 1000.0 * kp[1] / kp[2]
     kv_bytes = float(((P + n_nodes) * Hkv * d * 2 * 2).sum() + 2 * n_nodes.sum() * Hq * d * 2)
     flops = float((4 * n_nodes * Hq * (P + n_nodes) * d).sum())
     shapes = "LLaMA-3.3-70B shapes: B=8, Hq/Hkv/d=64/8/128, prefix 8192, V=128256, k=10, %d..%d tree rows" % (n_nodes.min(), n_nodes.max())
     out = []
     ka = {"avg_us": us_attn, "alg_bytes_per_launch": kv_bytes, "gbs": kv_bytes / us_attn / 1e3, "tflops": flops / us_attn / 1e6}
     out.append(roofline_entry("tree_attention", ka, peaks, NCU_TRAFFIC_RATIO.get(("tree_attention", 4))))
+    kpg = {"avg_us": us_attn_paged, "alg_bytes_per_launch": kv_bytes, "gbs": kv_bytes / us_attn_paged / 1e3,
+           "tflops": flops / us_attn_paged / 1e6}
+    out.append(roofline_entry("tree_attention(paged cache, 16-token pages)", kpg, peaks, None))
     b_acc = float(n_nodes.sum()) * V * 4
     out.append(roofline_entry("vocab_pass(accept)", {"avg_us": us_acc, "alg_bytes_per_launch": b_acc,
                                                      "gbs": b_acc / us_acc / 1e3}, peaks,

@@ -198,6 +198,13 @@ int radar_rerank_build_tree(radar_ctx* ctx, const radar_tree_args* args, void* s
  * bf16 with Hq / Hkv a power of two (<= 128) and 16-byte aligned tensors runs on the tensor cores
  * (TMA-staged K/V tiles, tcgen05 MMA for QK^T and PV); every other case, and all of fp32, runs on
  * an fp32 FMA kernel.
+ * Paged prefix cache (block_table != NULL): prefix token j of sequence b is cache row
+ *   block_table[b * max_pages + j / page_size] * page_size + j % page_size
+ * and kv_start is not read (it may be NULL).  page_size is 16, 32, 64 or a multiple of 128; a
+ * sequence needs ceil(prefix_len / page_size) <= max_pages entries; entries past that are not read.
+ * A page index whose page does not lie inside [0, cache_rows) records RADAR_ERR_INVALID_ARG on the
+ * device status word (the read goes to page 0).  The paper has no paged cache; this is the layout
+ * serving systems keep their KV in, so that verification can read it in place.
  * Limits: d in {64, 128}; Hq a multiple of Hkv; cache_rows < 2^31.
  */
 typedef struct {
@@ -217,6 +224,9 @@ typedef struct {
     float* lse;                         /* or NULL */
     void* workspace;
     size_t workspace_bytes;
+    const int32_t* block_table;         /* [B][max_pages] page indices, or NULL for the contiguous layout */
+    int page_size;                      /* tokens per page                                               */
+    int max_pages;                      /* entries per sequence in block_table                           */
 } radar_attn_args;
 
 size_t radar_attn_workspace_bytes(const radar_ctx* ctx, int B, int Hq, int Hkv, int d, int dtype, int max_prefix_len);

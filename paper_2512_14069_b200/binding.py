@@ -58,6 +58,7 @@ class AttnArgs(ctypes.Structure):
         ("Q", _vp), ("Kc", _vp), ("Vc", _vp), ("kv_start", _vp), ("prefix_len", _vp), ("max_prefix_len", _c_int),
         ("cache_rows", _c_i64), ("Kt", _vp), ("Vt", _vp), ("mask", _vp), ("n_nodes", _vp), ("scale", _c_f), ("O", _vp), ("lse", _vp),
         ("workspace", _vp), ("workspace_bytes", _sz),
+        ("block_table", _vp), ("page_size", _c_int), ("max_pages", _c_int),
     ]
 
 
@@ -283,7 +284,8 @@ def radar_rerank_build_tree(ctx: Context, *, B, N, t_max, pool_capacity, pool_to
 
 
 def radar_tree_attention(ctx: Context, *, B, Hq, Hkv, d, Q, Kc, Vc, kv_start, prefix_len, max_prefix_len, Kt, Vt,
-                         mask, n_nodes, O, workspace, lse=None, scale=0.0, stream=None):
+                         mask, n_nodes, O, workspace, lse=None, scale=0.0, stream=None, block_table=None, page_size=0):
+    """`block_table` [B, max_pages] int32 with `page_size` selects the paged prefix cache (kv_start may then be None)."""
     a = AttnArgs()
     a.B, a.Hq, a.Hkv, a.d, a.dtype = B, Hq, Hkv, d, dtype_code(Q)
     for t in (Kc, Vc, Kt, Vt, O):
@@ -296,6 +298,8 @@ def radar_tree_attention(ctx: Context, *, B, Hq, Hkv, d, Q, Kc, Vc, kv_start, pr
     a.Kt, a.Vt, a.mask, a.n_nodes = _ptr(Kt), _ptr(Vt), _ptr(mask, torch.int64), _ptr(n_nodes, torch.int32)
     a.scale, a.O, a.lse = scale, _ptr(O), _ptr(lse, torch.float32)
     a.workspace, a.workspace_bytes = _ptr(workspace), workspace.numel() * workspace.element_size()
+    if block_table is not None:
+        a.block_table, a.page_size, a.max_pages = _ptr(block_table, torch.int32), page_size, block_table.shape[-1]
     _check("radar_tree_attention", lib().radar_tree_attention(ctx.handle, ctypes.byref(a), _stream(stream)))
 
 

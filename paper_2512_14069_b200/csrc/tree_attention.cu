@@ -84,7 +84,9 @@ __global__ void __launch_bounds__(kThreads) tree_attn_fp32_kernel(const AttnPara
     const T* Vc = reinterpret_cast<const T*>(a.Vc);
     const T* Kt = reinterpret_cast<const T*>(a.Kt);
     const T* Vt = reinterpret_cast<const T*>(a.Vt);
-    const int64_t kv0 = a.kv_start[b];
+    const bool paged = a.block_table != nullptr;
+    const int64_t kv0 = paged ? 0 : a.kv_start[b];
+    const int64_t n_cache_pages = paged ? P.a.cache_rows / a.page_size : 0;
 
     // ---- stage the block's query rows (pre-scaled) ----
     for (int e = tid; e < kRowsPerBlock * (D / 16); e += kThreads) {
@@ -128,7 +130,13 @@ __global__ void __launch_bounds__(kThreads) tree_attn_fp32_kernel(const AttnPara
             if (kidx < k_end) {
                 const T *ksrc, *vsrc;
                 if (kidx < Pb) {
-                    const int64_t off = ((kv0 + kidx) * Hkv + g) * D + seg * 16;
+                    int64_t row = kv0 + kidx;
+                    if (paged) {
+                        int64_t page = a.block_table[(int64_t)b * a.max_pages + kidx / a.page_size];
+                        if (page < 0 || page >= n_cache_pages) { set_status(P.status, RADAR_ERR_INVALID_ARG); page = 0; }
+                        row = page * a.page_size + kidx % a.page_size;
+                    }
+                    const int64_t off = (row * Hkv + g) * D + seg * 16;
                     ksrc = Kc + off; vsrc = Vc + off;
                 } else {
                     const int64_t off = (((int64_t)b * kMaxNodes + (kidx - Pb)) * Hkv + g) * D + seg * 16;
@@ -324,7 +332,12 @@ extern "C" int radar_tree_attention(radar_ctx* ctx, const radar_attn_args* a, vo
     if (a->Hq % a->Hkv != 0) return RADAR_ERR_INVALID_ARG;
     if (a->d != 64 && a->d != 128) return RADAR_ERR_UNSUPPORTED;
     if (a->dtype != RADAR_F32 && a->dtype != RADAR_BF16) return RADAR_ERR_UNSUPPORTED;
-    if (!a->Q || !a->kv_start || !a->prefix_len || !a->Kt || !a->Vt || !a->mask || !a->n_nodes || !a->O ||
+    const bool paged = a->block_table != nullptr;
+    if (paged && (a->max_pages <= 0 || !(a->page_size == 16 || a->page_size == 32 || a->page_size == 64 ||
+                                         (a->page_size > 0 && a->page_size % 128 == 0)) ||
+                  (long long)a->max_pages * a->page_size < a->max_prefix_len || a->cache_rows < a->page_size))
+        return RADAR_ERR_INVALID_ARG;
+    if (!a->Q || (!paged && !a->kv_start) || !a->prefix_len || !a->Kt || !a->Vt || !a->mask || !a->n_nodes || !a->O ||
         !a->workspace)
         return RADAR_ERR_INVALID_ARG;
     if (a->max_prefix_len > 0 && (!a->Kc || !a->Vc)) return RADAR_ERR_INVALID_ARG;

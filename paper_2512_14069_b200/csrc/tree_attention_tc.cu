@@ -89,20 +89,22 @@ struct SeqInfo {
     long long kv0;
 };
 
+template <bool PAGED>
 __device__ __forceinline__ SeqInfo seq_info(const TcParams& P, int b, int pp) {
     const radar_attn_args& a = P.a;
     SeqInfo s;
     s.M = min(max(a.n_nodes[b], 0), kMaxNodes);
     s.Pb = a.prefix_len[b];
-    s.kv0 = a.kv_start[b];
+    s.kv0 = PAGED ? 0 : a.kv_start[b];          // paged: the host has checked max_pages * page_size >= max_prefix_len
     const bool ok = s.Pb >= 0 && s.Pb <= a.max_prefix_len && s.kv0 >= 0 && s.kv0 + s.Pb <= P.cache_rows;
     s.rows = ok ? min(max(s.M * P.G - pp * P.pair_rows, 0), P.pair_rows) : 0;
     s.nt = (max(s.Pb, 0) + kTileKeys - 1) / kTileKeys + 1;
     s.w = s.rows > 128 ? kCostTwo : kCostOne;
     return s;
 }
+template <bool PAGED>
 __device__ __forceinline__ long long seq_cost(const TcParams& P, int b, int pp) {
-    const SeqInfo s = seq_info(P, b, pp);
+    const SeqInfo s = seq_info<PAGED>(P, b, pp);
     return s.rows > 0 ? (long long)P.a.Hkv * s.nt * s.w : 0;
 }
 // number of tiles of a unit (start position U, nt tiles of cost w) that start before position x
@@ -113,6 +115,7 @@ __device__ __forceinline__ int tiles_before(long long x, long long U, int nt, in
 }
 
 // One CTA's walk over its range [.., hi) of the class's space: segments (sequence b, KV head g, tiles [t0, t1)).
+template <bool PAGED>
 struct Cursor {
     int b, g, t0, t1;
     long long U, hi;     // start position of the current unit, end of the CTA's range
@@ -124,7 +127,7 @@ struct Cursor {
         t0 = 0;
         if (++g == P.a.Hkv) {
             g = 0;
-            do { ++b; if (b >= P.a.B) { t1 = 0; return; } s = seq_info(P, b, pp); } while (s.rows == 0);
+            do { ++b; if (b >= P.a.B) { t1 = 0; return; } s = seq_info<PAGED>(P, b, pp); } while (s.rows == 0);
         }
         clip();
     }
@@ -149,7 +152,9 @@ struct Smem {
 };
 
 // TWO: the launch may contain units with two live row blocks; decides the shared-memory layout
-template <int D, bool TWO>
+// PAGED: the prefix cache is read through a block table (a separate instantiation, so that the contiguous
+// layout's code is not touched by it)
+template <int D, bool TWO, bool PAGED>
 __global__ void __launch_bounds__(kTcThreads, 1)
 tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmKc,
                     const __grid_constant__ CUtensorMap tmVc, const __grid_constant__ CUtensorMap tmKt,
@@ -184,10 +189,10 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         long long tot = 0;
         for (int b0 = 0; b0 < a.B; b0 += 32) {
             const int b = b0 + lane;
-            long long sz = b < a.B ? seq_cost(P, b, pp) : 0;
+            long long sz = b < a.B ? seq_cost<PAGED>(P, b, pp) : 0;
             if (pp == 0 && ci == 0 && b < a.B) {
                 const int Pb = a.prefix_len[b];
-                const long long kv0 = a.kv_start[b];
+                const long long kv0 = PAGED ? 0 : a.kv_start[b];
                 if (Pb < 0 || Pb > a.max_prefix_len || kv0 < 0 || kv0 + Pb > P.cache_rows) set_status(P.status, RADAR_ERR_INVALID_ARG);
             }
 #pragma unroll
@@ -199,7 +204,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         int fb = -1, fg = 0;
         for (int b0 = 0; b0 < a.B && fb < 0; b0 += 32) {
             const int b = b0 + lane;
-            const long long sz = b < a.B ? seq_cost(P, b, pp) : 0;
+            const long long sz = b < a.B ? seq_cost<PAGED>(P, b, pp) : 0;
             long long incl = sz;
 #pragma unroll
             for (int o = 1; o < 32; o <<= 1) {
@@ -211,7 +216,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 const int src = __ffs(hit) - 1;
                 const long long before = cum + __shfl_sync(kFull, incl - sz, src);
                 fb = b0 + src;
-                const SeqInfo si = seq_info(P, fb, pp);
+                const SeqInfo si = seq_info<PAGED>(P, fb, pp);
                 const long long unit = (long long)si.nt * si.w;
                 fg = (int)((lo - before) / unit);
                 fU = before + fg * unit;
@@ -252,13 +257,13 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     volatile int* ab = &s_abort;
 
     // first segment: the unit that contains the range's start, from its first tile starting at or after it
-    Cursor cur;
+    Cursor<PAGED> cur;
     cur.b = s_start[0]; cur.g = s_start[1];
     cur.hi = s_range[1];
     cur.U = s_range[3];
     cur.t0 = cur.t1 = 0;
     if (cur.b >= 0) {
-        cur.s = seq_info(P, cur.b, pp);
+        cur.s = seq_info<PAGED>(P, cur.b, pp);
         cur.t0 = tiles_before(s_range[0], cur.U, cur.s.nt, cur.s.w);
         if (cur.t0 >= cur.s.nt) cur.next_unit(P, pp);       // every tile of that unit starts before the range
         else cur.clip();
@@ -307,11 +312,27 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                         mbar_arrive_expect_tx(full, kTreeKeys * D * 2);
                         for (int h = 0; h < H; ++h)
                             tma_load_3d(dst + h * (kTreeKeys * 128), is_k ? &tmKt : &tmVt, full, h * 64, g, b * kMaxNodes);
-                    } else {
+                    } else if (!PAGED) {
                         mbar_arrive_expect_tx(full, kTileKeys * D * 2);
                         const int row = (int)(cur.s.kv0 + (long long)t * kTileKeys);
                         for (int h = 0; h < H; ++h)
                             tma_load_3d(dst + h * (kTileKeys * 128), is_k ? &tmKc : &tmVc, full, h * 64, g, row);
+                    } else {
+                        // paged cache: one box per page (or per tile when a page holds whole tiles); only pages
+                        // that hold live keys are fetched, what stays stale in the slot is masked / never read
+                        const int ps = a.page_size, per = min(ps, kTileKeys);
+                        const int key0 = t * kTileKeys;
+                        const int n_ld = (min(kTileKeys, cur.s.Pb - key0) + per - 1) / per;
+                        const long long n_cache_pages = P.cache_rows / ps;
+                        mbar_arrive_expect_tx(full, n_ld * per * D * 2);
+                        for (int p = 0; p < n_ld; ++p) {
+                            const int key = key0 + p * per;
+                            long long page = __ldg(a.block_table + (long long)b * a.max_pages + key / ps);
+                            if (page < 0 || page >= n_cache_pages) { set_status(P.status, RADAR_ERR_INVALID_ARG); page = 0; }
+                            const int row = (int)(page * ps + key % ps);
+                            for (int h = 0; h < H; ++h)
+                                tma_load_3d(dst + h * (kTileKeys * 128) + p * per * 128, is_k ? &tmKc : &tmVc, full, h * 64, g, row);
+                        }
                     }
                 };
                 // same order as the MMA warp consumes: the first K tile(s), then V(i), K(i + lookahead)
@@ -919,27 +940,28 @@ size_t tree_attn_tc_workspace_bytes(const radar_ctx* ctx, int B, int Hq, int Hkv
            align_up((size_t)n_cls * ncc * sizeof(CutUnit), 256);
 }
 
-template <int D, bool TWO>
+template <int D, bool TWO, bool PAGED>
 static int launch_tc(radar_ctx* ctx, TcParams& P, cudaStream_t stream) {
     const radar_attn_args& a = P.a;
     CUtensorMap tmQ, tmKc, tmVc, tmKt, tmVt;
     const long long tree_rows = (long long)a.B * kMaxNodes;
     const bool have_prefix = a.Kc != nullptr && a.Vc != nullptr && a.cache_rows > 0;
+    const int cache_box = a.block_table != nullptr && a.page_size < kTileKeys ? a.page_size : kTileKeys;   // rows per TMA box
     if (!make_map(&tmQ, a.Q, D, a.Hq, tree_rows, P.G, P.nodes_per_rb) ||
         !make_map(&tmKt, a.Kt, D, a.Hkv, tree_rows, 1, kTreeKeys) ||
         !make_map(&tmVt, a.Vt, D, a.Hkv, tree_rows, 1, kTreeKeys) ||
-        !make_map(&tmKc, have_prefix ? a.Kc : a.Kt, D, a.Hkv, have_prefix ? a.cache_rows : tree_rows, 1, kTileKeys) ||
-        !make_map(&tmVc, have_prefix ? a.Vc : a.Vt, D, a.Hkv, have_prefix ? a.cache_rows : tree_rows, 1, kTileKeys))
+        !make_map(&tmKc, have_prefix ? a.Kc : a.Kt, D, a.Hkv, have_prefix ? a.cache_rows : tree_rows, 1, cache_box) ||
+        !make_map(&tmVc, have_prefix ? a.Vc : a.Vt, D, a.Hkv, have_prefix ? a.cache_rows : tree_rows, 1, cache_box))
         return RADAR_ERR_CUDA;
     static bool attr_done = false;                  // once per process and instantiation: not a stream operation
     if (!attr_done) {
-        RADAR_CUDA_CHECK(cudaFuncSetAttribute(tree_attn_tc_kernel<D, TWO>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        RADAR_CUDA_CHECK(cudaFuncSetAttribute(tree_attn_tc_kernel<D, TWO, PAGED>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                               Smem<D, TWO>::kDynamic));
         attr_done = true;
     }
     {
         radar_launch_scope scope(ctx, RADAR_K_ATTN, stream);
-        RADAR_CUDA_CHECK(launch_chained(tree_attn_tc_kernel<D, TWO>, dim3((unsigned)(P.n_cls * P.ncc)), dim3(kTcThreads),
+        RADAR_CUDA_CHECK(launch_chained(tree_attn_tc_kernel<D, TWO, PAGED>, dim3((unsigned)(P.n_cls * P.ncc)), dim3(kTcThreads),
                                         (size_t)Smem<D, TWO>::kDynamic, stream, tmQ, tmKc, tmVc, tmKt, tmVt, P));
     }
     RADAR_CUDA_CHECK(cudaGetLastError());
@@ -972,8 +994,12 @@ int tree_attn_tc_launch(radar_ctx* ctx, const radar_attn_args* a, cudaStream_t s
     P.part_o = reinterpret_cast<float*>(reinterpret_cast<char*>(a->workspace) + align_up(rec * sizeof(float2), 256));
     P.cut = reinterpret_cast<CutUnit*>(reinterpret_cast<char*>(P.part_o) + align_up(rec * a->d * sizeof(float), 256));
     const bool two = P.pair_rows > 128 && P.G * kMaxNodes > 128;      // some unit can have two live row blocks
-    if (a->d == 128) return two ? launch_tc<128, true>(ctx, P, stream) : launch_tc<128, false>(ctx, P, stream);
-    return two ? launch_tc<64, true>(ctx, P, stream) : launch_tc<64, false>(ctx, P, stream);
+    if (a->block_table != nullptr) {
+        if (a->d == 128) return two ? launch_tc<128, true, true>(ctx, P, stream) : launch_tc<128, false, true>(ctx, P, stream);
+        return two ? launch_tc<64, true, true>(ctx, P, stream) : launch_tc<64, false, true>(ctx, P, stream);
+    }
+    if (a->d == 128) return two ? launch_tc<128, true, false>(ctx, P, stream) : launch_tc<128, false, false>(ctx, P, stream);
+    return two ? launch_tc<64, true, false>(ctx, P, stream) : launch_tc<64, false, false>(ctx, P, stream);
 }
 
 }  // namespace radar

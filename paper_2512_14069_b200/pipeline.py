@@ -103,12 +103,12 @@ class SpecStep:
             tree_score=self.tree_score, tree_mask=self.tree_mask, n_nodes=self.n_nodes, retrieve=self.retrieve,
             n_leaves=self.n_leaves)
 
-    def attention(self, Q, Kc, Vc, kv_start, prefix_len, Kt, Vt, mask=None, n_nodes=None):
+    def attention(self, Q, Kc, Vc, kv_start, prefix_len, Kt, Vt, mask=None, n_nodes=None, block_table=None, page_size=0):
         rb.radar_tree_attention(
             self.ctx, B=self.B, Hq=self.Hq, Hkv=self.Hkv, d=self.d, Q=Q, Kc=Kc, Vc=Vc, kv_start=kv_start,
             prefix_len=prefix_len, max_prefix_len=self.max_prefix_len, Kt=Kt, Vt=Vt,
             mask=self.tree_mask if mask is None else mask, n_nodes=self.n_nodes if n_nodes is None else n_nodes,
-            O=self.O, lse=self.lse, workspace=self.ws_attn)
+            O=self.O, lse=self.lse, workspace=self.ws_attn, block_table=block_table, page_size=page_size)
 
     def accept(self, target_logits, draft_logits=None, u_accept=None, u_sample=None):
         rb.radar_verify_accept(

@@ -116,13 +116,40 @@ class GpuRun:
         s.build_tree(self.root_tok, self.prefix_len, self.n_keep)
         self.ctx.check_device_status()
 
-    def upload_attention(self):
+    def upload_attention(self, page_size=None, spare_pages=3):
+        """Contiguous (packed) prefix cache, or with `page_size` a paged one: the same K/V rows scattered
+        over shuffled pages, a block table per sequence, unused table entries -1, and NaN in every cache
+        row that belongs to no token (page tails, spare pages), so that a read of them cannot go unnoticed."""
         inp, torch = self.inp, self.torch
         self.Q, self.Kt, self.Vt = to_dev(inp["Q"]), to_dev(inp["Kt"]), to_dev(inp["Vt"])
-        self.Kc = to_dev(np.concatenate(inp["Kc"], 0))
-        self.Vc = to_dev(np.concatenate(inp["Vc"], 0))
-        start = np.concatenate([[0], np.cumsum(inp["prefix_len"])[:-1]]).astype(np.int64)
-        self.kv_start = to_dev(start)
+        self.block_table, self.page_size = None, 0
+        if page_size is None:
+            self.Kc = to_dev(np.concatenate(inp["Kc"], 0))
+            self.Vc = to_dev(np.concatenate(inp["Vc"], 0))
+            start = np.concatenate([[0], np.cumsum(inp["prefix_len"])[:-1]]).astype(np.int64)
+            self.kv_start = to_dev(start)
+            return
+        ps = page_size
+        need = [(int(p) + ps - 1) // ps for p in inp["prefix_len"]]
+        n_pages = sum(need) + spare_pages
+        order = np.random.default_rng(1000 + ps).permutation(n_pages)
+        max_pages = max(max(need), 1) + 1
+        table = np.full((self.cfg.B, max_pages), -1, np.int32)
+        sample = inp["Kc"][0]
+        nan = np.uint16(0x7FC0) if sample.dtype == np.uint16 else np.float32(np.nan)
+        Kc = np.full((n_pages * ps,) + sample.shape[1:], nan, sample.dtype)
+        Vc = np.full_like(Kc, nan)
+        nxt = 0
+        for b in range(self.cfg.B):
+            for p in range(need[b]):
+                page = int(order[nxt]); nxt += 1
+                table[b, p] = page
+                rows = inp["Kc"][b][p * ps:(p + 1) * ps]
+                Kc[page * ps:page * ps + len(rows)] = rows
+                Vc[page * ps:page * ps + len(rows)] = inp["Vc"][b][p * ps:(p + 1) * ps]
+        self.Kc, self.Vc = to_dev(Kc), to_dev(Vc)
+        self.kv_start = None
+        self.block_table, self.page_size = to_dev(table), ps
 
     def attention(self, trees=None):
         """With `trees` (oracle trees) the masks come from the generator side, so attention can be
@@ -133,7 +160,8 @@ class GpuRun:
             n_nodes = to_dev(np.array([t["n_nodes"] for t in trees], np.int32))
         else:
             mask = n_nodes = None
-        s.attention(self.Q, self.Kc, self.Vc, self.kv_start, self.prefix_len, self.Kt, self.Vt, mask, n_nodes)
+        s.attention(self.Q, self.Kc, self.Vc, self.kv_start, self.prefix_len, self.Kt, self.Vt, mask, n_nodes,
+                    block_table=self.block_table, page_size=self.page_size)
         self.ctx.check_device_status()
         return s.O.float().cpu().numpy(), s.lse.cpu().numpy()
 

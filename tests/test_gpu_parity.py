@@ -207,6 +207,49 @@ def test_attention_bf16_head_layouts(ctx, Hq, Hkv, d):
     H.compare_attention(cfg, O_gpu, lse_gpu, O_ref, lse_ref, trees)
 
 
+@pytest.mark.parametrize("page_size,Hq,Hkv,dtype", [(16, 8, 2, "bf16"), (64, 8, 8, "bf16"), (128, 16, 2, "bf16"),
+                                                    (256, 8, 2, "bf16"), (32, 6, 3, "bf16"), (16, 4, 2, "f32")])
+def test_attention_paged_prefix_cache(ctx, page_size, Hq, Hkv, dtype):
+    """The prefix K/V scattered over shuffled pages (16 to 256 tokens) and read through a block table: same
+    outputs as the oracle computes from the logical rows.  Ragged prefixes, one empty, one shorter than a page,
+    one ending exactly on a page boundary; rows of the cache that belong to no token hold NaN.
+    (6 query / 3 KV heads and fp32 take the FMA kernel, the others the tensor-core kernel.)"""
+    base = W.CONFIGS[5] if dtype == "bf16" else W.CONFIGS[1]
+    cfg = W.shrink(base, cid=120 + page_size + Hq, B=5, Hq=Hq, Hkv=Hkv, d=128 if dtype == "bf16" else 64,
+                   P=(200, 1500), V=2000, k=4, t_max=5, N=50)
+    inp = H.make_inputs(cfg)
+    for b, plen in ((0, 0), (1, 5), (2, 4 * page_size)):
+        inp["prefix_len"][b] = plen
+        inp["Kc"][b], inp["Vc"][b] = W.attn_prefix_kv(cfg, b, plen) if plen else (inp["Kc"][b][:0], inp["Vc"][b][:0])
+    _, _, trees = H.oracle_expand_and_tree(cfg, inp)
+    g = H.GpuRun(cfg, inp, ctx)
+    g.upload_attention(page_size=page_size)
+    O_gpu, lse_gpu = g.attention(trees)
+    O_ref, lse_ref = H.oracle_attention(cfg, inp, trees)
+    H.compare_attention(cfg, O_gpu, lse_gpu, O_ref, lse_ref, trees)
+
+
+def test_attention_paged_reports_bad_page(ctx):
+    """A block-table entry outside the cache is reported on the device status word; nothing faults."""
+    import torch
+    from paper_2512_14069_b200 import binding as rb
+    cfg = W.shrink(W.CONFIGS[5], cid=97, B=2, Hq=8, Hkv=2, P=(300, 300), V=2000, k=4, t_max=4, N=30)
+    inp = H.make_inputs(cfg)
+    _, _, trees = H.oracle_expand_and_tree(cfg, inp)
+    g = H.GpuRun(cfg, inp, ctx)
+    g.upload_attention(page_size=64)
+    table = g.block_table.cpu().numpy().copy()
+    table[1, 2] = 10 ** 6
+    g.block_table = H.to_dev(table)
+    s = g.step
+    mask = H.to_dev(np.stack([t["mask"] for t in trees]).view(np.int64))
+    n_nodes = H.to_dev(np.array([t["n_nodes"] for t in trees], np.int32))
+    s.attention(g.Q, g.Kc, g.Vc, None, g.prefix_len, g.Kt, g.Vt, mask, n_nodes, block_table=g.block_table, page_size=64)
+    torch.cuda.synchronize()
+    assert ctx.read_device_status() == -1
+    assert ctx.read_device_status() == rb.RADAR_OK
+
+
 def test_attention_long_prefix_many_segments(ctx):
     """One long and three short sequences: the long one's units are cut across many CTAs (partials + combine),
     the short ones share CTAs with it."""
