@@ -278,7 +278,11 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
 
     if (warp == kProducerWarp) {
         // =================================== TMA producer ===================================
-        if (lane == 0) {
+        // One lane does everything for the contiguous cache.  With a paged cache the whole warp walks the same
+        // loop and lane p looks up and fetches page p of a tile (up to eight boxes per tile), the leading lane
+        // still doing the waits, the byte counts, Q and the tree tile.
+        if (PAGED || lane == 0) {
+            const bool lead = lane == 0;
             uint32_t kc = 0, vc = 0;
             bool ok = true;
             CutUnit cu;
@@ -290,8 +294,8 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                     cu.valid = 1; cu.b = b; cu.g = g; cu.nt = cur.s.nt; cu.slot = seg == 0 ? 0 : 1;
                     cu.rows = cur.s.rows; cu.w = cur.s.w; cu.u0 = cur.U; cu.tot = s_range[2];
                 }
-                ok = ok && mbar_wait(&bar_qempty, (seg & 1) ^ 1, ab);
-                if (ok) {
+                if (lead) ok = ok && mbar_wait(&bar_qempty, (seg & 1) ^ 1, ab);
+                if (lead && ok) {
                     mbar_arrive_expect_tx(&bar_qfull, two ? 2 * SM::kQBlock : SM::kQBlock);
                     for (int q = 0; q < (two ? 2 : 1); ++q)
                         for (int h = 0; h < H; ++h)
@@ -307,11 +311,15 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                     uint64_t* full = is_k ? &bar_kfull[slot] : &bar_vfull[slot];
                     uint64_t* empty = is_k ? &bar_kempty[slot] : &bar_vempty[slot];
                     unsigned char* dst = (is_k ? sK : sV) + slot * SM::kTileBytes;
-                    if (!ok || !mbar_wait(empty, (use & 1) ^ 1, ab)) { ok = false; return; }
+                    if (lead && (!ok || !mbar_wait(empty, (use & 1) ^ 1, ab))) ok = false;
+                    if (PAGED) ok = __shfl_sync(kFull, ok, 0);
+                    if (!ok) return;
                     if (t == cur.s.nt - 1) {
-                        mbar_arrive_expect_tx(full, kTreeKeys * D * 2);
-                        for (int h = 0; h < H; ++h)
-                            tma_load_3d(dst + h * (kTreeKeys * 128), is_k ? &tmKt : &tmVt, full, h * 64, g, b * kMaxNodes);
+                        if (lead) {
+                            mbar_arrive_expect_tx(full, kTreeKeys * D * 2);
+                            for (int h = 0; h < H; ++h)
+                                tma_load_3d(dst + h * (kTreeKeys * 128), is_k ? &tmKt : &tmVt, full, h * 64, g, b * kMaxNodes);
+                        }
                     } else if (!PAGED) {
                         mbar_arrive_expect_tx(full, kTileKeys * D * 2);
                         const int row = (int)(cur.s.kv0 + (long long)t * kTileKeys);
@@ -324,8 +332,9 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                         const int key0 = t * kTileKeys;
                         const int n_ld = (min(kTileKeys, cur.s.Pb - key0) + per - 1) / per;
                         const long long n_cache_pages = P.cache_rows / ps;
-                        mbar_arrive_expect_tx(full, n_ld * per * D * 2);
-                        for (int p = 0; p < n_ld; ++p) {
+                        if (lead) mbar_arrive_expect_tx(full, n_ld * per * D * 2);
+                        __syncwarp();
+                        if (const int p = lane; p < n_ld) {
                             const int key = key0 + p * per;
                             long long page = __ldg(a.block_table + (long long)b * a.max_pages + key / ps);
                             if (page < 0 || page >= n_cache_pages) { set_status(P.status, RADAR_ERR_INVALID_ARG); page = 0; }
@@ -343,7 +352,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                     if (i + la < n) load_tile(cur.t0 + i + la, true);
                 }
             }
-            P.cut[blockIdx.x] = cu;
+            if (lead) P.cut[blockIdx.x] = cu;
         }
         __syncwarp();
     } else if (warp == kMmaWarp) {
