@@ -352,5 +352,22 @@ def test_host_side_argument_errors(ctx):
         s.d = 96
         s.attention(s.O, s.O, s.O, torch.zeros(1, dtype=torch.int64, device="cuda"), g.prefix_len, s.O, s.O)
     assert e.value.status == -2
+    s.d = cfg.d
+    # policy variants: an unknown policy, a hidden-state policy without features or with a ragged feature width
+    for kw in (dict(policy=7), dict(policy=rb.RADAR_POLICY_LSTM_HIDDEN),
+               dict(policy=rb.RADAR_POLICY_LSTM_HIDDEN, features=torch.zeros(cfg.t_max - 1, cfg.B, 6, device="cuda"))):
+        with pytest.raises(rb.RadarError) as e:
+            s.expand(1, g.draft, g.gate, **kw)
+        assert e.value.status == -1
+    # the memoryless policy needs only its own four tensors
+    mlp = {n: H.to_dev(v) for n, v in W.policy_weights(cfg, "mlp_scores").items()}
+    s.expand(1, g.draft, mlp, policy=rb.RADAR_POLICY_MLP_SCORES)
+    # paged cache: a page size that is neither 16/32/64 nor a multiple of 128, and a table too short for the prefix
+    kv = torch.zeros(512, cfg.Hkv, cfg.d, device="cuda")
+    table = torch.zeros(cfg.B, 1, dtype=torch.int32, device="cuda")
+    for ps in (48, 64):
+        with pytest.raises(rb.RadarError) as e:
+            s.attention(s.O, kv, kv, None, g.prefix_len, s.O[:, :, :cfg.Hkv], s.O[:, :, :cfg.Hkv], block_table=table, page_size=ps)
+        assert e.value.status == -1, ps
     torch.cuda.synchronize()
     assert ctx.read_device_status() == 0
