@@ -86,7 +86,7 @@ def to_dev(x, bf16=False):
     return t.cuda()
 
 
-class GpuRun:
+class CudaRun:
     """Uploads a workload and drives the library through `SpecStep`."""
 
     def __init__(self, cfg: W.Config, inp, ctx=None, max_prefix_len=None, logits_bf16=False):
@@ -187,7 +187,7 @@ def check_margins(cfg, traces, trees, accepts=None):
             assert accepts[b]["accept_margin"] > TAU_PROB and accepts[b]["sample_margin"] > TAU_PROB, (b, accepts[b])
 
 
-def compare_expansion(cfg, gpu: GpuRun, pools, traces):
+def compare_expansion(cfg, gpu: CudaRun, pools, traces):
     s = gpu.step
     g = lambda t: t.cpu().numpy()
     k = cfg.k
@@ -222,7 +222,7 @@ def compare_expansion(cfg, gpu: GpuRun, pools, traces):
             assert ch[i, b] == 0
 
 
-def compare_tree(cfg, gpu: GpuRun, trees):
+def compare_tree(cfg, gpu: CudaRun, trees):
     s = gpu.step
     g = lambda t: t.cpu().numpy()
     for b in range(cfg.B):
@@ -238,7 +238,7 @@ def compare_tree(cfg, gpu: GpuRun, trees):
         assert np.array_equal(g(s.retrieve)[b, :rows], t["retrieve"]) and np.all(g(s.retrieve)[b, rows:] == -1)
 
 
-def compare_accept(cfg, gpu: GpuRun, accepts):
+def compare_accept(cfg, gpu: CudaRun, accepts):
     s = gpu.step
     g = lambda t: t.cpu().numpy()
     for b in range(cfg.B):

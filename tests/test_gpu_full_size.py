@@ -41,7 +41,7 @@ def test_full_size_step_matches_oracle(ctx, cid):
     accepts = H.oracle_accept(cfg, inp, trees, target)
     H.check_margins(cfg, traces, trees, accepts)
 
-    g = H.GpuRun(cfg, inp, ctx)
+    g = H.CudaRun(cfg, inp, ctx)
     g.expand_and_tree()
     H.compare_expansion(cfg, g, pools, traces)
     H.compare_tree(cfg, g, trees)

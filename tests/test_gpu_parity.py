@@ -40,7 +40,7 @@ def test_whole_step_matches_oracle(ctx, cid):
     accepts = H.oracle_accept(cfg, inp, trees, target)
     H.check_margins(cfg, traces, trees, accepts)
 
-    g = H.GpuRun(cfg, inp, ctx)
+    g = H.CudaRun(cfg, inp, ctx)
     g.expand_and_tree()
     H.compare_expansion(cfg, g, pools, traces)
     H.compare_tree(cfg, g, trees)
@@ -74,7 +74,7 @@ def test_regression_workloads_match_oracle(ctx, name):
     target = H.make_target(cfg, inp, trees)
     accepts = H.oracle_accept(cfg, inp, trees, target)
     H.check_margins(cfg, traces, trees, accepts)
-    g = H.GpuRun(cfg, inp, ctx)
+    g = H.CudaRun(cfg, inp, ctx)
     g.expand_and_tree()
     H.compare_expansion(cfg, g, pools, traces)
     H.compare_tree(cfg, g, trees)
@@ -106,7 +106,7 @@ def test_policy_variants_match_oracle(ctx, policy, feat_dim):
         for tr in trace:
             assert tr["margin"] > H.TAU_SCORE and tr.get("gate_margin", 1.0) > H.TAU_SCORE
     assert len({len(t) for t in traces}) > 1 or policy == "mlp_scores"      # the hidden-state gate stops at different depths
-    g = H.GpuRun(cfg, inp, ctx)
+    g = H.CudaRun(cfg, inp, ctx)
     code = rb.RADAR_POLICY_MLP_SCORES if policy == "mlp_scores" else rb.RADAR_POLICY_LSTM_HIDDEN
     g.step.run_expansion(g.draft, {n: H.to_dev(v) for n, v in w.items()}, None, policy=code,
                          features=None if feats is None else H.to_dev(feats))
@@ -125,7 +125,7 @@ def test_accept_length_distribution_matches_oracle(ctx, cid, temperature):
     inp = H.make_inputs(cfg, with_attention=False)
     pools, traces, trees = H.oracle_expand_and_tree(cfg, inp)
     target = H.make_target(cfg, inp, trees)
-    g = H.GpuRun(cfg, inp, ctx)
+    g = H.CudaRun(cfg, inp, ctx)
     g.expand_and_tree()
     H.compare_tree(cfg, g, trees)
     s = g.step
@@ -160,7 +160,7 @@ def test_bf16_logits_with_many_ties(ctx, cid):
     target = W.bf16_bits_to_f32(W.f32_to_bf16_bits(target)).reshape(target.shape)
     gcfg = W.shrink(cfg, mode="greedy")
     accepts = H.oracle_accept(gcfg, inp, trees, target)
-    g = H.GpuRun(gcfg, inp, ctx, logits_bf16=True)
+    g = H.CudaRun(gcfg, inp, ctx, logits_bf16=True)
     g.expand_and_tree()
     for b in range(cfg.B):
         for tr in traces[b]:
@@ -183,7 +183,7 @@ def test_attention_with_oracle_masks_and_ragged_trees(ctx):
     inp["Kc"][0], inp["Vc"][0] = inp["Kc"][0][:1], inp["Vc"][0][:1]
     _, _, trees = H.oracle_expand_and_tree(cfg, inp)
     trees[1] = dict(trees[1]); trees[1]["n_nodes"] = 1                        # root only
-    g = H.GpuRun(cfg, inp, ctx)
+    g = H.CudaRun(cfg, inp, ctx)
     g.upload_attention()
     O_gpu, lse_gpu = g.attention(trees)
     O_ref, lse_ref = H.oracle_attention(cfg, inp, trees)
@@ -200,7 +200,7 @@ def test_attention_bf16_head_layouts(ctx, Hq, Hkv, d):
     inp["Kc"][0], inp["Vc"][0] = inp["Kc"][0][:0], inp["Vc"][0][:0]
     _, _, trees = H.oracle_expand_and_tree(cfg, inp)
     trees[2] = dict(trees[2]); trees[2]["n_nodes"] = 1
-    g = H.GpuRun(cfg, inp, ctx)
+    g = H.CudaRun(cfg, inp, ctx)
     g.upload_attention()
     O_gpu, lse_gpu = g.attention(trees)
     O_ref, lse_ref = H.oracle_attention(cfg, inp, trees)
@@ -222,7 +222,7 @@ def test_attention_paged_prefix_cache(ctx, page_size, Hq, Hkv, dtype):
         inp["prefix_len"][b] = plen
         inp["Kc"][b], inp["Vc"][b] = W.attn_prefix_kv(cfg, b, plen) if plen else (inp["Kc"][b][:0], inp["Vc"][b][:0])
     _, _, trees = H.oracle_expand_and_tree(cfg, inp)
-    g = H.GpuRun(cfg, inp, ctx)
+    g = H.CudaRun(cfg, inp, ctx)
     g.upload_attention(page_size=page_size)
     O_gpu, lse_gpu = g.attention(trees)
     O_ref, lse_ref = H.oracle_attention(cfg, inp, trees)
@@ -236,7 +236,7 @@ def test_attention_paged_reports_bad_page(ctx):
     cfg = W.shrink(W.CONFIGS[5], cid=97, B=2, Hq=8, Hkv=2, P=(300, 300), V=2000, k=4, t_max=4, N=30)
     inp = H.make_inputs(cfg)
     _, _, trees = H.oracle_expand_and_tree(cfg, inp)
-    g = H.GpuRun(cfg, inp, ctx)
+    g = H.CudaRun(cfg, inp, ctx)
     g.upload_attention(page_size=64)
     table = g.block_table.cpu().numpy().copy()
     table[1, 2] = 10 ** 6
@@ -260,7 +260,7 @@ def test_attention_long_prefix_many_segments(ctx):
     kc, vc = W.attn_prefix_kv(cfg, 1, long_len)
     inp["Kc"][1], inp["Vc"][1] = kc, vc
     _, _, trees = H.oracle_expand_and_tree(cfg, inp)
-    g = H.GpuRun(cfg, inp, ctx)
+    g = H.CudaRun(cfg, inp, ctx)
     g.upload_attention()
     O_gpu, lse_gpu = g.attention(trees)
     O_ref, lse_ref = H.oracle_attention(cfg, inp, trees)
@@ -274,7 +274,7 @@ def test_attention_reports_prefix_beyond_cache(ctx):
     cfg = W.shrink(W.CONFIGS[5], cid=98, B=2, Hq=8, Hkv=2, P=(300, 300), V=2000, k=4, t_max=4, N=30)
     inp = H.make_inputs(cfg)
     _, _, trees = H.oracle_expand_and_tree(cfg, inp)
-    g = H.GpuRun(cfg, inp, ctx, max_prefix_len=4096)
+    g = H.CudaRun(cfg, inp, ctx, max_prefix_len=4096)
     g.upload_attention()
     g.prefix_len = H.to_dev(np.array([300, 4000], np.int32))          # sequence 1 claims more rows than the cache holds
     s = g.step
@@ -291,7 +291,7 @@ def test_attention_fp32_head_dim_64_and_128(ctx):
         cfg = W.shrink(W.CONFIGS[1], cid=40 + d, B=2, Hq=4, Hkv=2, d=d, P=(257, 257))
         inp = H.make_inputs(cfg)
         _, _, trees = H.oracle_expand_and_tree(cfg, inp)
-        g = H.GpuRun(cfg, inp, ctx)
+        g = H.CudaRun(cfg, inp, ctx)
         g.upload_attention()
         O_gpu, lse_gpu = g.attention(trees)
         O_ref, lse_ref = H.oracle_attention(cfg, inp, trees)
@@ -305,7 +305,7 @@ def test_expansion_edge_sizes(ctx, k, V):
     inp = H.make_inputs(cfg, with_attention=False)
     pools, traces, trees = H.oracle_expand_and_tree(cfg, inp)
     H.check_margins(cfg, traces, trees)
-    g = H.GpuRun(cfg, inp, ctx)
+    g = H.CudaRun(cfg, inp, ctx)
     g.expand_and_tree()
     H.compare_expansion(cfg, g, pools, traces)
     H.compare_tree(cfg, g, trees)
@@ -317,12 +317,12 @@ def test_minus_inf_logits_and_nan_status(ctx):
     inp = H.make_inputs(cfg, with_attention=False)
     inp["draft"][0, :, 5:200] = -np.inf
     pools, traces, trees = H.oracle_expand_and_tree(cfg, inp)
-    g = H.GpuRun(cfg, inp, ctx)
+    g = H.CudaRun(cfg, inp, ctx)
     g.expand_and_tree()
     H.compare_expansion(cfg, g, pools, traces)
     # a NaN is reported through the status word, nothing faults
     inp["draft"][0, 0, 17] = np.nan
-    g2 = H.GpuRun(cfg, inp, ctx)
+    g2 = H.CudaRun(cfg, inp, ctx)
     g2.step.run_expansion(g2.draft, g2.gate, g2.force)
     from paper_2512_14069_b200 import binding as rb
     assert ctx.read_device_status() == -6
@@ -335,7 +335,7 @@ def test_host_side_argument_errors(ctx):
     from paper_2512_14069_b200 import binding as rb
     cfg = W.CONFIGS[1]
     inp = H.make_inputs(cfg, with_attention=False)
-    g = H.GpuRun(cfg, inp, ctx)
+    g = H.CudaRun(cfg, inp, ctx)
     s = g.step
     with pytest.raises(rb.RadarError) as e:
         s.k = 33

@@ -28,7 +28,7 @@ def test_noalloc_greedy_accept_matches_regular_entry_point_twice_in_a_row():
     ctx = rb.Context(0)
     cfg = W.shrink(W.CONFIGS[4], B=3, Hq=8, Hkv=2, P=(64, 64), V=20011)
     inp = H.make_inputs(cfg, with_attention=False)
-    g = H.GpuRun(cfg, inp, ctx)
+    g = H.CudaRun(cfg, inp, ctx)
     g.expand_and_tree()
     s = g.step
     n_nodes = s.n_nodes.cpu().numpy()
