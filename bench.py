@@ -498,6 +498,7 @@ def run_ours(args):
         del copies, graphs
         torch.cuda.empty_cache()
         out["rooflines_at_scale"] = scale_probe(ctx, dev, peaks)
+        out["next_rows"] = next_rows_probe(ctx, dev)
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         out["cpu_baseline"] = cpu_baseline(cfg, budget_s=15.0)
     if rank == 0:
@@ -552,6 +553,72 @@ def _single_thread():
     except Exception:
         import contextlib
         return contextlib.nullcontext()
+
+
+def next_rows_probe(ctx, dev, reps=10):
+    """Device times of the kernels beyond the step itself: the acceptance-length distribution (Eq. 11-13) on the
+    trees of the Vicuna-13B configuration, and the
+    input-side kernel of the hidden-state policy at the draft model's width."""
+    import torch
+    from paper_2512_14069_b200 import binding as rb
+    from paper_2512_14069_b200.pipeline import SpecStep
+    cfg = W.CONFIGS[3]
+    B, V, k, t_max = cfg.B, cfg.V, cfg.k, cfg.t_max
+    step = SpecStep(ctx, B=B, V=V, k=k, t_max=t_max, N=cfg.N, Hq=cfg.Hq, Hkv=cfg.Hkv, d=cfg.d, kv_dtype=torch.bfloat16,
+                    max_prefix_len=128, mode=rb.RADAR_STOCHASTIC, device=dev)
+    draft_h = np.stack([W.draft_logits(cfg, b) for b in range(B)])
+    draft = torch.from_numpy(draft_h).to(dev)
+    gate = {n: torch.from_numpy(v).to(dev) for n, v in W.gate_weights(cfg).items()}
+    force = torch.full((B,), t_max, dtype=torch.int32, device=dev)
+    step.run_expansion(draft, gate, force)
+    step.build_tree(torch.from_numpy(W.root_tokens(cfg)).to(dev), torch.full((B,), 128, dtype=torch.int32, device=dev), None)
+    dr, nn = step.tree_draft_row.cpu().numpy(), step.n_nodes.cpu().numpy()
+    target_h = np.stack([W.target_logits(cfg, b, draft_h[b], dr[b], int(nn[b])) for b in range(B)])
+    target = torch.from_numpy(target_h).to(dev)
+    dist = torch.zeros(B, t_max + 1, dtype=torch.float64, device=dev)
+    pacc = torch.zeros(B, 64, dtype=torch.float64, device=dev)
+    wb = rb.radar_acclen_workspace_bytes(ctx, B, V)
+    ws = torch.zeros(wb + 256, dtype=torch.uint8, device=dev)
+    off = (-ws.data_ptr()) % 256
+
+    def run_acclen():
+        rb.radar_accept_length_distribution(
+            ctx, B=B, V=V, t_max=t_max, temperature=1.0, target_logits=target, tree_tok=step.tree_tok,
+            tree_parent=step.tree_parent, tree_depth=step.tree_depth, tree_draft_row=step.tree_draft_row,
+            n_nodes=step.n_nodes, draft_logits=draft, R=step.R, dist=dist, p_acc_node=pacc, workspace=ws[off:off + wb])
+
+    # hidden-state policy: input-side products at width 4096 for 8 sequences (one expansion call, t = 2)
+    cfg4 = W.shrink(W.CONFIGS[4], V=4096)
+    step4 = SpecStep(ctx, B=cfg4.B, V=cfg4.V, k=cfg4.k, t_max=cfg4.t_max, N=cfg4.N, Hq=cfg4.Hq, Hkv=cfg4.Hkv, d=cfg4.d,
+                     kv_dtype=torch.bfloat16, max_prefix_len=128, mode=rb.RADAR_GREEDY, device=dev)
+    w_hid = {n: torch.from_numpy(v).to(dev) for n, v in W.policy_weights(cfg4, "lstm_hidden", 4096).items()}
+    feats = torch.from_numpy(W.gate_features(cfg4, 4096)).to(dev)
+    draft4 = torch.randn(cfg4.B, step4.R, cfg4.V, device=dev)
+    force4 = torch.full((cfg4.B,), cfg4.t_max, dtype=torch.int32, device=dev)
+    step4.expand(1, draft4, w_hid, force4, rb.RADAR_POLICY_LSTM_HIDDEN, feats)
+
+    run_acclen()
+    torch.cuda.synchronize()
+    ctx.profile_begin(reps * 6)
+    torch.cuda._sleep(8_000_000)
+    for _ in range(reps):
+        run_acclen()
+        step4.active.fill_(1)
+        step4.pool_len.fill_(cfg4.k)
+        step4.expand(2, draft4, w_hid, force4, rb.RADAR_POLICY_LSTM_HIDDEN, feats)
+    torch.cuda.synchronize()
+    ctx.profile_end()
+    ctx.check_device_status()
+    ks = {n: 1000.0 * v[1] / v[2] for n, v in ctx.kernel_stats().items() if v[2] > 0}
+    internal = int(sum(len(set(step.tree_parent.cpu().numpy()[b, 1:nn[b]])) for b in range(B)))
+    return {
+        "accept_length_distribution": {
+            "workload": "Vicuna-13B configuration: %d trees, %d tree rows, %d internal rows, V = %d" % (B, int(nn.sum()), internal, V),
+            "nodes_kernel_us": round(ks.get("accept_length_nodes", 0.0), 1), "dist_kernel_us": round(ks.get("accept_length_dist", 0.0), 1)},
+        "hidden_state_policy": {
+            "workload": "8 sequences, feature width 4096: 640 x 4096 fp32 weights read once",
+            "gate_features_us": round(ks.get("gate_features", 0.0), 1), "select_gate_us": round(ks.get("expand_select_gate", 0.0), 1)},
+    }
 
 
 def cpu_baseline(cfg, budget_s):

@@ -25,39 +25,53 @@ struct SelectParams {
 };
 
 // Hidden-state policy (Table 3): the input-side products of the prediction model, W_ih f_b (4H rows) and the
-// head's columns for the input, W_1[:, H:] f_b (H rows), for every sequence.  One warp per output row; the
-// weights are read once, the feature rows come from L1/L2.  It needs nothing from the vocabulary pass and is
-// launched ahead of it.
-constexpr int kFeatRowsPerBlock = 8;
-__global__ void __launch_bounds__(kFeatRowsPerBlock * 32) gate_features_kernel(const radar_expand_args a, float* pre, float* hid) {
+// head's columns for the input, W_1[:, H:] f_b (H rows), for every sequence.  One block per output row, one
+// warp per 512-element segment of it: every weight is requested at once (the matrix is read at memory speed,
+// once), the feature rows come from L1/L2, the segments meet in shared memory.  It needs nothing from the
+// vocabulary pass and is launched ahead of it.
+constexpr int kFeatSeg = 512;                        // elements of a row per warp: 4 x float4 per lane
+__global__ void __launch_bounds__(1024) gate_features_kernel(const radar_expand_args a, float* pre, float* hid) {
     chain_wait();
-    const int H = kHidden, lane = threadIdx.x & 31;
-    const int r = blockIdx.x * kFeatRowsPerBlock + (threadIdx.x >> 5);          // 0 .. 5H-1
-    if (r >= 5 * H) return;
+    const int H = kHidden, lane = threadIdx.x & 31, seg = threadIdx.x >> 5, nseg = blockDim.x >> 5;
+    const int r = blockIdx.x;                        // 0 .. 5H-1
     const int d = a.feat_dim;
+    __shared__ float s_part[32][8];
     const float* w = r < 4 * H ? a.w_ih + (size_t)r * d : a.w1 + (size_t)(r - 4 * H) * (H + d) + H;
+    float4 wv[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int c = seg * kFeatSeg + i * 128 + lane * 4;
+        wv[i] = c < d ? __ldg(reinterpret_cast<const float4*>(w + c)) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
     for (int b0 = 0; b0 < a.B; b0 += 8) {
         float acc[8];
 #pragma unroll
-        for (int i = 0; i < 8; ++i) acc[i] = 0.f;
-        for (int c = lane * 4; c < d; c += 128) {
-            const float4 wv = __ldg(reinterpret_cast<const float4*>(w + c));
+        for (int j = 0; j < 8; ++j) acc[j] = 0.f;
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                if (b0 + i < a.B) {
-                    const float4 f = __ldg(reinterpret_cast<const float4*>(a.features + (size_t)(b0 + i) * d + c));
-                    acc[i] = fmaf(wv.x, f.x, fmaf(wv.y, f.y, fmaf(wv.z, f.z, fmaf(wv.w, f.w, acc[i]))));
+        for (int i = 0; i < 4; ++i) {
+            const int c = seg * kFeatSeg + i * 128 + lane * 4;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                if (c < d && b0 + j < a.B) {
+                    const float4 f = __ldg(reinterpret_cast<const float4*>(a.features + (size_t)(b0 + j) * d + c));
+                    acc[j] = fmaf(wv[i].x, f.x, fmaf(wv[i].y, f.y, fmaf(wv[i].z, f.z, fmaf(wv[i].w, f.w, acc[j]))));
                 }
             }
         }
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            const float v = warp_sum(acc[i]);
-            if (lane == 0 && b0 + i < a.B) {
-                if (r < 4 * H) pre[(size_t)(b0 + i) * 4 * H + r] = v;
-                else hid[(size_t)(b0 + i) * H + (r - 4 * H)] = v;
-            }
+        for (int j = 0; j < 8; ++j) {
+            const float v = warp_sum(acc[j]);
+            if (lane == 0) s_part[seg][j] = v;
         }
+        __syncthreads();
+        if (threadIdx.x < 8 && b0 + (int)threadIdx.x < a.B) {
+            float v = 0.f;
+            for (int q = 0; q < nseg; ++q) v += s_part[q][threadIdx.x];
+            const int b = b0 + threadIdx.x;
+            if (r < 4 * H) pre[(size_t)b * 4 * H + r] = v;
+            else hid[(size_t)b * H + (r - 4 * H)] = v;
+        }
+        __syncthreads();
     }
 }
 
@@ -459,8 +473,9 @@ extern "C" int radar_expand_step(radar_ctx* ctx, const radar_expand_args* a, voi
     sp.feat_hid = feat_pre + (size_t)a->B * 4 * kHidden;
     if (gate_runs && a->policy == RADAR_POLICY_LSTM_HIDDEN) {
         radar_launch_scope scope(ctx, RADAR_K_GATE_FEATURES, stream);
-        RADAR_CUDA_CHECK(launch_chained(gate_features_kernel, dim3((5 * kHidden + kFeatRowsPerBlock - 1) / kFeatRowsPerBlock),
-                                        dim3(kFeatRowsPerBlock * 32), 0, stream, *a, feat_pre, feat_pre + (size_t)a->B * 4 * kHidden));
+        const int nseg = (a->feat_dim + kFeatSeg - 1) / kFeatSeg;
+        RADAR_CUDA_CHECK(launch_chained(gate_features_kernel, dim3(5 * kHidden), dim3(nseg * 32), 0, stream, *a, feat_pre,
+                                        feat_pre + (size_t)a->B * 4 * kHidden));
     }
 
     RADAR_CUDA_CHECK(vocab_pass_launch(ctx, RADAR_K_VOCAB_EXPAND, vp, stream));
