@@ -125,7 +125,7 @@ __global__ void __launch_bounds__(kSelThreads, 1) expand_select_gate_kernel(cons
     __shared__ int s_ctok[kMaxF * RADAR_MAX_K];
     __shared__ float s_x[RADAR_MAX_K];                 // gate input
     __shared__ __align__(16) float s_h[kHidden];
-    __shared__ float s_hn[kHidden], s_pre[4 * kHidden], s_hid[kHidden];
+    __shared__ float s_hn[kHidden], s_pre[4 * kHidden], s_hid[kHidden], s_c[kHidden];
     __shared__ float s_b1[kHidden], s_w2[2 * kHidden], s_b2[2];
     __shared__ float s_y[2];
     __shared__ int s_base;
@@ -141,7 +141,11 @@ __global__ void __launch_bounds__(kSelThreads, 1) expand_select_gate_kernel(cons
         const int* gi = P.vp.part_i + row0 * per_row;
         chain_sync();
         if (P.staged) {
-            for (int e = tid; e < F * per_row; e += kMergeWarps * 32) { cp_async4(st_v + e, gv + e); cp_async4(st_i + e, gi + e); }
+            if ((per_row & 3) == 0) {       // rows of records are 16-byte aligned (the partial arrays are 256-byte aligned)
+                for (int e = tid; e < F * per_row / 4; e += kMergeWarps * 32) { cp_async16(st_v + 4 * e, gv + 4 * e); cp_async16(st_i + 4 * e, gi + 4 * e); }
+            } else {
+                for (int e = tid; e < F * per_row; e += kMergeWarps * 32) { cp_async4(st_v + e, gv + e); cp_async4(st_i + e, gi + e); }
+            }
             cp_async_wait_all();
             group_barrier(2);
         }
@@ -273,7 +277,11 @@ __global__ void __launch_bounds__(kSelThreads, 1) expand_select_gate_kernel(cons
             for (int e = gt; e < H * k; e += 512) cp_async16(s_wih + 4 * e, a.w_ih + 4 * e);          // 4H*k floats
             for (int e = gt; e < H * (H + k) / 4; e += 512) cp_async16(s_w1 + 4 * e, a.w1 + 4 * e);
         }
-        if (gt < H) s_h[gt] = a.t > 1 && policy != RADAR_POLICY_MLP_SCORES ? a.h[(size_t)b * H + gt] : 0.f;
+        if (gt < H) {
+            const bool state = a.t > 1 && policy != RADAR_POLICY_MLP_SCORES;
+            s_h[gt] = state ? a.h[(size_t)b * H + gt] : 0.f;
+            s_c[gt] = state ? a.c[(size_t)b * H + gt] : 0.f;
+        }
         group_barrier(3);
         const float4 h4 = *reinterpret_cast<const float4*>(&s_h[lane * 4]);
         constexpr int kBatch = 8;
@@ -373,7 +381,7 @@ __global__ void __launch_bounds__(kSelThreads, 1) expand_select_gate_kernel(cons
             const float fg = sigmoidf_(s_pre[H + tid]);
             const float gg = tanhf(s_pre[2 * H + tid]);
             const float og = sigmoidf_(s_pre[3 * H + tid]);
-            const float cn = fg * (a.t > 1 ? a.c[(size_t)b * H + tid] : 0.f) + ig * gg;
+            const float cn = fg * s_c[tid] + ig * gg;
             const float hn = og * tanhf(cn);
             a.c[(size_t)b * H + tid] = cn;
             a.h[(size_t)b * H + tid] = hn;
