@@ -34,10 +34,10 @@ L2_BYTES = 126 * 1024 * 1024
 # captures summarised under profiles/ (kernel name, config id); traffic of a launch at the same shapes =
 # ratio x its algorithmic bytes (both grow with the rows processed).  Absent = not captured.
 NCU_TRAFFIC_RATIO = {
-    ("tree_attention", 4): 452.14 / 284.58,
-    ("tree_attention", 3): 353.33 / 343.57,
-    ("vocab_pass(expand)", 4): 35.946 / 35.912,
-    ("vocab_pass(accept)", 4): 228.53 / 224.70,
+    ("tree_attention", 4): 451.76 / 284.58,
+    ("tree_attention", 3): 354.38 / 343.57,
+    ("vocab_pass(expand)", 4): 35.949 / 35.912,
+    ("vocab_pass(accept)", 4): 228.71 / 224.70,
 }
 
 
