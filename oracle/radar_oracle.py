@@ -142,6 +142,9 @@ def expand_step_seq(logits, parent_score, parent_pool_idx, pool: Pool, t: int, k
         "frontier_pool_idx": (base + sel).astype(np.int32),
         "frontier_src_row": (sel // k).astype(np.int32),
         "margin": margin,
+        # which candidates the margin is about (reporting only): pool indices and scores of the best k+1
+        "head_pool_idx": (base + order[: min(k + 1, flat.size)]).astype(np.int64),
+        "head_score": head.copy(),
     }
 
 
@@ -276,8 +279,10 @@ def rerank_build_tree(pool: Pool, N: int, root_tok: int, prefix_len: int, t_max:
         raise ValueError("tree does not fit a 64-bit mask")
     order = order_desc(pool.score[:L])
     margin = np.inf
+    cut_pair = None                     # the last kept and the first dropped entry (reporting only)
     if n_eff < L and n_eff > 0:
         margin = float(np.float64(pool.score[order[n_eff - 1]]) - np.float64(pool.score[order[n_eff]]))
+        cut_pair = (int(order[n_eff - 1]), int(order[n_eff]))
     kept = np.sort(order[:n_eff])
     M = n_eff + 1
     node_of = {-1: 0}
@@ -328,7 +333,7 @@ def rerank_build_tree(pool: Pool, N: int, root_tok: int, prefix_len: int, t_max:
     return {
         "n_nodes": M, "tok": tok, "parent": parent, "depth": depth, "pos": pos,
         "pool_idx": pidx, "score": score, "draft_row": drow, "mask": mask,
-        "retrieve": retrieve, "n_leaves": len(leaves), "margin": margin,
+        "retrieve": retrieve, "n_leaves": len(leaves), "margin": margin, "cut_pair": cut_pair,
     }
 
 

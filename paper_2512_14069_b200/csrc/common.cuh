@@ -4,6 +4,8 @@
 #include <cuda_runtime.h>
 #include <math_constants.h>
 #include <stdint.h>
+#include <stdio.h>
+#include <stdlib.h>
 
 #include "../../include/radar.h"
 
@@ -88,10 +90,15 @@ __device__ __forceinline__ void chain_wait() {
 __device__ __forceinline__ void chain_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void chain_sync() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
-#define RADAR_CUDA_CHECK(expr)                         \
-    do {                                               \
-        cudaError_t _e = (expr);                       \
-        if (_e != cudaSuccess) return RADAR_ERR_CUDA;  \
+// A failing runtime call becomes RADAR_ERR_CUDA; with RADAR_DEBUG set in the environment the call and the
+// runtime's message are also written to stderr.
+#define RADAR_CUDA_CHECK(expr)                                                                     \
+    do {                                                                                           \
+        cudaError_t _e = (expr);                                                                   \
+        if (_e != cudaSuccess) {                                                                   \
+            if (getenv("RADAR_DEBUG")) fprintf(stderr, "radar: %s -> %s\n", #expr, cudaGetErrorString(_e)); \
+            return RADAR_ERR_CUDA;                                                                 \
+        }                                                                                          \
     } while (0)
 
 namespace radar {

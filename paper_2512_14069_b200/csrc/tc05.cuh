@@ -35,12 +35,14 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
     return ok != 0;
 }
 // Bounded wait: gives up after `limit` polls (each poll itself blocks for a hardware-defined short
-// time) or as soon as *abort is set by another thread.  Returns false on give-up and sets *abort.
+// time) or once *abort_flag has been set by another thread.  Returns false on give-up and sets the
+// flag.  A wait that is satisfied at once costs one try_wait and nothing else: the flag is looked at
+// only while polling (reading it on every wait cost more than the wait itself).
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
                                           uint32_t limit = 4u << 20) {
-    if (mbar_try_wait(bar, parity)) return !*abort_flag;
+    if (mbar_try_wait(bar, parity)) return true;
     for (uint32_t it = 0; it < limit; ++it) {
-        if (mbar_try_wait(bar, parity)) return !*abort_flag;
+        if (mbar_try_wait(bar, parity)) return true;
         if ((it & 63u) == 63u) {
             if (*abort_flag) return false;
             __nanosleep(64);
@@ -128,6 +130,99 @@ __device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_
         "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
         ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"((uint32_t)accumulate)
         : "memory");
+}
+// Predicated forms for a warp that runs the issue code converged: every lane executes the instruction
+// stream (so the descriptor arithmetic stays warp-uniform), the lane with `pred` != 0 issues.
+__device__ __forceinline__ uint32_t elect_one() {
+    uint32_t pred;
+    asm volatile("{\n\t.reg .pred p;\n\t.reg .b32 r;\n\telect.sync r|p, 0xffffffff;\n\tselp.u32 %0, 1, 0, p;\n\t}" : "=r"(pred));
+    return pred;
+}
+__device__ __forceinline__ void mma_ss_if(uint32_t pred, uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                          bool accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "setp.ne.b32 q, %5, 0;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"((uint32_t)accumulate), "r"(pred)
+        : "memory");
+}
+__device__ __forceinline__ void mma_ts_if(uint32_t pred, uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
+                                          bool accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "setp.ne.b32 q, %5, 0;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"((uint32_t)accumulate), "r"(pred)
+        : "memory");
+}
+__device__ __forceinline__ void mma_commit_if(uint32_t pred, uint64_t* bar) {
+    asm volatile(
+        "{\n\t.reg .pred q;\n\t"
+        "setp.ne.b32 q, %1, 0;\n\t"
+        "@q tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}"
+        ::"r"(smem_u32(bar)), "r"(pred)
+        : "memory");
+}
+// Groups of MMAs over consecutive K steps in ONE instruction sequence: the descriptor low words advance by a
+// constant per step, the predicates are set once.  All lanes execute the sequence, the lane with pred != 0
+// issues.  `hi` is the high word shared by all shared-memory descriptors of the kernel.
+//   SS: four steps of 16 K-elements inside one 64-element swizzle block (32 B = 2 descriptor units per step).
+__device__ __forceinline__ void mma_ss_x4(uint32_t pred, uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t hi,
+                                          uint32_t idesc, bool acc_first) {
+    asm volatile(
+        "{\n\t.reg .pred q, p0, p1;\n\t.reg .b32 a, b;\n\t.reg .b64 da, db;\n\t"
+        "setp.ne.b32 q, %0, 0;\n\t"
+        "setp.ne.b32 p0, %6, 0;\n\t"
+        "setp.eq.b32 p1, 0, 0;\n\t"
+        "mov.b64 da, {%2, %4};\n\tmov.b64 db, {%3, %4};\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], da, db, %5, p0;\n\t"
+        "add.u32 a, %2, 2;\n\tadd.u32 b, %3, 2;\n\tmov.b64 da, {a, %4};\n\tmov.b64 db, {b, %4};\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], da, db, %5, p1;\n\t"
+        "add.u32 a, %2, 4;\n\tadd.u32 b, %3, 4;\n\tmov.b64 da, {a, %4};\n\tmov.b64 db, {b, %4};\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], da, db, %5, p1;\n\t"
+        "add.u32 a, %2, 6;\n\tadd.u32 b, %3, 6;\n\tmov.b64 da, {a, %4};\n\tmov.b64 db, {b, %4};\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], da, db, %5, p1;\n\t}"
+        ::"r"(pred), "r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(hi), "r"(idesc), "r"((uint32_t)acc_first)
+        : "memory");
+}
+//   TS: four steps; A advances by 8 tensor-memory columns (16 bf16) and B by 128 descriptor units (16 rows of
+//   an N-major tile) per step.  Steps at or beyond `nsteps` are not issued.
+__device__ __forceinline__ void mma_ts_x4(uint32_t pred, uint32_t nsteps, uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo,
+                                          uint32_t hi, uint32_t idesc, bool acc_first) {
+#define RADAR_TS_STEP(K, P)                                                                            \
+        "setp.gt.and.u32 qk, %1, " #K ", q;\n\t"                                                        \
+        "add.u32 a, %3, " #K " * 8;\n\tadd.u32 b, %4, " #K " * 128;\n\tmov.b64 db, {b, %5};\n\t"         \
+        "@qk tcgen05.mma.cta_group::1.kind::f16 [%2], [a], db, %6, " #P ";\n\t"
+    asm volatile(
+        "{\n\t.reg .pred q, qk, p0, p1;\n\t.reg .b32 a, b;\n\t.reg .b64 db;\n\t"
+        "setp.ne.b32 q, %0, 0;\n\t"
+        "setp.ne.b32 p0, %7, 0;\n\t"
+        "setp.eq.b32 p1, 0, 0;\n\t"
+        RADAR_TS_STEP(0, p0) RADAR_TS_STEP(1, p1) RADAR_TS_STEP(2, p1) RADAR_TS_STEP(3, p1)
+        "}"
+        ::"r"(pred), "r"(nsteps), "r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(hi), "r"(idesc), "r"((uint32_t)acc_first)
+        : "memory");
+#undef RADAR_TS_STEP
+}
+//   TS, all four steps, no per-step predicate.
+__device__ __forceinline__ void mma_ts_x4_full(uint32_t pred, uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t hi,
+                                               uint32_t idesc, bool acc_first) {
+#define RADAR_TS_STEP(K, P)                                                                            \
+        "add.u32 a, %2, " #K " * 8;\n\tadd.u32 b, %3, " #K " * 128;\n\tmov.b64 db, {b, %4};\n\t"         \
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%1], [a], db, %5, " #P ";\n\t"
+    asm volatile(
+        "{\n\t.reg .pred q, p0, p1;\n\t.reg .b32 a, b;\n\t.reg .b64 db;\n\t"
+        "setp.ne.b32 q, %0, 0;\n\t"
+        "setp.ne.b32 p0, %6, 0;\n\t"
+        "setp.eq.b32 p1, 0, 0;\n\t"
+        RADAR_TS_STEP(0, p0) RADAR_TS_STEP(1, p1) RADAR_TS_STEP(2, p1) RADAR_TS_STEP(3, p1)
+        "}"
+        ::"r"(pred), "r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(hi), "r"(idesc), "r"((uint32_t)acc_first)
+        : "memory");
+#undef RADAR_TS_STEP
 }
 // The barrier receives one arrival once every MMA issued so far by this thread has completed.
 __device__ __forceinline__ void mma_commit(uint64_t* bar) {

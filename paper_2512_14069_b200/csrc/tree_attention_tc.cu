@@ -38,8 +38,9 @@ namespace {
 
 using namespace tc05;
 
-constexpr int kTcThreads = 320;      // 8 softmax warps, TMA producer, MMA issuer
-constexpr int kProducerWarp = 8, kMmaWarp = 9;
+constexpr int kTcThreads = 576;      // 16 softmax warps, TMA producer, MMA issuer
+constexpr int kProducerWarp = 16, kMmaWarp = 17;
+constexpr int kStaticSmem = 3072;    // barriers and exchange arrays: with the tiles exactly the 227 KB a block may have
 constexpr int kTileKeys = 128;       // keys per prefix tile
 constexpr int kTreeKeys = 64;        // keys of the tree tile (RADAR_MAX_NODES)
 constexpr int kPairRows = 256;       // query rows of a row-block pair (and the stride of partial records)
@@ -148,14 +149,14 @@ struct Smem {
     static constexpr int kRingK = 3;
     static constexpr int kRingV = TWO ? 2 : 3;
     static constexpr int kTotal = kQBytes + (kRingK + kRingV) * kTileBytes;
-    static constexpr int kDynamic = kTotal + 1024;          // slack for the 1024-byte alignment
+    static constexpr int kDynamic = kTotal;                 // starts on a 1024-byte boundary behind the static block
 };
 
 // TWO: the launch may contain units with two live row blocks; decides the shared-memory layout
 // PAGED: the prefix cache is read through a block table (a separate instantiation, so that the contiguous
 // layout's code is not touched by it)
 template <int D, bool TWO, bool PAGED>
-__global__ void __launch_bounds__(kTcThreads, 1)
+__global__ void __launch_bounds__(kTcThreads, 1)      // 18 warps are allocated as 20: 96 registers per thread
 tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmKc,
                     const __grid_constant__ CUtensorMap tmVc, const __grid_constant__ CUtensorMap tmKt,
                     const __grid_constant__ CUtensorMap tmVt, const TcParams P) {
@@ -170,18 +171,44 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     const int ci = blockIdx.x / P.n_cls;
     const int G = P.G;
 
-    extern __shared__ unsigned char smem_raw[];
-    unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    // Static block first (padded to a multiple of 1024 bytes and aligned to it), the tiles behind it: the
+    // swizzled tiles need a 1024-byte boundary and there is no room left for alignment slack.
+    struct __align__(1024) Static {
+        uint64_t bar_qfull, bar_qempty, bar_kfull[3], bar_kempty[3], bar_vfull[3], bar_vempty[3];
+        uint64_t bar_sfull[2], bar_pready[2], bar_odone[2], bar_ofree[2];
+        long long range[4];      // this CTA's range [lo, hi), size of the class's space, start of its first unit
+        int start[2];            // sequence and KV head of the unit that contains lo
+        uint32_t tmem_base;
+        int abort;
+        float xm[128];           // group 1's running max at the end of a segment (one live row block)
+        float mx[2][2][128];     // per group and column half: row maxima of a tile; row sums at the end of a segment
+        unsigned char pad[kStaticSmem - (22 * 8 + 4 * 8 + 2 * 4 + 4 + 4 + 128 * 4 + 2 * 2 * 128 * 4)];
+    };
+    static_assert(sizeof(Static) == kStaticSmem, "static shared-memory block");
+    __shared__ Static st;
+    extern __shared__ __align__(1024) unsigned char smem_raw[];
+    unsigned char* smem = smem_raw;
     unsigned char* sQ = smem;
     unsigned char* sK = smem + SM::kQBytes;
     unsigned char* sV = sK + RK * SM::kTileBytes;
-    __shared__ uint64_t bar_qfull, bar_qempty, bar_kfull[3], bar_kempty[3], bar_vfull[3], bar_vempty[3];
-    __shared__ uint64_t bar_sfull[2], bar_pready[2], bar_odone[2], bar_ofree[2];
-    __shared__ uint32_t s_tmem_base;
-    __shared__ int s_abort;
-    __shared__ float s_xm[128], s_xl[128];
-    __shared__ long long s_range[4];     // this CTA's range [lo, hi), size of the class's space, start of its first unit
-    __shared__ int s_start[2];           // sequence and KV head of the unit that contains lo
+    uint64_t& bar_qfull = st.bar_qfull;
+    uint64_t& bar_qempty = st.bar_qempty;
+    uint64_t (&bar_kfull)[3] = st.bar_kfull;
+    uint64_t (&bar_kempty)[3] = st.bar_kempty;
+    uint64_t (&bar_vfull)[3] = st.bar_vfull;
+    uint64_t (&bar_vempty)[3] = st.bar_vempty;
+    uint64_t (&bar_sfull)[2] = st.bar_sfull;
+    uint64_t (&bar_pready)[2] = st.bar_pready;
+    uint64_t (&bar_odone)[2] = st.bar_odone;
+    uint64_t (&bar_ofree)[2] = st.bar_ofree;
+    uint32_t& s_tmem_base = st.tmem_base;
+    int& s_abort = st.abort;
+    float (&s_xm)[128] = st.xm;
+    float (&s_mx)[2][2][128] = st.mx;
+    float (&s_xl)[2][2][128] = st.mx;        // same storage: the two uses never overlap in time
+    long long (&s_range)[4] = st.range;
+    int (&s_start)[2] = st.start;
+    const bool smem_aligned = (smem_u32(smem_raw) & 1023u) == 0;
 
     // ---- set-up: warp 0 finds this CTA's range while the barriers and tensor memory are prepared ----
     if (warp == 0) {
@@ -237,8 +264,8 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 mbar_init(&bar_vfull[i], 1); mbar_init(&bar_vempty[i], 1);
             }
             for (int i = 0; i < 2; ++i) {
-                mbar_init(&bar_sfull[i], 1); mbar_init(&bar_pready[i], 4);
-                mbar_init(&bar_odone[i], 1); mbar_init(&bar_ofree[i], 4);
+                mbar_init(&bar_sfull[i], 1); mbar_init(&bar_pready[i], 8);
+                mbar_init(&bar_odone[i], 1); mbar_init(&bar_ofree[i], 8);
             }
             fence_barrier_init();
         }
@@ -268,8 +295,11 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         if (cur.t0 >= cur.s.nt) cur.next_unit(P, pp);       // every tile of that unit starts before the range
         else cur.clip();
     }
-    if (!cur.valid()) {                                     // nothing for this CTA (uniform)
-        if (tid == 0) P.cut[blockIdx.x].valid = 0;
+    if (!cur.valid() || !smem_aligned) {                    // nothing for this CTA (uniform)
+        if (tid == 0) {
+            P.cut[blockIdx.x].valid = 0;
+            if (!smem_aligned) set_status(P.status, RADAR_ERR_CUDA);   // the tiles would not sit on their swizzle boundary
+        }
         tc_fence_before_sync();
         __syncthreads();
         if (warp == kProducerWarp) tmem_dealloc(tmem, 512);
@@ -357,126 +387,185 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         __syncwarp();
     } else if (warp == kMmaWarp) {
         // =================================== MMA issuer ===================================
-        // One thread waits, issues and commits; a tcgen05.mma takes some 60 cycles to issue, about as long
-        // as a 128 x 128 x 16 product runs, so whatever else this thread executes between two of them
-        // costs tensor-pipe time: the issue sequences are straight-line with precomputed descriptor words.
-        // The other lanes follow the same control flow and only help to clear V rows (rare).
+        // The warp runs converged: every lane waits on the barriers and executes the same straight-line issue
+        // sequences with warp-uniform descriptor words, and the elected lane issues the instructions and the
+        // commits (predicated, no branch around them).  Whatever this warp executes between two MMAs costs
+        // tensor-pipe time, so no control flow depends on a wait's outcome: after a wait that ran out the
+        // predicate is off and the loops run dry.
         constexpr uint32_t idesc_s128 = idesc_bf16_f32(128, kTileKeys, false, false);
         constexpr uint32_t idesc_s64 = idesc_bf16_f32(128, kTreeKeys, false, false);
         constexpr uint32_t idesc_pv = idesc_bf16_f32(128, D, false, true);
         // high word of every shared-memory descriptor (stride between 8-row groups 1024 B, version, swizzle)
-        constexpr uint64_t kDescHi = (uint64_t)((1024u >> 4) | (1u << 14) | (2u << 29)) << 32;
+        constexpr uint32_t kDescHi = (1024u >> 4) | (1u << 14) | (2u << 29);
         const uint32_t q_lo = ((smem_u32(sQ) & 0x3ffff) >> 4) | (1u << 16);
         const uint32_t k_lo = ((smem_u32(sK) & 0x3ffff) >> 4) | (1u << 16);
         const uint32_t v_lo = (smem_u32(sV) & 0x3ffff) >> 4;
-        const bool lead = lane == 0;
+        const uint32_t elected = elect_one();
         uint32_t k_next = 0, k_par = 0, v_next = 0, v_par = 0;   // ring slot to take next and its phase parity
-        uint32_t pr0 = 0, pr1 = 0;               // P tiles awaited per group
-        bool ok = true;                          // meaningful in the leading lane only
-        for (uint32_t seg = 0; cur.valid(); cur.next(P, pp), ++seg) {
-            const int n = cur.t1 - cur.t0;
-            const bool two = TWO && cur.two_rb();
-            const int M = cur.s.M, Pb = cur.s.Pb, nt_unit = cur.s.nt;
-            if (lead) ok = ok && mbar_wait(&bar_qfull, seg & 1, ab);
+        uint32_t p_par[2] = {0, 0};              // phase parity of the next P tile per group
+        bool ok = true;
+        // The segment's shape comes from global memory; passing it through a broadcast from lane 0 tells the
+        // compiler that it is the same in every lane, so that the loops below and the descriptor arithmetic in
+        // them stay on the uniform datapath (this warp's own instruction stream is what bounds the issue rate).
+        auto uni = [](int v) { return __shfl_sync(kFull, v, 0); };
+        for (uint32_t seg = 0; uni(cur.valid()); cur.next(P, pp), ++seg) {
+            const int seg_t0 = uni(cur.t0);
+            const int n = uni(cur.t1) - seg_t0;
+            const bool two = TWO && uni(cur.two_rb());
+            const int M = uni(cur.s.M), Pb = uni(cur.s.Pb), nt_unit = uni(cur.s.nt);
+            ok = ok && mbar_wait(&bar_qfull, seg & 1, ab);
             uint32_t k_slot = 0, v_slot = 0;      // ring slots of the K and V tiles in use
-            bool acc0 = false, acc1 = false;      // accumulator holds a product of this segment
+            bool acc[2] = {false, false};         // accumulator holds a product of this segment
+
+            // ---- O[q] (+)= P[q] V for tile i (q is a literal at every call site) ----
+            auto pv = [&](const int q, const int i, const bool fresh_v, const bool release_v) {
+                const bool tree = seg_t0 + i == nt_unit - 1;
+                const int nk = tree ? kTreeKeys : kTileKeys;
+                const int valid = tree ? M : min(kTileKeys, Pb - (seg_t0 + i) * kTileKeys);
+                const int ksteps = (valid + 15) >> 4;
+                ok = ok && mbar_wait(&bar_pready[q], p_par[q], ab);
+                p_par[q] ^= 1;
+                if (fresh_v) {
+                    v_slot = v_next;
+                    ok = ok && mbar_wait(&bar_vfull[v_slot], v_par, ab);
+                    if (++v_next == RV) { v_next = 0; v_par ^= 1; }
+                    if (valid < ksteps * 16) {
+                        // rows past the last live key meet P = 0; they must not hold NaN/Inf bit patterns
+                        unsigned char* vtile = sV + v_slot * SM::kTileBytes;
+                        const int nrows = ksteps * 16 - valid;
+                        for (int e = lane; e < nrows * 8 * H; e += 32) {
+                            const int h = e / (nrows * 8), rem = e % (nrows * 8);
+                            const int r = valid + rem / 8, c = rem % 8;
+                            *reinterpret_cast<uint4*>(vtile + h * (nk * 128) + r * 128 + c * 16) = make_uint4(0, 0, 0, 0);
+                        }
+                        fence_proxy_async_smem();
+                        __syncwarp();
+                    }
+                    if (i == 0) {                 // the previous segment's epilogue has read both accumulators
+                        ok = ok && mbar_wait(&bar_ofree[0], (seg & 1) ^ 1, ab);
+                        ok = ok && mbar_wait(&bar_ofree[1], (seg & 1) ^ 1, ab);
+                    }
+                }
+                tc_fence_after_sync();
+                const uint32_t go = ok ? elected : 0u;
+                // V is consumed N-major: 16 keys are 2048 B; 64-column blocks are nk * 128 B apart
+                const uint32_t b_lo = (v_lo + v_slot * (SM::kTileBytes >> 4)) | ((uint32_t)(nk * 128 >> 4) << 16);
+                // P of the first half of the tile's keys sits at column 0 of the group's buffer, of the second half
+                // at column 64 (each softmax thread writes inside its own column range)
+                const int hs = tree ? 2 : 4;
+                const uint32_t n1 = (uint32_t)min(ksteps, hs), n2 = (uint32_t)ksteps - n1;
+                mma_ts_x4(go, n1, tmem + 256 + q * 128, tmem + q * 128, b_lo, kDescHi, idesc_pv, acc[q]);
+                mma_ts_x4(go, n2, tmem + 256 + q * 128, tmem + q * 128 + 64, b_lo + hs * 128, kDescHi, idesc_pv, true);
+                acc[q] = true;
+                if (release_v) mma_commit_if(go, &bar_vempty[v_slot]);
+                if (two ? i == n - 1 : i + 2 >= n) mma_commit_if(go, &bar_odone[q]);
+            };
+            // ---- S[q] = Q K^T for tile si.  Nothing in tensor memory changes hands here: K arrives through the
+            // async proxy, and the buffer was last read by this thread's own P V, which runs first. ----
+            auto qk = [&](const int q, const int si, const bool fresh_k, const bool release_k) {
+                if (fresh_k) {
+                    k_slot = k_next;
+                    ok = ok && mbar_wait(&bar_kfull[k_slot], k_par, ab);
+                    if (++k_next == RK) { k_next = 0; k_par ^= 1; }
+                }
+                const uint32_t go = ok ? elected : 0u;
+                const bool tree = seg_t0 + si == nt_unit - 1;
+                const uint32_t a0 = q_lo + (two ? q : 0) * (SM::kQBlock >> 4);
+                const uint32_t b0 = k_lo + k_slot * (SM::kTileBytes >> 4);
+                const uint32_t idesc = tree ? idesc_s64 : idesc_s128;
+                mma_ss_x4(go, tmem + q * 128, a0, b0, kDescHi, idesc, false);
+                if (D == 128)                     // second 64-column block of Q and K
+                    mma_ss_x4(go, tmem + q * 128, a0 + (128 * 128 >> 4), b0 + ((uint32_t)((tree ? kTreeKeys : kTileKeys) * 128) >> 4),
+                              kDescHi, idesc, true);
+                if (release_k) mma_commit_if(go, &bar_kempty[k_slot]);
+                mma_commit_if(go, &bar_sfull[q]);
+                // the last S of the segment: Q may be overwritten once it has run
+                if (si == n - 1 && release_k) mma_commit_if(go, &bar_qempty);
+            };
             // Schedule.  Two live row blocks: group s owns row block s; per tile PV0(i) S0(i+1) PV1(i) S1(i+1),
             // both groups sharing K(i+1) and V(i).  One live row block: the groups take alternate tiles,
             // PV(i) S(i+2) for group i & 1.  S of the first tile(s) comes from the iterations with i < 0.
-            for (int i = two ? -1 : -2; i < n; ++i) {
-#pragma unroll 1
-                for (int qq = 0; qq < (two ? 2 : 1); ++qq) {
-                    const int q = two ? qq : (i & 1);
-                    if (i >= 0) {
-                        // ---- O[q] (+)= P V for tile i ----
-                        const bool tree = cur.t0 + i == nt_unit - 1;
-                        const int nk = tree ? kTreeKeys : kTileKeys;
-                        const int valid = tree ? M : min(kTileKeys, Pb - (cur.t0 + i) * kTileKeys);
-                        const int ksteps = (valid + 15) >> 4;
-                        if (lead) {
-                            ok = ok && mbar_wait(&bar_pready[q], (q ? pr1 : pr0) & 1, ab);
-                            if (q) ++pr1; else ++pr0;
-                        }
-                        if (!two || q == 0) {
-                            v_slot = v_next;
-                            if (lead) ok = ok && mbar_wait(&bar_vfull[v_slot], v_par, ab);
-                            if (++v_next == RV) { v_next = 0; v_par ^= 1; }
-                            if (valid < ksteps * 16) {
-                                // rows past the last live key meet P = 0; they must not hold NaN/Inf bit patterns
-                                __syncwarp();                                    // the tile has landed (leading lane waited)
-                                unsigned char* vtile = sV + v_slot * SM::kTileBytes;
-                                const int nrows = ksteps * 16 - valid;
-                                for (int e = lane; e < nrows * 8 * H; e += 32) {
-                                    const int h = e / (nrows * 8), rem = e % (nrows * 8);
-                                    const int r = valid + rem / 8, c = rem % 8;
-                                    *reinterpret_cast<uint4*>(vtile + h * (nk * 128) + r * 128 + c * 16) = make_uint4(0, 0, 0, 0);
-                                }
-                                fence_proxy_async_smem();
-                                __syncwarp();
-                            }
-                        }
-                        if (lead) {
-                            if (i == 0 && qq == 0) {      // the previous segment's epilogue has read both accumulators
-                                ok = ok && mbar_wait(&bar_ofree[0], (seg & 1) ^ 1, ab);
-                                ok = ok && mbar_wait(&bar_ofree[1], (seg & 1) ^ 1, ab);
-                            }
-                            tc_fence_after_sync();
-                            if (ok) {
-                                // V is consumed N-major: 16 keys are 2048 B; 64-column blocks are nk * 128 B apart
-                                const uint32_t b_lo = (v_lo + v_slot * (SM::kTileBytes >> 4)) | ((uint32_t)(nk * 128 >> 4) << 16);
-                                const uint32_t p_addr = tmem + q * 128;
-                                const uint32_t o_addr = tmem + 256 + q * 128;
-                                const bool acc = q ? acc1 : acc0;
-#pragma unroll
-                                for (int kk = 0; kk < kTileKeys / 16; ++kk)
-                                    if (kk < ksteps) mma_ts(o_addr, p_addr + kk * 8, kDescHi | (b_lo + kk * 128), idesc_pv, kk > 0 || acc);
-                                if (!two || q == 1) mma_commit(&bar_vempty[v_slot]);
-                                if (two ? i == n - 1 : i + 2 >= n) mma_commit(&bar_odone[q]);
-                            }
-                        }
-                        if (q) acc1 = true; else acc0 = true;
+            // Steady state (both tiles involved are full prefix tiles): the same steps with nothing to decide,
+            // so that the issuing warp executes as few instructions per MMA as possible.
+            const uint32_t a_q0 = q_lo, a_q1 = q_lo + (SM::kQBlock >> 4);
+            auto wait_all = [&](uint64_t* bar, uint32_t parity) { ok = mbar_wait(bar, parity, ab) && ok; };
+            auto pv_full = [&](const int q, const bool fresh_v, const bool release_v) {
+                wait_all(&bar_pready[q], p_par[q]);
+                p_par[q] ^= 1;
+                if (fresh_v) {
+                    v_slot = v_next;
+                    wait_all(&bar_vfull[v_slot], v_par);
+                    if (++v_next == RV) { v_next = 0; v_par ^= 1; }
+                }
+                tc_fence_after_sync();
+                const uint32_t go = ok ? elected : 0u;
+                const uint32_t b_lo = (v_lo + v_slot * (SM::kTileBytes >> 4)) | ((uint32_t)(kTileKeys * 128 >> 4) << 16);
+                mma_ts_x4_full(go, tmem + 256 + q * 128, tmem + q * 128, b_lo, kDescHi, idesc_pv, acc[q]);
+                mma_ts_x4_full(go, tmem + 256 + q * 128, tmem + q * 128 + 64, b_lo + 4 * 128, kDescHi, idesc_pv, true);
+                acc[q] = true;
+                if (release_v) mma_commit_if(go, &bar_vempty[v_slot]);
+            };
+            auto qk_full = [&](const int q, const uint32_t a0, const bool fresh_k, const bool release_k) {
+                if (fresh_k) {
+                    k_slot = k_next;
+                    wait_all(&bar_kfull[k_slot], k_par);
+                    if (++k_next == RK) { k_next = 0; k_par ^= 1; }
+                }
+                const uint32_t go = ok ? elected : 0u;
+                const uint32_t b0 = k_lo + k_slot * (SM::kTileBytes >> 4);
+                mma_ss_x4(go, tmem + q * 128, a0, b0, kDescHi, idesc_s128, false);
+                if (D == 128) mma_ss_x4(go, tmem + q * 128, a0 + (128 * 128 >> 4), b0 + (kTileKeys * 128 >> 4), kDescHi, idesc_s128, true);
+                if (release_k) mma_commit_if(go, &bar_kempty[k_slot]);
+                mma_commit_if(go, &bar_sfull[q]);
+            };
+            const int n_full = min(n, Pb / kTileKeys - seg_t0);   // tiles [0, n_full) of the segment are full prefix tiles
+            if (two) {
+                for (int i = -1; i < n; ++i) {
+                    if (i >= 0 && i + 2 < n_full) {           // tiles i and i+1 full, and S(i+1) is not the segment's last
+                        pv_full(0, true, false);
+                        qk_full(0, a_q0, true, false);
+                        pv_full(1, false, true);
+                        qk_full(1, a_q1, false, true);
+                    } else {
+                        if (i >= 0) pv(0, i, true, false);
+                        if (i + 1 < n) qk(0, i + 1, true, false);
+                        if (i >= 0) pv(1, i, false, true);
+                        if (i + 1 < n) qk(1, i + 1, false, true);
                     }
-                    const int si = two ? i + 1 : i + 2;
-                    if (si >= 0 && si < n) {
-                        // ---- S = Q K^T for tile si into group q's buffer (one live row block: si & 1 == q) ----
-                        const bool fresh_k = !two || q == 0, release_k = !two || q == 1;
-                        if (fresh_k) {
-                            k_slot = k_next;
-                            if (lead) ok = ok && mbar_wait(&bar_kfull[k_slot], k_par, ab);
-                            if (++k_next == RK) { k_next = 0; k_par ^= 1; }
+                }
+            } else {
+                for (int i = -2; i < n; ++i) {
+                    const bool fast = i >= 0 && i + 3 < n_full;   // tiles i and i+2 full, S(i+2) not the last
+                    if (i & 1) {
+                        if (fast) { pv_full(1, true, true); qk_full(1, a_q0, true, true); }
+                        else {
+                            if (i >= 0) pv(1, i, true, true);
+                            if (i + 2 < n) qk(1, i + 2, true, true);
                         }
-                        if (lead) {
-                            tc_fence_after_sync();
-                            if (ok) {
-                                const bool tree = cur.t0 + si == nt_unit - 1;
-                                const uint32_t a0 = q_lo + (two ? q : 0) * (SM::kQBlock >> 4);
-                                const uint32_t b0 = k_lo + k_slot * (SM::kTileBytes >> 4);
-                                const uint32_t b1 = b0 + ((uint32_t)((tree ? kTreeKeys : kTileKeys) * 128) >> 4);   // second 64-column block of K
-                                const uint32_t idesc = tree ? idesc_s64 : idesc_s128;
-                                const uint32_t d_addr = tmem + q * 128;
-#pragma unroll
-                                for (int kk = 0; kk < D / 16; ++kk) {
-                                    const uint32_t ko = (kk & 3) * 2;                 // 16 elements = 32 B within the 128-B row
-                                    mma_ss(d_addr, kDescHi | (a0 + (kk >> 2) * (128 * 128 >> 4) + ko), kDescHi | ((kk >> 2 ? b1 : b0) + ko), idesc, kk > 0);
-                                }
-                                if (release_k) mma_commit(&bar_kempty[k_slot]);
-                                mma_commit(&bar_sfull[q]);
-                            }
+                    } else {
+                        if (fast) { pv_full(0, true, true); qk_full(0, a_q0, true, true); }
+                        else {
+                            if (i >= 0) pv(0, i, true, true);
+                            if (i + 2 < n) qk(0, i + 2, true, true);
                         }
                     }
                 }
             }
-            if (lead && ok) mma_commit(&bar_qempty);           // every S of this segment has read Q
         }
         __syncwarp();
     } else {
         // =================================== softmax groups ===================================
-        const int grp = warp >> 2;
+        // Two threads per query row: warp w of a group's eight serves tensor-memory lanes 32 (w & 3) .. + 31
+        // and the column half (w >> 2) & 1, so a row's 128 scores are exponentiated by two threads at once
+        // and the chain S -> softmax -> P V of a group is about half as long.
+        const int grp = warp >> 3;
+        const int half = (warp >> 2) & 1;
         const int row = (warp & 3) * 32 + lane;                 // row of the block == tensor-memory lane
         const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
         const uint32_t tS = tmem + grp * 128 + lane_addr;
         const uint32_t tO = tmem + 256 + grp * 128 + lane_addr;
         const uint32_t tO_other = tmem + 256 + (grp ^ 1) * 128 + lane_addr;
+        constexpr int DH = D / 2;                               // accumulator columns per thread
         uint32_t sc = 0, oc = 0;                 // S tiles and accumulators this group has waited for
         bool ok = true;
         for (uint32_t seg = 0; cur.valid(); cur.next(P, pp), ++seg) {
@@ -488,10 +577,13 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             const int node = r_glob / G;
             const int hq = g * G + r_glob % G;
             const bool row_live = prow < cur.s.rows;
+            // A warp none of whose 32 rows is live does no arithmetic (the products of its rows are never read):
+            // it only keeps the barriers going.
+            const bool warp_live = prow - lane < cur.s.rows;
             const unsigned long long live_bits = M >= 64 ? ~0ull : ((1ull << M) - 1ull);
             const unsigned long long mask_bits = row_live ? (a.mask[(int64_t)b * kMaxNodes + node] & live_bits) : 0ull;
             const int n_my = two ? n : (n - grp + 1) >> 1;
-            float m_run = -CUDART_INF_F, l_run = 0.f;
+            float m_run = -CUDART_INF_F, l_run = 0.f;            // l_run: this thread's columns only
 
             for (int j = 0; j < n_my; ++j) {
                 const int i = two ? j : 2 * j + grp;             // local tile index
@@ -499,39 +591,46 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 ok = __all_sync(kFull, ok && mbar_wait(&bar_sfull[grp], sc & 1, ab));    // warp-uniform: guards .aligned ops
                 ++sc;
                 tc_fence_after_sync();
-                if (ok) {
-                    const bool tree = t == nt_unit - 1;
-                    const int nchunks = tree ? kTreeKeys / 32 : kTileKeys / 32;
-                    uint32_t sv[4][32];
-#pragma unroll
-                    for (int c = 0; c < 4; ++c)
-                        if (c < nchunks) tmem_ld32(tS + c * 32, sv[c]);
-                    tmem_wait_ld();
-                    // ---- masking ----
-                    if (tree) {
-#pragma unroll
-                        for (int c = 0; c < 2; ++c)
+                // This thread's chunks of 32 score columns: a prefix tile has four (two per thread), the tree tile
+                // two (one per thread).  Half h of a row works in columns 64 h .. 64 h + 63 of the buffer only: its
+                // scores sit there (the tree tile's second chunk is read from columns 32 .. 63 but belongs to
+                // half 1 alone) and its P goes to columns 64 h + 16 cc, so the halves never touch each other's
+                // columns and a thread overwrites only scores it has already taken into registers.
+                const bool tree = t == nt_unit - 1;
+                const int nch = tree ? 1 : 2;
+                const int c0 = tree ? half : 2 * half;
+                const int valid = tree ? kTreeKeys : min(kTileKeys, Pb - t * kTileKeys);
+                const bool partial = tree || valid < kTileKeys;
+                auto allowed_bits = [&](int c) -> uint32_t {        // keys of chunk c this row may attend to
+                    if (tree) return (uint32_t)(mask_bits >> (c * 32));
+                    const int lim = valid - c * 32;
+                    return lim >= 32 ? 0xffffffffu : (lim <= 0 ? 0u : ((1u << lim) - 1u));
+                };
+                float mx = -CUDART_INF_F;
+                if (ok && warp_live) {
+#pragma unroll 1
+                    for (int cc = 0; cc < nch; ++cc) {
+                        uint32_t sv[32];
+                        tmem_ld32(tS + (c0 + cc) * 32, sv);
+                        tmem_wait_ld();
+                        if (partial) {
+                            const uint32_t al = allowed_bits(c0 + cc);
 #pragma unroll
                             for (int e = 0; e < 32; ++e)
-                                if (!((mask_bits >> (c * 32 + e)) & 1ull)) sv[c][e] = 0xff800000u;     // -inf
-                    } else {
-                        const int valid = min(kTileKeys, Pb - t * kTileKeys);
-                        if (valid < kTileKeys) {
-#pragma unroll
-                            for (int c = 0; c < 4; ++c)
-#pragma unroll
-                                for (int e = 0; e < 32; ++e)
-                                    if (c * 32 + e >= valid) sv[c][e] = 0xff800000u;
+                                if (!((al >> e) & 1u)) sv[e] = 0xff800000u;     // -inf
                         }
+                        float mxa[4] = {-CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F};
+#pragma unroll
+                        for (int e = 0; e < 32; ++e) mxa[e & 3] = fmaxf(mxa[e & 3], __uint_as_float(sv[e]));
+                        mx = fmaxf(mx, fmaxf(fmaxf(mxa[0], mxa[1]), fmaxf(mxa[2], mxa[3])));
                     }
-                    // ---- running max (log2 units), lazy rescale decision ----
-                    float mxa[4] = {-CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F};   // short dependency chains
-#pragma unroll
-                    for (int c = 0; c < 4; ++c)
-                        if (c < nchunks)
-#pragma unroll
-                            for (int e = 0; e < 32; ++e) mxa[e & 3] = fmaxf(mxa[e & 3], __uint_as_float(sv[c][e]));
-                    const float mx = fmaxf(fmaxf(mxa[0], mxa[1]), fmaxf(mxa[2], mxa[3]));
+                }
+                // the two halves of a row exchange their maxima
+                s_mx[grp][half][row] = mx;
+                if (grp == 0) asm volatile("bar.sync 1, 256;" ::: "memory"); else asm volatile("bar.sync 2, 256;" ::: "memory");
+                if (ok && warp_live) {
+                    mx = fmaxf(mx, s_mx[grp][half ^ 1][row]);
+                    // ---- running max (log2 units), lazy rescale decision: the same in both halves of a row ----
                     const float m_tile = mx * P.scale_log2;
                     float factor = 1.f;
                     if (j == 0) {
@@ -541,34 +640,41 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                         m_run = m_tile;
                     }
                     const float m_use = m_run == -CUDART_INF_F ? 0.f : m_run;
-                    // ---- P = exp2(s * scale - m), row sum, bf16 pairs back to tensor memory (over S) ----
+                    // ---- P = exp2(s * scale - m), row sum, bf16 pairs back to tensor memory ----
                     float ls[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll 1
+                    for (int cc = 0; cc < nch; ++cc) {
+                        uint32_t sv[32];
+                        tmem_ld32(tS + (c0 + cc) * 32, sv);
+                        tmem_wait_ld();
+                        if (partial) {
+                            const uint32_t al = allowed_bits(c0 + cc);
 #pragma unroll
-                    for (int c = 0; c < 4; ++c) {
-                        if (c < nchunks) {
-                            uint32_t pk[16];
-#pragma unroll
-                            for (int e = 0; e < 16; ++e) {
-                                const float p0 = ex2(fmaf(__uint_as_float(sv[c][2 * e]), P.scale_log2, -m_use));
-                                const float p1 = ex2(fmaf(__uint_as_float(sv[c][2 * e + 1]), P.scale_log2, -m_use));
-                                ls[e & 3] += p0 + p1;
-                                const __nv_bfloat162 v = __floats2bfloat162_rn(p0, p1);
-                                pk[e] = *reinterpret_cast<const uint32_t*>(&v);
-                            }
-                            tmem_st16(tS + c * 16, pk);
+                            for (int e = 0; e < 32; ++e)
+                                if (!((al >> e) & 1u)) sv[e] = 0xff800000u;
                         }
+                        uint32_t pk[16];
+#pragma unroll
+                        for (int e = 0; e < 16; ++e) {
+                            const float p0 = ex2(fmaf(__uint_as_float(sv[2 * e]), P.scale_log2, -m_use));
+                            const float p1 = ex2(fmaf(__uint_as_float(sv[2 * e + 1]), P.scale_log2, -m_use));
+                            ls[e & 3] += p0 + p1;
+                            const __nv_bfloat162 v = __floats2bfloat162_rn(p0, p1);
+                            pk[e] = *reinterpret_cast<const uint32_t*>(&v);
+                        }
+                        tmem_st16(tS + half * 64 + cc * 16, pk);
                     }
                     l_run = l_run * factor + ((ls[0] + ls[1]) + (ls[2] + ls[3]));
-                    // ---- rescale the accumulator when some row of this warp moved its reference max ----
+                    // ---- rescale this thread's half of the accumulator when some row of the warp moved its max ----
                     if (j > 0 && __any_sync(kFull, factor != 1.f)) {
-#pragma unroll
-                        for (int c = 0; c < D / 32; ++c) {
+#pragma unroll 1
+                        for (int c = 0; c < DH / 32; ++c) {
                             uint32_t o[32];
-                            tmem_ld32(tO + c * 32, o);
+                            tmem_ld32(tO + half * DH + c * 32, o);
                             tmem_wait_ld();
 #pragma unroll
                             for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * factor);
-                            tmem_st32(tO + c * 32, o);
+                            tmem_st32(tO + half * DH + c * 32, o);
                         }
                     }
                     tmem_wait_st();
@@ -587,45 +693,49 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             const bool final_rows = cur.complete();
             const int slot = seg == 0 ? 0 : 1;                   // a CTA has at most a cut first and a cut last segment
             const int64_t rec = ((int64_t)blockIdx.x * 2 + slot) * kPairRows + prow;
-            float m_out = m_run, l_out = l_run, w0 = 1.f, w1 = 0.f;
+            // the row sum is the two halves' sums; with one live row block group 1 also hands its (m, l) to group 0
+            s_xl[grp][half][row] = l_run;
+            if (grp == 1 && half == 0) s_xm[row] = n_my > 0 ? m_run : -CUDART_INF_F;
+            asm volatile("bar.sync 3, 512;" ::: "memory");
+            float l_out = s_xl[grp][0][row] + s_xl[grp][1][row];
+            float m_out = m_run, w0 = 1.f, w1 = 0.f;
             bool writer = true, merge_any = false;
             if (!two) {
                 // group 0 merges group 1's accumulator, which sits in the same tensor-memory lanes
-                if (grp == 1) { s_xm[row] = n_my > 0 ? m_run : -CUDART_INF_F; s_xl[row] = l_run; }
-                asm volatile("bar.sync 1, 256;" ::: "memory");
                 writer = grp == 0;
                 if (writer) {
-                    const float m1 = s_xm[row], l1 = s_xl[row];
+                    const float m1 = s_xm[row], l1 = s_xl[1][0][row] + s_xl[1][1][row];
                     const bool merge = m1 != -CUDART_INF_F;
                     m_out = fmaxf(m_run, m1);
                     const float ms = m_out == -CUDART_INF_F ? 0.f : m_out;
                     w0 = ex2(m_run - ms);                        // exp2(-inf) = 0
                     w1 = ex2(m1 - ms);
-                    l_out = l_run * w0 + l1 * w1;
+                    l_out = l_out * w0 + l1 * w1;
                     merge_any = __any_sync(kFull, merge);        // rows that do not merge carry w1 = 0
                 }
             }
-            if (writer && ok) {
+            if (writer && ok && warp_live) {
                 const float m_safe = m_out == -CUDART_INF_F ? 0.f : m_out;
                 const float inv = final_rows ? 1.f / l_out : 1.f;
                 const int64_t out_row = ((int64_t)b * kMaxNodes + node) * a.Hq + hq;
-#pragma unroll
-                for (int c = 0; c < D / 32; ++c) {
+#pragma unroll 1
+                for (int c = 0; c < DH / 32; ++c) {
+                    const int col = half * DH + c * 32;          // first accumulator column of this chunk
                     uint32_t o[32];
-                    tmem_ld32(tO + c * 32, o);
+                    tmem_ld32(tO + col, o);
                     tmem_wait_ld();
                     float v[32];
 #pragma unroll
                     for (int e = 0; e < 32; ++e) v[e] = __uint_as_float(o[e]) * w0;
                     if (merge_any) {
-                        tmem_ld32(tO_other + c * 32, o);
+                        tmem_ld32(tO_other + col, o);
                         tmem_wait_ld();
 #pragma unroll
                         for (int e = 0; e < 32; ++e) v[e] = fmaf(__uint_as_float(o[e]), w1, v[e]);
                     }
                     if (row_live) {
                         if (final_rows) {
-                            __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(a.O) + out_row * D + c * 32;
+                            __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(a.O) + out_row * D + col;
 #pragma unroll
                             for (int q = 0; q < 4; ++q) {
                                 uint32_t w[4];
@@ -637,14 +747,14 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                                 *reinterpret_cast<uint4*>(dst + q * 8) = make_uint4(w[0], w[1], w[2], w[3]);
                             }
                         } else {
-                            float* dst = P.part_o + rec * D + c * 32;
+                            float* dst = P.part_o + rec * D + col;
 #pragma unroll
                             for (int q = 0; q < 8; ++q)
                                 *reinterpret_cast<float4*>(dst + q * 4) = make_float4(v[q * 4], v[q * 4 + 1], v[q * 4 + 2], v[q * 4 + 3]);
                         }
                     }
                 }
-                if (row_live) {
+                if (row_live && half == 0) {
                     const float m_nat = m_safe * 0.6931471805599453f;
                     if (final_rows) {
                         if (a.lse != nullptr) a.lse[((int64_t)b * a.Hq + hq) * kMaxNodes + node] = m_nat + logf(l_out);
@@ -653,7 +763,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                     }
                 }
             }
-            if (!two) asm volatile("bar.sync 2, 256;" ::: "memory");   // group 1's accumulator and (m, l) have been read
+            asm volatile("bar.sync 4, 512;" ::: "memory");       // the exchanged (m, l) and group 1's accumulator have been read
             tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) mbar_arrive(&bar_ofree[grp]);

@@ -175,14 +175,36 @@ class CudaRun:
 
 
 # ---- comparisons -------------------------------------------------------------------------------
-def check_margins(cfg, traces, trees, accepts=None):
-    """The seeds must not put any float-keyed decision within rounding distance of a tie."""
+def _same_bits_siblings(inp, b, pool, p, q):
+    """Pool entries p and q are children of one parent whose logits are bit-identical: both sides then hold
+    exactly equal scores for them (the same function of the same inputs) and order them by index."""
+    if pool.parent[p] != pool.parent[q]:
+        return False
+    par = int(pool.parent[p])
+    row = 0 if par < 0 else int(pool.draft_row[par])
+    z = inp["draft"][b][row]
+    return z[pool.tok[p]].tobytes() == z[pool.tok[q]].tobytes()
+
+
+def check_margins(cfg, traces, trees, accepts=None, inp=None, pools=None):
+    """The seeds must not put any float-keyed decision within rounding distance of a tie.  With `inp` and
+    `pools`, a gap of exactly zero between siblings whose logits are bit-identical is not a near-tie (low
+    precision logits collide often): it is decided by index on both sides."""
+    def gap_ok(b, gap, p, q):
+        if gap > TAU_SCORE:
+            return True
+        return gap == 0.0 and inp is not None and _same_bits_siblings(inp, b, pools[b], int(p), int(q))
+
     for b in range(cfg.B):
         for tr in traces[b]:
-            assert tr["margin"] > TAU_SCORE, ("frontier near-tie", b, tr["t"], tr["margin"])
+            hp, hs = tr["head_pool_idx"], tr["head_score"]
+            for a in range(len(hp) - 1):
+                gap = float(hs[a] - hs[a + 1])
+                assert not np.isfinite(gap) or gap_ok(b, gap, hp[a], hp[a + 1]), ("frontier near-tie", b, tr["t"], gap)
             if "gate_margin" in tr:
                 assert tr["gate_margin"] > TAU_SCORE, ("gate near-tie", b, tr["t"], tr["gate_margin"])
-        assert trees[b]["margin"] > TAU_SCORE, ("rerank near-tie", b, trees[b]["margin"])
+        if trees[b]["cut_pair"] is not None:
+            assert gap_ok(b, trees[b]["margin"], *trees[b]["cut_pair"]), ("rerank near-tie", b, trees[b]["margin"])
         if accepts is not None and "accept_margin" in accepts[b]:
             assert accepts[b]["accept_margin"] > TAU_PROB and accepts[b]["sample_margin"] > TAU_PROB, (b, accepts[b])
 

@@ -1,9 +1,9 @@
 """Parity at the full sizes of the batched configurations, in the launch configuration the benchmark
 times (same `SpecStep`, same workspaces, same grid plans).  The expansion, the tree and the
-acceptance are compared in full (the oracle handles them in seconds even at V = 128256); the
-attention output is compared on sampled (sequence, query head) pairs that the oracle computes one
-by one, chosen to cover the first and last sequence, the longest and the shortest prefix and
-both ends of the head range."""
+acceptance are compared in full (the oracle handles them in seconds even at V = 128256), and so is
+the attention output: every (sequence, query head) pair, one sequence at a time so that only one
+sequence's cache is widened to float64 at once (the failure modes of the attention kernel depend
+on where the persistent grid cuts a unit, which differs from the reduced cases)."""
 import numpy as np
 import pytest
 
@@ -19,16 +19,6 @@ def ctx():
     c = rb.Context(0)
     yield c
     c.close()
-
-
-def sampled_pairs(cfg, prefix_len, n_random=6):
-    B, Hq = cfg.B, cfg.Hq
-    longest, shortest = int(np.argmax(prefix_len)), int(np.argmin(prefix_len))
-    pairs = {(0, 0), (B - 1, Hq - 1), (longest, Hq // 2), (shortest, 1 % Hq), (longest, Hq - 1), (shortest, 0)}
-    g = np.random.Generator(np.random.Philox(1234 + cfg.cid))
-    while len(pairs) < 6 + n_random:
-        pairs.add((int(g.integers(0, B)), int(g.integers(0, Hq))))
-    return sorted(pairs)
 
 
 @pytest.mark.parametrize("cid", [3, 4, 5])
@@ -48,9 +38,13 @@ def test_full_size_step_matches_oracle(ctx, cid):
 
     g.upload_attention()
     O_gpu, lse_gpu = g.attention()
-    pairs = sampled_pairs(cfg, inp["prefix_len"])
-    O_ref, lse_ref = H.oracle_attention(cfg, inp, trees, pairs=pairs)
-    H.compare_attention(cfg, O_gpu, lse_gpu, O_ref, lse_ref, trees, pairs=pairs)
+    compared = 0
+    for b in range(cfg.B):
+        pairs = [(b, h) for h in range(cfg.Hq)]
+        O_ref, lse_ref = H.oracle_attention(cfg, inp, trees, pairs=pairs)
+        H.compare_attention(cfg, O_gpu, lse_gpu, O_ref, lse_ref, trees, pairs=pairs)
+        compared += len(pairs)
+    assert compared == cfg.B * cfg.Hq
     # every live output row is finite and rows past a tree's end were left alone (the buffer starts at zero)
     for b in range(cfg.B):
         n = trees[b]["n_nodes"]

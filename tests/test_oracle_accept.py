@@ -229,3 +229,106 @@ def test_accept_length_distribution_single_child_closed_form():
     p = scipy.special.softmax(tl[0].astype(np.float64)); q = scipy.special.softmax(dl[0].astype(np.float64))
     a = min(1.0, p[x] / q[x])
     assert np.allclose(dist, [1 - a, a], atol=1e-14) and abs(pacc[1] - a) < 1e-14
+
+
+# ---- hand-computed edge branches of the accept rule (4-token vocabulary) ---------------------------
+# Each case is small enough to follow on paper; the expected values in the comments are worked out from
+# Eq. 1-2 and the stated readings (q(x) = 0: accepted iff p(x) > 0; a draft row with no mass left stops
+# the sibling loop; the draw is the inverse CDF in token order), not from running the oracle.
+def _hand_tree(toks, parents):
+    n = len(toks)
+    tok = np.full(64, -1, np.int32); tok[:n] = toks
+    par = np.full(64, -1, np.int32); par[:n] = parents
+    drow = np.full(64, -1, np.int32)
+    for i in range(n):
+        if any(p == i for p in parents[1:]):
+            drow[i] = 0                                   # every internal node reads draft row 0 in these cases
+    leaves = [i for i in range(n) if i not in parents[1:]]
+    retrieve = np.full((max(len(leaves), 1), 3), -1, np.int32)
+    for r, l in enumerate(leaves):
+        path = [l]
+        while par[path[-1]] >= 0:
+            path.append(int(par[path[-1]]))
+        retrieve[r, :len(path)] = path[::-1]
+    return {"n_nodes": n, "tok": tok, "parent": par, "draft_row": drow, "retrieve": retrieve, "n_leaves": len(leaves)}
+
+
+NEG = -np.inf
+
+
+def _logs(p):
+    with np.errstate(divide="ignore"):
+        return np.log(np.asarray(p, np.float64)).astype(np.float32)
+
+
+def test_accept_when_draft_probability_is_zero_and_target_positive():
+    # q(x) = 0, p(x) = 1/4 > 0: the ratio is +inf, the child is accepted whatever u is.
+    tree = _hand_tree([9, 2], [-1, 0])
+    target = np.stack([_logs([.25, .25, .25, .25]), _logs([.1, .2, .3, .4])])
+    draft = _logs([1 / 3, 1 / 3, 0, 1 / 3])[None]
+    ua = np.full(64, 0.999, np.float32)
+    r = A.verify_stochastic(target, draft, tree, ua, 0.55, 1.0, 2)
+    assert r["accept_len"] == 1 and r["path_nodes"][:2].tolist() == [0, 1]
+    # leaf reached: bonus token from softmax(target[1]) = (.1, .2, .3, .4); CDF .1 .3 .6 1: first step above .55 is token 2
+    assert r["next_token"] == 2
+
+
+def test_reject_when_both_probabilities_are_zero():
+    # q(x) = 0 and p(x) = 0: rejected.  p = (1/3, 1/3, 0, 1/3), q = (1/4, 1/4, 0, 1/2):
+    # residual max(0, p - q) = (1/12, 1/12, 0, 0) -> (1/2, 1/2, 0, 0); u = .7 -> token 1.
+    tree = _hand_tree([9, 2], [-1, 0])
+    target = np.stack([_logs([1 / 3, 1 / 3, 0, 1 / 3]), _logs([.25, .25, .25, .25])])
+    draft = _logs([.25, .25, 0, .5])[None]
+    ua = np.zeros(64, np.float32)                         # u = 0 would accept anything with a positive ratio
+    r = A.verify_stochastic(target, draft, tree, ua, 0.7, 1.0, 2)
+    assert r["accept_len"] == 0 and r["next_token"] == 1
+    r = A.verify_stochastic(target, draft, tree, ua, 0.3, 1.0, 2)
+    assert r["next_token"] == 0
+
+
+def test_draft_row_with_all_mass_on_the_rejected_token_stops_the_sibling_loop():
+    # q = (0, 1, 0, 0); children x1 = token 1, x2 = token 0.  p = (.4, .1, .3, .2): ratio for x1 = .1 < u = .5 -> reject.
+    # Residual max(0, p - q) = (.4, 0, .3, .2) / .9.  Removing token 1 leaves q with no mass: nothing is left to
+    # propose, so x2 is NOT tried (it would be accepted, its q being 0 and its p positive) and the next token is
+    # drawn from the residual: CDF 4/9, 4/9, 7/9, 1: u = .5 -> token 2, u = .4 -> token 0.
+    tree = _hand_tree([9, 1, 0], [-1, 0, 0])
+    target = np.stack([_logs([.4, .1, .3, .2]), _logs([.25] * 4), _logs([.25] * 4)])
+    draft = _logs([0, 1, 0, 0])[None]
+    ua = np.full(64, 0.5, np.float32)
+    r = A.verify_stochastic(target, draft, tree, ua, 0.5, 1.0, 2)
+    assert r["accept_len"] == 0 and r["next_token"] == 2
+    assert A.verify_stochastic(target, draft, tree, ua, 0.4, 1.0, 2)["next_token"] == 0
+    # Eq. 13 on the same tree: P_acc(x1) = .1, P_acc(x2) = 0 (never tried), P_stop(root) = .9
+    dist, pacc = A.accept_length_distribution(target, draft, dict(tree, depth=np.array([0, 1, 1] + [0] * 61, np.int32)), 1.0, 2)
+    assert abs(pacc[1] - 0.1) < 1e-7 and pacc[2] == 0.0           # the logits are float32: ln(.1) is rounded
+    assert abs(dist[0] - 0.9) < 1e-7 and abs(dist[1] - 0.1) < 1e-7
+
+
+def test_second_sibling_is_tried_on_the_residual_and_the_renormalised_draft():
+    # The ordinary multi-draft step, by hand: p = (.4, .1, .3, .2), q = (.1, .6, .2, .1); x1 = token 1, x2 = token 2.
+    # x1: ratio 1/6 < u = .5 -> reject.  p' = max(0, p - q) = (.3, 0, .1, .1) / .5 = (.6, 0, .2, .2);
+    # q' = (.1, 0, .2, .1) / .4 = (.25, 0, .5, .25).  x2: ratio .2 / .5 = .4 < .5 -> reject.
+    # p'' = max(0, p' - q') = (.35, 0, 0, 0) / .35 = (1, 0, 0, 0): next token 0 for every u.
+    tree = _hand_tree([9, 1, 2], [-1, 0, 0])
+    target = np.stack([_logs([.4, .1, .3, .2]), _logs([.25] * 4), _logs([.25] * 4)])
+    draft = _logs([.1, .6, .2, .1])[None]
+    r = A.verify_stochastic(target, draft, tree, np.full(64, 0.5, np.float32), 0.9, 1.0, 2)
+    assert r["accept_len"] == 0 and r["next_token"] == 0
+    assert abs(r["accept_margin"] - 0.1) < 1e-6                      # |u - ratio| of the closer test (x2)
+    # with u = .3 the second sibling (ratio .4) is accepted; it is a leaf: bonus token from its uniform target row
+    ua = np.full(64, 0.5, np.float32); ua[2] = 0.3
+    r = A.verify_stochastic(target, draft, tree, ua, 0.6, 1.0, 2)
+    assert r["accept_len"] == 1 and r["path_nodes"][:2].tolist() == [0, 2] and r["next_token"] == 2
+
+
+def test_inverse_cdf_upper_end_returns_the_last_token_with_mass():
+    # u = 1 is outside [0, 1) but defined: no step of the CDF lies above u * total, and the draw falls back to the
+    # last token with positive weight (token 2 here, not the zero-weight token 3).
+    tree = _hand_tree([9], [-1])
+    target = _logs([.2, .3, .5, 0])[None]
+    draft = _logs([.25] * 4)[None]
+    r = A.verify_stochastic(target, draft, tree, np.zeros(64, np.float32), 1.0, 1.0, 2)
+    assert r["accept_len"] == 0 and r["next_token"] == 2
+    # just below the top step the ordinary rule applies: largest float32 below 1
+    assert A.verify_stochastic(target, draft, tree, np.zeros(64, np.float32), np.float32(1) - np.float32(2 ** -24), 1.0, 2)["next_token"] == 2
+    assert A.verify_stochastic(target, draft, tree, np.zeros(64, np.float32), 0.4999, 1.0, 2)["next_token"] == 1
