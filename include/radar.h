@@ -54,7 +54,8 @@ enum { RADAR_GREEDY = 0, RADAR_STOCHASTIC = 1 };
 typedef struct radar_ctx radar_ctx;
 
 /* Context: remembers the device, its SM count and owns the 4-byte device status word
- * (the only allocation the library ever makes).  `out` is a host pointer. */
+ * (the only allocation the library ever makes).  `out` is a host pointer.  A context belongs to one
+ * device and is used by one host thread at a time; make one per device. */
 int radar_create(radar_ctx** out, int device);
 int radar_destroy(radar_ctx* ctx);
 const char* radar_status_string(int status);
@@ -195,9 +196,12 @@ int radar_rerank_build_tree(radar_ctx* ctx, const radar_tree_args* args, void* s
  * of token rows allocated in Kc / Vc and bounds every read of them.  A sequence whose device-side
  * prefix_len is negative or larger than max_prefix_len, or whose kv_start + prefix_len exceeds
  * cache_rows, records RADAR_ERR_INVALID_ARG on the device status word and is skipped.
- * bf16 with Hq / Hkv a power of two (<= 128) and 16-byte aligned tensors runs on the tensor cores
- * (TMA-staged K/V tiles, tcgen05 MMA for QK^T and PV); every other case, and all of fp32, runs on
- * an fp32 FMA kernel.
+ * Q, Kc, Vc, Kt, Vt and O must be 16-byte aligned (both kernels move them in 16-byte pieces); a misaligned
+ * tensor is refused on the host with RADAR_ERR_INVALID_ARG.
+ * bf16 with Hq / Hkv a power of two (<= 128) runs on the tensor cores (TMA-staged K/V tiles, tcgen05 MMA for
+ * QK^T and PV); every other case, and all of fp32, runs on an fp32 FMA kernel.  radar_tree_attention_path()
+ * tells which of the two a given argument struct will take, so that a caller (or a benchmark) is never
+ * switched to the other kernel unawares.
  * Paged prefix cache (block_table != NULL): prefix token j of sequence b is cache row
  *   block_table[b * max_pages + j / page_size] * page_size + j % page_size
  * and kv_start is not read (it may be NULL).  page_size is 16, 32, 64 or a multiple of 128; a
@@ -229,8 +233,13 @@ typedef struct {
     int max_pages;                      /* entries per sequence in block_table                           */
 } radar_attn_args;
 
+enum { RADAR_ATTN_PATH_FMA = 0, RADAR_ATTN_PATH_TENSOR_CORE = 1 };
+
 size_t radar_attn_workspace_bytes(const radar_ctx* ctx, int B, int Hq, int Hkv, int d, int dtype, int max_prefix_len);
 int radar_tree_attention(radar_ctx* ctx, const radar_attn_args* args, void* stream);
+/* Which kernel radar_tree_attention runs for these arguments (host pointer): RADAR_ATTN_PATH_TENSOR_CORE or
+ * RADAR_ATTN_PATH_FMA; negative status if args is NULL.  Reads only the host fields of the struct. */
+int radar_tree_attention_path(const radar_attn_args* args);
 
 /* ------------------------------------------------------------------------------------------
  * radar_verify_accept - acceptance of the verified tree.
@@ -310,16 +319,20 @@ int radar_accept_length_distribution(radar_ctx* ctx, const radar_acclen_args* ar
  * all free device memory to its own cache pool at start-up, or a decode loop that must not take
  * the device-wide synchronisation of cudaMalloc / cudaFree - and that have no spare buffer to pass
  * as `workspace`.  The scratch is a fixed array of radar_noalloc_scratch_bytes() = 1 MiB inside
- * the library image, resident on every GPU that has the library loaded until the process exits.
+ * the library image.  The driver materialises it (and the kernels' code) on a GPU when the image is
+ * first used there; radar_create does that for its device, so create the context before the host
+ * freezes device memory - the array then stays until the process exits.
  * `workspace` / `workspace_bytes` of the argument struct are ignored; `mode` must be RADAR_GREEDY.
  *   - Sizes whose chunk records (about 16 bytes x B x 64 x chunks-per-row) exceed the array, and
  *     stochastic mode, return RADAR_ERR_UNSUPPORTED and launch nothing.
- *   - The call makes no cudaMalloc / cudaFree and calls no allocating routine.
+ *   - The call makes no cudaMalloc / cudaFree and calls no allocating routine; after radar_create on the
+ *     same device it leaves the amount of free device memory unchanged.
  *   - Every call on a device uses the same array, which still holds the previous call's records;
  *     nothing needs to be cleared because each record is written before it is read within a call.
  *     Calls that may overlap on the GPU (two streams, concurrent graph replays) race: serialise them.
- *   - The first call on each device resolves the array's device address (ctx's device must be the
- *     current device, otherwise RADAR_ERR_INVALID_ARG); make that first call outside stream capture. */
+ *   - ctx's device must be the current device (otherwise RADAR_ERR_INVALID_ARG).  radar_create has
+ *     resolved the array's device address; should a call find none cached it resolves it itself, so make
+ *     the first call outside stream capture. */
 size_t radar_noalloc_scratch_bytes(void);
 int radar_verify_accept_greedy_noalloc(radar_ctx* ctx, const radar_accept_args* args, void* stream);
 

@@ -19,6 +19,7 @@ RADAR_F32, RADAR_BF16 = 0, 1
 RADAR_GREEDY, RADAR_STOCHASTIC = 0, 1
 RADAR_POLICY_LSTM_SCORES, RADAR_POLICY_MLP_SCORES, RADAR_POLICY_LSTM_HIDDEN = 0, 1, 2
 RADAR_OK = 0
+RADAR_ATTN_PATH_FMA, RADAR_ATTN_PATH_TENSOR_CORE = 0, 1
 
 _c_int, _c_i64, _c_f, _vp, _sz = ctypes.c_int, ctypes.c_int64, ctypes.c_float, ctypes.c_void_p, ctypes.c_size_t
 
@@ -283,9 +284,8 @@ def radar_rerank_build_tree(ctx: Context, *, B, N, t_max, pool_capacity, pool_to
     _check("radar_rerank_build_tree", lib().radar_rerank_build_tree(ctx.handle, ctypes.byref(a), _stream(stream)))
 
 
-def radar_tree_attention(ctx: Context, *, B, Hq, Hkv, d, Q, Kc, Vc, kv_start, prefix_len, max_prefix_len, Kt, Vt,
-                         mask, n_nodes, O, workspace, lse=None, scale=0.0, stream=None, block_table=None, page_size=0):
-    """`block_table` [B, max_pages] int32 with `page_size` selects the paged prefix cache (kv_start may then be None)."""
+def _attn_args(*, B, Hq, Hkv, d, Q, Kc, Vc, kv_start, prefix_len, max_prefix_len, Kt, Vt, mask, n_nodes, O, workspace,
+               lse=None, scale=0.0, block_table=None, page_size=0):
     a = AttnArgs()
     a.B, a.Hq, a.Hkv, a.d, a.dtype = B, Hq, Hkv, d, dtype_code(Q)
     for t in (Kc, Vc, Kt, Vt, O):
@@ -300,7 +300,23 @@ def radar_tree_attention(ctx: Context, *, B, Hq, Hkv, d, Q, Kc, Vc, kv_start, pr
     a.workspace, a.workspace_bytes = _ptr(workspace), workspace.numel() * workspace.element_size()
     if block_table is not None:
         a.block_table, a.page_size, a.max_pages = _ptr(block_table, torch.int32), page_size, block_table.shape[-1]
+    return a
+
+
+def radar_tree_attention(ctx: Context, *, stream=None, **kw):
+    """Arguments as in `_attn_args` (the fields of radar_attn_args as tensors).  `block_table` [B, max_pages] int32
+    with `page_size` selects the paged prefix cache (kv_start may then be None)."""
+    a = _attn_args(**kw)
     _check("radar_tree_attention", lib().radar_tree_attention(ctx.handle, ctypes.byref(a), _stream(stream)))
+
+
+def radar_tree_attention_path(**kw) -> int:
+    """RADAR_ATTN_PATH_TENSOR_CORE or RADAR_ATTN_PATH_FMA for the same keyword arguments as radar_tree_attention."""
+    L = lib()
+    L.radar_tree_attention_path.restype = _c_int
+    L.radar_tree_attention_path.argtypes = [ctypes.POINTER(AttnArgs)]
+    a = _attn_args(**kw)
+    return int(L.radar_tree_attention_path(ctypes.byref(a)))
 
 
 def radar_verify_accept(ctx: Context, *, B, V, t_max, N, mode, target_logits, tree_tok, tree_parent, tree_draft_row,

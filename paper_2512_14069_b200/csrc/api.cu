@@ -24,10 +24,17 @@ extern "C" int radar_create(radar_ctx** out, int device) {
     c->ev_kernel = nullptr;
     c->ev_cap = c->ev_used = 0;
     for (int i = 0; i < RADAR_K_COUNT; ++i) { c->launches[i] = 0; c->prof_ms[i] = 0.0; c->prof_n[i] = 0; }
+    for (int i = 0; i < RADAR_SMEM_COUNT; ++i) c->smem_opt_in[i] = 0;
     if (cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, device) != cudaSuccess ||
         cudaMalloc(&c->d_status, 2 * sizeof(int)) != cudaSuccess ||
         cudaMemset(c->d_status, 0, 2 * sizeof(int)) != cudaSuccess) {
         if (c->d_status) cudaFree(c->d_status);
+        delete c;
+        return RADAR_ERR_CUDA;
+    }
+    // the workspace-free acceptance path must find everything in place later, when its host may not allocate
+    if (radar::noalloc_prepare_device(device) != RADAR_OK) {
+        cudaFree(c->d_status);
         delete c;
         return RADAR_ERR_CUDA;
     }

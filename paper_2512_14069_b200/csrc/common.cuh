@@ -25,9 +25,21 @@ enum radar_kernel_id {
     RADAR_K_COUNT
 };
 
+// kernels that opt in to more than 48 KB of dynamic shared memory: one slot per instantiation
+enum radar_smem_slot {
+    RADAR_SMEM_SELECT_GATE = 0,
+    RADAR_SMEM_TREE_BUILD,
+    RADAR_SMEM_ATTN_FMA,        // + 2 * (bf16) + (d == 128)
+    RADAR_SMEM_ATTN_TC = RADAR_SMEM_ATTN_FMA + 4,   // + 4 * (d == 128) + 2 * two + paged
+    RADAR_SMEM_COUNT = RADAR_SMEM_ATTN_TC + 8
+};
+
 struct radar_ctx {
     int device;
     int sm_count;
+    // largest dynamic shared-memory size opted in to so far, per kernel, ON THIS CONTEXT'S DEVICE (the attribute
+    // is per device: a second device in the same process needs its own opt-in)
+    size_t smem_opt_in[RADAR_SMEM_COUNT];
     int* d_status;          // sticky device status word
     // launch accounting (host side)
     long long launches[RADAR_K_COUNT];
@@ -92,6 +104,17 @@ __device__ __forceinline__ void chain_sync() { asm volatile("griddepcontrol.wait
 
 // A failing runtime call becomes RADAR_ERR_CUDA; with RADAR_DEBUG set in the environment the call and the
 // runtime's message are also written to stderr.
+// Raises a kernel's dynamic shared-memory limit on the context's device when `bytes` exceeds what has been
+// set there before (48 KB need no opt-in).  Not a stream operation.
+template <typename K>
+inline cudaError_t radar_opt_in_smem(radar_ctx* ctx, int slot, K kernel, size_t bytes) {
+    const size_t have = ctx->smem_opt_in[slot] > 48 * 1024 ? ctx->smem_opt_in[slot] : 48 * 1024;
+    if (bytes <= have) return cudaSuccess;
+    const cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+    if (e == cudaSuccess) ctx->smem_opt_in[slot] = bytes;
+    return e;
+}
+
 #define RADAR_CUDA_CHECK(expr)                                                                     \
     do {                                                                                           \
         cudaError_t _e = (expr);                                                                   \
@@ -185,6 +208,12 @@ int vocab_pass_plan_chunks(int sm_count, int rows, int V, int* chunk_out);   // 
 size_t vocab_pass_partial_bytes(int rows, int n_chunks, int k);
 void vocab_pass_carve(void* ws, int rows, int n_chunks, int k, VocabPassParams* p);
 cudaError_t vocab_pass_launch(radar_ctx* ctx, int kernel_id, const VocabPassParams& p, cudaStream_t stream);
+cudaError_t vocab_pass_preload_argbest();
+
+// --- workspace-free greedy acceptance (verify_accept.cu) --------------------------------------
+// Resolves the device address of the library's scratch array on the current device and loads the two kernels of
+// that path, so that nothing is left for the driver to allocate at the first call.  Called by radar_create.
+int noalloc_prepare_device(int device);
 
 // --- tensor-core tree attention (tree_attention_tc.cu) --------------------------------------
 bool tree_attn_tc_supported(const radar_attn_args* a);

@@ -487,16 +487,14 @@ extern "C" int radar_expand_step(radar_ctx* ctx, const radar_expand_args* a, voi
     }
 
     RADAR_CUDA_CHECK(vocab_pass_launch(ctx, RADAR_K_VOCAB_EXPAND, vp, stream));
+    // The chunk records are staged in shared memory only if they fit next to the survivor lists and the gate
+    // weights inside the 227 KB a block may have; otherwise the merge reads them from global memory.
     const size_t stage_bytes = (size_t)a->F * vp.n_chunks * a->k * 8;
-    sp.staged = stage_bytes <= kStageLimit ? 1 : 0;
-    const size_t smem = 2 * up16(sp.staged ? stage_bytes / 2 : 0) + (size_t)kMergeWarps * kSurvCap * 8 +
-                        sizeof(float) * ((size_t)4 * kHidden * a->k + (size_t)kHidden * (kHidden + a->k));
-    static size_t attr_smem = 0;                    // raised at most a few times per process
-    if (smem > attr_smem) {
-        RADAR_CUDA_CHECK(cudaFuncSetAttribute(expand_select_gate_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                              (int)smem));
-        attr_smem = smem;
-    }
+    const size_t fixed_smem = (size_t)kMergeWarps * kSurvCap * 8 +
+                              sizeof(float) * ((size_t)4 * kHidden * a->k + (size_t)kHidden * (kHidden + a->k));
+    sp.staged = stage_bytes <= kStageLimit && 2 * up16(stage_bytes / 2) + fixed_smem <= 227 * 1024 ? 1 : 0;
+    const size_t smem = 2 * up16(sp.staged ? stage_bytes / 2 : 0) + fixed_smem;
+    RADAR_CUDA_CHECK(radar_opt_in_smem(ctx, RADAR_SMEM_SELECT_GATE, expand_select_gate_kernel, smem));
     {
         radar_launch_scope scope(ctx, RADAR_K_SELECT_GATE, stream);
         RADAR_CUDA_CHECK(launch_chained(expand_select_gate_kernel, dim3(a->B), dim3(kSelThreads), smem, stream, sp));

@@ -67,7 +67,11 @@ __global__ void __launch_bounds__(kThreads) tree_attn_fp32_kernel(const AttnPara
 
     const int M = min(max(a.n_nodes[b], 0), kMaxNodes);
     const int Pb = a.prefix_len[b];
-    if (Pb < 0 || Pb > a.max_prefix_len) {
+    const bool paged = a.block_table != nullptr;
+    const int64_t kv0 = paged ? 0 : a.kv_start[b];
+    // the same bounds as the tensor-core kernel: a sequence whose prefix does not lie inside the cache is
+    // reported and skipped before anything of the cache is read
+    if (Pb < 0 || Pb > a.max_prefix_len || kv0 < 0 || kv0 + Pb > a.cache_rows) {
         if (tid == 0) set_status(P.status, RADAR_ERR_INVALID_ARG);
         return;
     }
@@ -84,8 +88,6 @@ __global__ void __launch_bounds__(kThreads) tree_attn_fp32_kernel(const AttnPara
     const T* Vc = reinterpret_cast<const T*>(a.Vc);
     const T* Kt = reinterpret_cast<const T*>(a.Kt);
     const T* Vt = reinterpret_cast<const T*>(a.Vt);
-    const bool paged = a.block_table != nullptr;
-    const int64_t kv0 = paged ? 0 : a.kv_start[b];
     const int64_t n_cache_pages = paged ? P.a.cache_rows / a.page_size : 0;
 
     // ---- stage the block's query rows (pre-scaled) ----
@@ -241,7 +243,8 @@ __global__ void __launch_bounds__(128) tree_attn_combine_kernel(const AttnParams
     if (b >= a.B) return;
     const int M = min(max(a.n_nodes[b], 0), kMaxNodes);
     const int Pb = a.prefix_len[b];
-    if (node >= M || Pb < 0 || Pb > a.max_prefix_len) return;
+    const int64_t kv0 = a.block_table != nullptr ? 0 : a.kv_start[b];
+    if (node >= M || Pb < 0 || Pb > a.max_prefix_len || kv0 < 0 || kv0 + Pb > a.cache_rows) return;   // skipped by the main kernel
     const int n_valid = (Pb + M + P.split_len - 1) / P.split_len;
     const int64_t rec0 = (((int64_t)b * a.Hq + hq) * kMaxNodes + node) * P.n_splits;
     float mx = -CUDART_INF_F;
@@ -287,12 +290,7 @@ int launch(radar_ctx* ctx, const AttnParams& P, cudaStream_t stream) {
     const radar_attn_args& a = P.a;
     const int rblocks = (kMaxNodes * P.G + kRowsPerBlock - 1) / kRowsPerBlock;
     const size_t smem = sizeof(float) * (kRowsPerBlock * D + kTile * (D + 4) + kTile * D);
-    static bool attr_done = false;                  // once per process: not a stream operation
-    if (smem > 48 * 1024 && !attr_done) {
-        RADAR_CUDA_CHECK(cudaFuncSetAttribute(tree_attn_fp32_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                              (int)smem));
-        attr_done = true;
-    }
+    RADAR_CUDA_CHECK(radar_opt_in_smem(ctx, RADAR_SMEM_ATTN_FMA + 2 * (sizeof(T) == 2) + (D == 128), tree_attn_fp32_kernel<T, D>, smem));
     dim3 grid((unsigned)(rblocks * P.n_splits), (unsigned)a.Hkv, (unsigned)a.B);
     {
         radar_launch_scope scope(ctx, RADAR_K_ATTN, stream);
@@ -325,6 +323,11 @@ extern "C" size_t radar_attn_workspace_bytes(const radar_ctx* ctx, int B, int Hq
     return need;
 }
 
+extern "C" int radar_tree_attention_path(const radar_attn_args* a) {
+    if (!a) return RADAR_ERR_INVALID_ARG;
+    return tree_attn_tc_supported(a) ? RADAR_ATTN_PATH_TENSOR_CORE : RADAR_ATTN_PATH_FMA;
+}
+
 extern "C" int radar_tree_attention(radar_ctx* ctx, const radar_attn_args* a, void* stream_) {
     if (!ctx || !a) return RADAR_ERR_INVALID_ARG;
     cudaStream_t stream = reinterpret_cast<cudaStream_t>(stream_);
@@ -342,6 +345,10 @@ extern "C" int radar_tree_attention(radar_ctx* ctx, const radar_attn_args* a, vo
         return RADAR_ERR_INVALID_ARG;
     if (a->max_prefix_len > 0 && (!a->Kc || !a->Vc)) return RADAR_ERR_INVALID_ARG;
     if ((reinterpret_cast<uintptr_t>(a->workspace) & 255) != 0) return RADAR_ERR_WORKSPACE;
+    // both kernels move Q, K, V and O in 16-byte pieces
+    if (((reinterpret_cast<uintptr_t>(a->Q) | reinterpret_cast<uintptr_t>(a->Kc) | reinterpret_cast<uintptr_t>(a->Vc) |
+          reinterpret_cast<uintptr_t>(a->Kt) | reinterpret_cast<uintptr_t>(a->Vt) | reinterpret_cast<uintptr_t>(a->O)) & 15) != 0)
+        return RADAR_ERR_INVALID_ARG;
     if (a->max_prefix_len > 0 && a->cache_rows <= 0) return RADAR_ERR_INVALID_ARG;
     if (tree_attn_tc_supported(a)) return tree_attn_tc_launch(ctx, a, stream);
 

@@ -1072,12 +1072,8 @@ static int launch_tc(radar_ctx* ctx, TcParams& P, cudaStream_t stream) {
         !make_map(&tmKc, have_prefix ? a.Kc : a.Kt, D, a.Hkv, have_prefix ? a.cache_rows : tree_rows, 1, cache_box) ||
         !make_map(&tmVc, have_prefix ? a.Vc : a.Vt, D, a.Hkv, have_prefix ? a.cache_rows : tree_rows, 1, cache_box))
         return RADAR_ERR_CUDA;
-    static bool attr_done = false;                  // once per process and instantiation: not a stream operation
-    if (!attr_done) {
-        RADAR_CUDA_CHECK(cudaFuncSetAttribute(tree_attn_tc_kernel<D, TWO, PAGED>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                              Smem<D, TWO>::kDynamic));
-        attr_done = true;
-    }
+    RADAR_CUDA_CHECK(radar_opt_in_smem(ctx, RADAR_SMEM_ATTN_TC + 4 * (D == 128) + 2 * TWO + PAGED, tree_attn_tc_kernel<D, TWO, PAGED>,
+                                       (size_t)Smem<D, TWO>::kDynamic));
     {
         radar_launch_scope scope(ctx, RADAR_K_ATTN, stream);
         RADAR_CUDA_CHECK(launch_chained(tree_attn_tc_kernel<D, TWO, PAGED>, dim3((unsigned)(P.n_cls * P.ncc)), dim3(kTcThreads),

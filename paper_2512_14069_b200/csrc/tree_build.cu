@@ -243,12 +243,7 @@ extern "C" int radar_rerank_build_tree(radar_ctx* ctx, const radar_tree_args* a,
     p.n2 = 2;
     while (p.n2 < a->pool_capacity) p.n2 <<= 1;
     const size_t smem = (size_t)(p.n2 + 32) * 8 + (size_t)a->pool_capacity * 6;
-    static size_t attr_smem = 48 * 1024;            // raised at most a few times per process
-    if (smem > attr_smem) {
-        RADAR_CUDA_CHECK(cudaFuncSetAttribute(rerank_build_tree_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                              (int)smem));
-        attr_smem = smem;
-    }
+    RADAR_CUDA_CHECK(radar_opt_in_smem(ctx, RADAR_SMEM_TREE_BUILD, rerank_build_tree_kernel, smem));
     {
         radar_launch_scope scope(ctx, RADAR_K_TREE_BUILD, stream);
         RADAR_CUDA_CHECK(launch_chained(rerank_build_tree_kernel, dim3(a->B), dim3(kThreads), smem, stream, p));

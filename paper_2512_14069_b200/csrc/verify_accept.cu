@@ -638,9 +638,12 @@ extern "C" int radar_accept_length_distribution(radar_ctx* ctx, const radar_accl
 // then on a cudaMalloc either fails or has to be carved out of that pool by hand, and cudaMalloc /
 // cudaFree also synchronise the whole device, which a decode loop cannot afford per step.  Such a
 // caller has inputs and outputs (they are part of its own pre-planned buffers) but no spare
-// scratch to lend.  For it the scratch lives in this library's image: one fixed array in device
-// memory that exists on every GPU from the moment the library is loaded there until the process
-// exits.
+// scratch to lend.  For it the scratch lives in this library's image: one fixed array per GPU.
+// The driver loads a library's device image lazily and allocates the array (and the kernels'
+// code) when it does, so radar_create makes that happen for its device - it resolves the array's
+// address and loads the two kernels of this path - and the array then stays until the process
+// exits.  Create the context BEFORE the host freezes device memory; the calls themselves then
+// allocate nothing.
 //
 // Consequences of that choice, all of which the caller must know:
 //   * the array has a fixed size (RADAR_NOALLOC_SCRATCH_BYTES = 1 MiB); a batch / vocabulary whose
@@ -650,9 +653,10 @@ extern "C" int radar_accept_length_distribution(radar_ctx* ctx, const radar_accl
 //     one stream are safe;
 //   * it keeps whatever the previous call left.  Nothing in this path needs zeroed scratch: every
 //     record that is read has been written earlier in the same call, so no clearing is done;
-//   * in host code the array's name is only a handle.  The first call on each device looks up the
-//     real device address with cudaGetSymbolAddress (that device must be current) and caches it;
-//     make that first call outside any stream capture.
+//   * in host code the array's name is only a handle.  radar_create looks up the real device
+//     address with cudaGetSymbolAddress (with its device current) and caches it per device; a call
+//     that finds no cached address (a context made by other means) does the look-up itself, so
+//     make the first call outside any stream capture.
 // ------------------------------------------------------------------------------------------
 #include <mutex>
 
@@ -663,6 +667,22 @@ static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoAllocScratch
 std::mutex g_noalloc_mutex;
 void* g_noalloc_addr[kNoAllocMaxDevices] = {nullptr};      // per device: device address of g_noalloc_scratch
 }  // namespace
+
+namespace radar {
+int noalloc_prepare_device(int device) {
+    if (device < 0 || device >= kNoAllocMaxDevices) return RADAR_OK;       // beyond the table: resolved per call
+    std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+    if (g_noalloc_addr[device] == nullptr) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_noalloc_scratch) != cudaSuccess || p == nullptr) return RADAR_ERR_CUDA;
+        g_noalloc_addr[device] = p;
+    }
+    cudaFuncAttributes fa;
+    if (cudaFuncGetAttributes(&fa, greedy_walk_kernel) != cudaSuccess || vocab_pass_preload_argbest() != cudaSuccess)
+        return RADAR_ERR_CUDA;
+    return RADAR_OK;
+}
+}  // namespace radar
 
 extern "C" size_t radar_noalloc_scratch_bytes(void) { return kNoAllocScratchBytes; }
 

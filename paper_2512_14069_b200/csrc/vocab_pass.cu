@@ -308,6 +308,17 @@ void vocab_pass_carve(void* ws, int rows, int n_chunks, int k, VocabPassParams* 
     p->part_s = reinterpret_cast<float*>(c);
 }
 
+// Makes the driver load the arg-best instantiations on the current device (kernel images are loaded lazily, at
+// first use, and loading allocates): a caller that must not allocate later can have it done at set-up.
+cudaError_t vocab_pass_preload_argbest() {
+    cudaFuncAttributes fa;
+    cudaError_t e = cudaFuncGetAttributes(&fa, vocab_pass_kernel<float, 16, false>);
+    if (e == cudaSuccess) e = cudaFuncGetAttributes(&fa, vocab_pass_kernel<float, 32, false>);
+    if (e == cudaSuccess) e = cudaFuncGetAttributes(&fa, vocab_pass_kernel<__nv_bfloat16, 16, false>);
+    if (e == cudaSuccess) e = cudaFuncGetAttributes(&fa, vocab_pass_kernel<__nv_bfloat16, 32, false>);
+    return e;
+}
+
 cudaError_t vocab_pass_launch(radar_ctx* ctx, int kernel_id, const VocabPassParams& p, cudaStream_t stream) {
     const int rows = p.n_seq * p.F;
     const unsigned grid = (unsigned)rows * (unsigned)p.n_chunks;

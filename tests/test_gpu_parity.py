@@ -288,11 +288,19 @@ def test_attention_long_prefix_many_segments(ctx):
     H.compare_attention(cfg, O_gpu, lse_gpu, O_ref, lse_ref, trees)
 
 
-def test_attention_reports_prefix_beyond_cache(ctx):
-    """A prefix that would read past the cache is refused on the device status word; nothing faults."""
+@pytest.mark.parametrize("kind", ["bf16_tensor_core", "f32_fma", "bf16_fma"])
+def test_attention_reports_prefix_beyond_cache(ctx, kind):
+    """A prefix that would read past the cache is refused on the device status word by both kernels (the
+    tensor-core one, and the FMA one for fp32 and for bf16 head ratios the tensor path does not take); the
+    sequence is skipped before anything of the cache is read, so nothing faults, and the other sequence's
+    output is still right."""
     import torch
     from paper_2512_14069_b200 import binding as rb
-    cfg = W.shrink(W.CONFIGS[5], cid=98, B=2, Hq=8, Hkv=2, P=(300, 300), V=2000, k=4, t_max=4, N=30)
+    if kind == "f32_fma":
+        cfg = W.shrink(W.CONFIGS[1], cid=97, B=2, Hq=4, Hkv=2, P=(300, 300), V=2000, k=4, t_max=4, N=30)
+    else:
+        Hq = 8 if kind == "bf16_tensor_core" else 6
+        cfg = W.shrink(W.CONFIGS[5], cid=98, B=2, Hq=Hq, Hkv=2, P=(300, 300), V=2000, k=4, t_max=4, N=30)
     inp = H.make_inputs(cfg)
     _, _, trees = H.oracle_expand_and_tree(cfg, inp)
     g = H.CudaRun(cfg, inp, ctx, max_prefix_len=4096)
@@ -301,10 +309,17 @@ def test_attention_reports_prefix_beyond_cache(ctx):
     s = g.step
     mask = H.to_dev(np.stack([t["mask"] for t in trees]).view(np.int64))
     n_nodes = H.to_dev(np.array([t["n_nodes"] for t in trees], np.int32))
+    path = rb.radar_tree_attention_path(B=cfg.B, Hq=cfg.Hq, Hkv=cfg.Hkv, d=cfg.d, Q=g.Q, Kc=g.Kc, Vc=g.Vc, kv_start=g.kv_start,
+                                        prefix_len=g.prefix_len, max_prefix_len=4096, Kt=g.Kt, Vt=g.Vt, mask=mask,
+                                        n_nodes=n_nodes, O=s.O, workspace=s.ws_attn)
+    assert path == (rb.RADAR_ATTN_PATH_TENSOR_CORE if kind == "bf16_tensor_core" else rb.RADAR_ATTN_PATH_FMA)
     s.attention(g.Q, g.Kc, g.Vc, g.kv_start, g.prefix_len, g.Kt, g.Vt, mask, n_nodes)
     torch.cuda.synchronize()
     assert ctx.read_device_status() == -1
     assert ctx.read_device_status() == rb.RADAR_OK
+    O_ref, _ = H.oracle_attention(cfg, inp, trees, pairs=[(0, h) for h in range(cfg.Hq)])
+    n0 = trees[0]["n_nodes"]
+    assert np.max(np.abs(s.O.float().cpu().numpy()[0, :n0] - O_ref[0, :n0])) <= H.TOL_ATTN[cfg.kv_dtype]
 
 
 def test_attention_fp32_head_dim_64_and_128(ctx):
@@ -319,8 +334,10 @@ def test_attention_fp32_head_dim_64_and_128(ctx):
         H.compare_attention(cfg, O_gpu, lse_gpu, O_ref, lse_ref, trees)
 
 
-@pytest.mark.parametrize("k,V", [(1, 77), (32, 4099), (7, 33)])
+@pytest.mark.parametrize("k,V", [(1, 77), (32, 4099), (7, 33), (32, 32003)])
 def test_expansion_edge_sizes(ctx, k, V):
+    """k = 1, k = 32 (the limit) and a vocabulary barely larger than k; k = 32 at V = 32003 is the size at which
+    the staged chunk records no longer fit next to the gate weights, so the unstaged merge has to take over."""
     t_max = 3 if k == 32 else 4
     cfg = W.shrink(W.CONFIGS[1], cid=60 + k, V=V, k=k, t_max=t_max, N=min(63, 3 * k), B=2, gate_b2_offset=5.0)
     inp = H.make_inputs(cfg, with_attention=False)
@@ -374,6 +391,14 @@ def test_host_side_argument_errors(ctx):
         s.attention(s.O, s.O, s.O, torch.zeros(1, dtype=torch.int64, device="cuda"), g.prefix_len, s.O, s.O)
     assert e.value.status == -2
     s.d = cfg.d
+    # a tensor that does not start on a 16-byte boundary is refused on the host by either kernel (nothing is launched)
+    qbuf = torch.zeros(s.O.numel() + 4, dtype=s.O.dtype, device="cuda")
+    q_off = qbuf[2:2 + s.O.numel()].view(s.O.shape)                  # 8 bytes past an aligned address (fp32)
+    kvz = torch.zeros(cfg.B * 64, cfg.Hkv, cfg.d, dtype=s.O.dtype, device="cuda")
+    with pytest.raises(rb.RadarError) as e:
+        s.attention(q_off, kvz, kvz, torch.zeros(cfg.B, dtype=torch.int64, device="cuda"), g.prefix_len, kvz.view(cfg.B, 64, cfg.Hkv, cfg.d),
+                    kvz.view(cfg.B, 64, cfg.Hkv, cfg.d))
+    assert e.value.status == -1
     # policy variants: an unknown policy, a hidden-state policy without features or with a ragged feature width
     for kw in (dict(policy=7), dict(policy=rb.RADAR_POLICY_LSTM_HIDDEN),
                dict(policy=rb.RADAR_POLICY_LSTM_HIDDEN, features=torch.zeros(cfg.t_max - 1, cfg.B, 6, device="cuda"))):
@@ -392,3 +417,49 @@ def test_host_side_argument_errors(ctx):
         assert e.value.status == -1, ps
     torch.cuda.synchronize()
     assert ctx.read_device_status() == 0
+
+
+def test_stochastic_acceptance_with_minus_inf_logits(ctx):
+    """-inf logits are legal (probability 0).  The accept call alone, on trees built from clean inputs, with
+    draft / target logits edited so that the walk meets: a child whose draft probability is 0 but whose target
+    probability is positive (accepted whatever the uniform), a child with both 0 (rejected), a draft row whose
+    whole mass sits on the rejected child (the sibling loop stops, the residual is sampled), and -inf scattered
+    over a fifth of both tensors."""
+    cfg = small(3)
+    assert cfg.mode == "stochastic"
+    inp = H.make_inputs(cfg, with_attention=False)
+    pools, traces, trees = H.oracle_expand_and_tree(cfg, inp)
+    g = H.CudaRun(cfg, inp, ctx)
+    g.expand_and_tree()
+    H.compare_tree(cfg, g, trees)
+    target = H.make_target(cfg, inp, trees).copy()
+    draft = inp["draft"].copy()
+    rng = np.random.Generator(np.random.Philox(4242))
+    for b in range(cfg.B):
+        draft[b][rng.random(draft[b].shape) < 0.2] = -np.inf
+        target[b][rng.random(target[b].shape) < 0.2] = -np.inf
+        t = trees[b]
+        kids = [j for j in range(1, t["n_nodes"]) if t["parent"][j] == 0]
+        x1, row = int(t["tok"][kids[0]]), int(t["draft_row"][0])
+        for j in kids:                                   # the root's children start from finite logits on both sides
+            draft[b, row, t["tok"][j]] = inp["draft"][b, row, t["tok"][j]]
+            target[b, 0, t["tok"][j]] = 0.0
+        if b == 0:
+            draft[b, row, x1] = -np.inf                  # q(x1) = 0 < p(x1): accepted
+        elif b == 1:
+            draft[b, row, x1] = -np.inf                  # q(x1) = p(x1) = 0: rejected, the siblings follow
+            target[b, 0, x1] = -np.inf
+        else:
+            keep = draft[b, row, x1]
+            draft[b, row, :] = -np.inf                   # all draft mass on x1 ...
+            draft[b, row, x1] = keep
+            target[b, 0, x1] = -40.0                     # ... which the target all but excludes: rejected, nothing left to propose
+    inp2 = dict(inp, draft=draft)
+    accepts = H.oracle_accept(cfg, inp2, trees, target)
+    assert accepts[0]["accept_len"] >= 1 and accepts[2]["accept_len"] == 0
+    for b in range(cfg.B):
+        assert accepts[b]["accept_margin"] > H.TAU_PROB and accepts[b]["sample_margin"] > H.TAU_PROB, (b, accepts[b])
+    g.draft = H.to_dev(draft)
+    g.inp = inp2
+    g.accept(target)
+    H.compare_accept(cfg, g, accepts)

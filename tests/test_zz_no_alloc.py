@@ -5,7 +5,9 @@ a serving engine that has given every free byte of the GPU to its own cache pool
 loop that must not pay cudaMalloc's device-wide synchronisation.  For them the library carries a
 fixed 1 MiB scratch array of its own.  This test drives that entry point through the C ABI twice
 in a row (the second call finds the first call's records still in the array) with different
-inputs and requires bit-identical results to radar_verify_accept, which gets a caller workspace.
+inputs and requires bit-identical results to radar_verify_accept, which gets a caller workspace,
+and to the CPU oracle's greedy walk; it also checks that a call leaves the amount of free device
+memory as it found it (the context's creation has already made the driver load what the path needs).
 It is collected last so that a stop-at-first-failure run has already covered everything else.
 """
 import numpy as np
@@ -39,24 +41,37 @@ def test_noalloc_greedy_accept_matches_regular_entry_point_twice_in_a_row():
         c = W.shrink(cfg, target_sigma=sigma)
         targets.append(H.to_dev(np.stack([W.target_logits(c, b, inp["draft"][b], drow[b], int(n_nodes[b]))
                                           for b in range(cfg.B)])))
+    from oracle import radar_oracle as O
+    _, _, trees = H.oracle_expand_and_tree(cfg, inp)
     expected = []
     for tl in targets:
         s.accept(tl)
         torch.cuda.synchronize()
         expected.append(_outputs(s))
+        for b in range(cfg.B):                                  # the regular entry point itself against the oracle
+            ref = O.verify_greedy(tl[b].cpu().numpy(), trees[b], cfg.t_max)
+            assert int(s.accept_len[b]) == ref["accept_len"] and int(s.next_token[b]) == ref["next_token"]
+            assert np.array_equal(s.path_nodes[b].cpu().numpy(), ref["path_nodes"])
     assert not torch.equal(expected[0][0], expected[1][0]) or not torch.equal(expected[0][3], expected[1][3])
 
-    for tl, exp in zip(targets, expected):                      # two calls in a row on the shared scratch
+    for it, (tl, exp) in enumerate(zip(targets, expected)):     # two calls in a row on the shared scratch
         for t in (s.accept_len, s.path_nodes, s.path_tokens, s.next_token, s.best_retrieve_row):
             t.fill_(-7)
+        torch.cuda.synchronize()
+        free_before = torch.cuda.mem_get_info()[0]
         rb.radar_verify_accept_greedy_noalloc(
             ctx, B=cfg.B, V=cfg.V, t_max=cfg.t_max, N=cfg.N, target_logits=tl, tree_tok=s.tree_tok,
             tree_parent=s.tree_parent, n_nodes=s.n_nodes, retrieve=s.retrieve, n_leaves=s.n_leaves,
             accept_len=s.accept_len, path_nodes=s.path_nodes, path_tokens=s.path_tokens, next_token=s.next_token,
             best_retrieve_row=s.best_retrieve_row)
         torch.cuda.synchronize()
+        assert torch.cuda.mem_get_info()[0] == free_before, "the call changed the amount of free device memory"
         for got, want in zip(_outputs(s), exp):
             assert torch.equal(got, want)                       # integer outputs: exact
+        for b in range(cfg.B):                                  # and directly against the oracle
+            ref = O.verify_greedy(tl[b].cpu().numpy(), trees[b], cfg.t_max)
+            assert int(s.accept_len[b]) == ref["accept_len"] and int(s.next_token[b]) == ref["next_token"]
+            assert int(s.best_retrieve_row[b]) == ref["best_retrieve_row"]
     assert ctx.read_device_status() == 0
 
     # a batch whose records cannot fit the fixed array is refused on the host, nothing is launched
