@@ -4,10 +4,13 @@ tree attention, acceptance) on seeded synthetic inputs.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--config C] [--impl ours|reference]
 
-Prints ONE JSON line (rank 0).  `value` = whole-job speculative steps per second with the
-inputs resident in HBM; `e2e` = the same through host buffers (H2D of every input and D2H of the
-result inside the timed region); `roofline` = the dominant kernel's algorithmic bytes / its
-CUDA-event duration against the measured HBM peak; `cpu_baseline` = the CPU oracle on the host.
+Prints ONE JSON line (rank 0).  The workload is the largest configuration (config 5: batch 32, ragged
+prefixes up to 32768) unless --config says otherwise.  `value` = whole-job speculative steps per second
+with the inputs resident in HBM (median of `blocks` timed blocks of K steps each; every block's time is
+listed); `e2e` = the same through host buffers (H2D of every input and D2H of the result inside the
+timed region); `roofline` = the dominant data-moving kernel's algorithmic bytes / its CUDA-event
+duration against the measured peak; `per_config` = a short timing of the other configurations;
+`cpu_baseline` = the CPU oracle on the host, single-threaded and on all cores.
 N > 1 runs independent replicas of the batch (the path has no cross-sequence exchange): weak
 scaling, no collective on the data path.
 """
@@ -34,8 +37,6 @@ L2_BYTES = 126 * 1024 * 1024
 # captures summarised under profiles/ (kernel name, config id); traffic of a launch at the same shapes =
 # ratio x its algorithmic bytes (both grow with the rows processed).  Absent = not captured.
 NCU_TRAFFIC_RATIO = {
-    ("tree_attention", 4): 451.76 / 284.58,
-    ("tree_attention", 3): 354.38 / 343.57,
     ("vocab_pass(expand)", 4): 35.949 / 35.912,
     ("vocab_pass(accept)", 4): 228.71 / 224.70,
 }
@@ -44,9 +45,12 @@ NCU_TRAFFIC_RATIO = {
 def parse():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=2000)
-    ap.add_argument("--warmup", type=int, default=20)
-    ap.add_argument("--config", type=int, default=2, choices=sorted(W.CONFIGS))
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--config", type=int, default=5, choices=sorted(W.CONFIGS))
+    ap.add_argument("--blocks", type=int, default=10, help="timed blocks of K steps (median and spread are reported)")
+    ap.add_argument("--batch", type=int, default=0, help="override the configuration's batch (reduced cases for ncu captures)")
+    ap.add_argument("--no-per-config", action="store_true", help="skip the short timing of the other configurations")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-graph", action="store_true", help="launch eagerly instead of replaying CUDA graphs")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -271,25 +275,35 @@ def scale_probe(ctx, dev, peaks, reps=20):
 # ------------------------------------------------------------------------------------------------
 # our arm
 # ------------------------------------------------------------------------------------------------
-def run_ours(args):
+def workload_string(cfg, plen):
+    return ("config %d (%s): B=%d, Hq/Hkv/d=%d/%d/%d, prefix %d..%d, V=%d, k=%d, t_max=%d, N=%d, %s"
+            % (cfg.cid, cfg.name, cfg.B, cfg.Hq, cfg.Hkv, cfg.d, int(np.min(plen)), int(np.max(plen)), cfg.V, cfg.k,
+               cfg.t_max, cfg.N, cfg.mode))
+
+
+def from_harness_inputs(inp_h, cfg):
+    """The harness' input dictionary (rank 0's sequences) in the layout host_inputs() produces."""
+    plen = np.asarray(inp_h["prefix_len"])
+    inp = {k: inp_h[k] for k in ("draft", "gate", "force_calls", "n_keep", "root_tok", "Q", "Kt", "Vt", "u_accept", "u_sample")}
+    inp["prefix_len"] = plen.astype(np.int32)
+    inp["Kc"], inp["Vc"] = np.concatenate(inp_h["Kc"], 0), np.concatenate(inp_h["Vc"], 0)
+    inp["kv_start"] = np.concatenate([[0], np.cumsum(plen)[:-1]]).astype(np.int64)
+    inp["big"] = cfg
+    return inp
+
+
+def measure_config(cfg, args, ctx, dev, rank, world, *, steps, warmup, blocks, with_e2e, inp=None, use_graph=True):
+    """Builds the device workload of `cfg`, times `blocks` blocks of `steps` steps (device time, max over ranks),
+    then per-kernel durations with an event pair around every kernel, and optionally the end-to-end figure."""
     import torch
     import torch.distributed as dist
     from paper_2512_14069_b200 import binding as rb
     from paper_2512_14069_b200.pipeline import SpecStep
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    torch.cuda.set_device(local)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
-    dev = torch.device("cuda", local)
-    cfg = W.CONFIGS[args.config]
     B, V, k, t_max = cfg.B, cfg.V, cfg.k, cfg.t_max
     sizeof_logit = 4
-
-    inp = host_inputs(cfg, rank)
-    ctx = rb.Context(local)
+    if inp is None:
+        inp = host_inputs(cfg, rank)
     kvdt = torch.float32 if cfg.kv_dtype == "f32" else torch.bfloat16
     mode = rb.RADAR_GREEDY if cfg.mode == "greedy" else rb.RADAR_STOCHASTIC
     max_p = int(inp["prefix_len"].max())
@@ -330,14 +344,20 @@ def run_ours(args):
         else:
             step.accept(c["target"], c["draft"], u_acc, u_smp)
 
+    attn_path = rb.radar_tree_attention_path(
+        B=B, Hq=cfg.Hq, Hkv=cfg.Hkv, d=cfg.d, Q=copies[0]["Q"], Kc=copies[0]["Kc"], Vc=copies[0]["Vc"], kv_start=kv_start,
+        prefix_len=prefix_len, max_prefix_len=max_p, Kt=copies[0]["Kt"], Vt=copies[0]["Vt"], mask=step.tree_mask,
+        n_nodes=step.n_nodes, O=step.O, workspace=step.ws_attn)
+
     stream = torch.cuda.Stream(dev)
     graphs = None
     with torch.cuda.stream(stream):
-        for i in range(max(args.warmup, 3)):
+        for i in range(max(warmup, 3)):
             one_step(copies[i % n_copies])
         stream.synchronize()
         ctx.check_device_status(stream)
-        if not args.no_graph:
+        accept_len = step.accept_len.cpu().numpy().tolist()
+        if use_graph:
             try:
                 graphs = []
                 for c in copies:
@@ -358,27 +378,29 @@ def run_ours(args):
             else:
                 one_step(copies[i % n_copies])
 
-        sampler = ClockSampler(local)                 # samples through the warm-up and the timed region
+        sampler = ClockSampler(torch.cuda.current_device())      # samples through the warm-up and the timed blocks
         if rank == 0:
             sampler.start()
-        for i in range(max(args.warmup, 3)):
+        for i in range(max(warmup, 3)):
             run(i)
         stream.synchronize()
 
-        # ---- timed region: exactly K steps, device time, max over ranks ----
-        ctx.reset_launch_counts()
-        if world > 1:
-            dist.barrier()
-        torch.cuda.synchronize()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record(stream)
-        for i in range(args.steps):
-            run(i)
-        e1.record(stream)
-        torch.cuda.synchronize()
-        if world > 1:
-            dist.barrier()
-        ms_total = e0.elapsed_time(e1)
+        # ---- timed blocks: exactly K steps each, device time, max over ranks ----
+        block_ms = []
+        for _ in range(blocks):
+            ctx.reset_launch_counts()
+            if world > 1:
+                dist.barrier()
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            for i in range(steps):
+                run(i)
+            e1.record(stream)
+            torch.cuda.synchronize()
+            if world > 1:
+                dist.barrier()
+            block_ms.append(reduce_max([e0.elapsed_time(e1)], dev)[0])
         clocks = sampler.stop() if rank == 0 else None
         # graph replays do not pass through the library's host-side counters: count what one step launches
         if graphs is not None:
@@ -387,13 +409,13 @@ def run_ours(args):
             stream.synchronize()
             launches_per_step = sum(v[0] for v in ctx.kernel_stats().values())
         else:
-            launches_per_step = sum(v[0] for v in ctx.kernel_stats().values()) // max(args.steps, 1)
+            launches_per_step = sum(v[0] for v in ctx.kernel_stats().values()) // max(steps, 1)
         ctx.check_device_status(stream)
 
         # ---- per-kernel durations (CUDA events around every kernel, eager launches, same rotation) ----
         # The host must stay ahead of the GPU, otherwise an event pair also spans the host's launch latency:
         # each batch of steps is enqueued behind a spinning kernel that holds the stream for a few ms.
-        prof_steps = min(args.steps, 50)
+        prof_steps = min(steps, 50)
         ctx.profile_begin(prof_steps * (2 * t_max + 8))
         for i0 in range(0, prof_steps, 5):
             torch.cuda._sleep(8_000_000)
@@ -404,37 +426,40 @@ def run_ours(args):
         kstats = ctx.kernel_stats()
 
         # ---- end to end through host buffers ----
-        pinned = {n: host[n].pin_memory() for n in names}
-        stage = copies[0]
-        res_dev = [step.accept_len, step.next_token, step.best_retrieve_row, step.path_nodes, step.path_tokens]
-        res_host = [torch.empty_like(t, device="cpu").pin_memory() for t in res_dev]
-        h2d = sum(t.numel() * t.element_size() for t in pinned.values())
-        d2h = sum(t.numel() * t.element_size() for t in res_host)
+        e2e = None
+        if with_e2e:
+            pinned = {n: host[n].pin_memory() for n in names}
+            stage = copies[0]
+            res_dev = [step.accept_len, step.next_token, step.best_retrieve_row, step.path_nodes, step.path_tokens]
+            res_host = [torch.empty_like(t, device="cpu").pin_memory() for t in res_dev]
+            h2d = sum(t.numel() * t.element_size() for t in pinned.values())
+            d2h = sum(t.numel() * t.element_size() for t in res_host)
 
-        def e2e_step():
-            for n in names:
-                stage[n].copy_(pinned[n], non_blocking=True)
-            if graphs is not None:
-                graphs[0].replay()
-            else:
-                one_step(stage)
-            for hst, dv in zip(res_host, res_dev):
-                hst.copy_(dv, non_blocking=True)
-            stream.synchronize()
+            def e2e_step():
+                for n in names:
+                    stage[n].copy_(pinned[n], non_blocking=True)
+                if graphs is not None:
+                    graphs[0].replay()
+                else:
+                    one_step(stage)
+                for hst, dv in zip(res_host, res_dev):
+                    hst.copy_(dv, non_blocking=True)
+                stream.synchronize()
 
-        for _ in range(3):
-            e2e_step()
-        e2e_steps = max(3, min(args.steps, 30))
-        if world > 1:
-            dist.barrier()
-        t0 = time.perf_counter()
-        for _ in range(e2e_steps):
-            e2e_step()
-        e2e_s = time.perf_counter() - t0
+            for _ in range(3):
+                e2e_step()
+            e2e_steps = max(3, min(steps, 30))
+            if world > 1:
+                dist.barrier()
+            t0 = time.perf_counter()
+            for _ in range(e2e_steps):
+                e2e_step()
+            e2e_s = reduce_max([time.perf_counter() - t0], dev)[0]
+            e2e = {"value": world * e2e_steps / e2e_s, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
 
-    ms_total, e2e_s = reduce_max([ms_total, e2e_s], dev)
-    ms_per_step = ms_total / args.steps
-    value = whole_job_value(world, args.steps, ms_total)
+    ms_total = float(np.median(block_ms))
+    ms_per_step = ms_total / steps
+    value = whole_job_value(world, steps, ms_total)
     tree_rows = int(n_nodes.sum())
 
     # ---- roofline of the dominant kernel ----
@@ -453,7 +478,6 @@ def run_ours(args):
     # cluster barriers, not by bandwidth: it is listed in `kernels` without a roofline model)
     timed = {n: v for n, v in kstats.items() if v[2] > 0}
     peaks = measured_peaks()
-    peak = peaks["hbm_gbs"]
     kernels = {n: {"launches_per_step": v[2] / prof_steps, "avg_us": 1000.0 * v[1] / v[2],
                    "share": v[1] / sum(x[1] for x in timed.values())} for n, v in timed.items()}
     for n in kernels:
@@ -475,32 +499,88 @@ def run_ours(args):
         if dom_overall != dom:
             roofline["note"] = ("%s has the largest share of device time (%.0f %%) but is a latency-bound per-sequence "
                                 "block with no bandwidth model" % (dom_overall, 100 * kernels[dom_overall]["share"]))
-
-    out = {
-        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
-        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "f32" if cfg.kv_dtype == "f32" else "bf16", "data": "synthetic",
-        "config": {"workload": "config %d (%s): B=%d, Hq/Hkv/d=%d/%d/%d, prefix %s, V=%d, k=%d, t_max=%d, N=%d, %s"
-                   % (cfg.cid, cfg.name, B, cfg.Hq, cfg.Hkv, cfg.d, "%d..%d" % (plen.min(), plen.max()), V, k, t_max,
-                      cfg.N, cfg.mode),
+    launch_kind = "cuda graph replay" if graphs is not None else "eager"
+    del copies, graphs
+    torch.cuda.empty_cache()
+    return {
+        "value": value, "ms_per_step": ms_per_step, "block_ms": block_ms, "clocks": clocks, "e2e": e2e,
+        "launches_per_step": int(launches_per_step), "roofline": roofline, "kernels": kernels, "tree_rows": tree_rows,
+        "config": {"workload": workload_string(cfg, plen),
                    "per_gpu_batch": B, "draft_calls_per_seq": calls.tolist(), "tree_rows_per_seq": n_nodes.tolist(),
+                   "accepted_draft_tokens_per_seq": accept_len,
                    "logits_dtype": "f32", "kv_dtype": cfg.kv_dtype, "layers_of_attention": 1,
+                   "attention_kernel": "tensor core (tcgen05)" if attn_path == rb.RADAR_ATTN_PATH_TENSOR_CORE else "fp32 FMA",
                    "l2": "inputs rotate over %d copies (%.0f MB each), more than L2 between reuses" % (n_copies, bytes_per_copy / 1e6),
-                   "launch": "cuda graph replay" if graphs is not None else "eager"},
-        "tree_tokens_per_s": value * tree_rows,
-        "clocks": clocks,
-        "e2e": {"value": world * e2e_steps / e2e_s, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
-        "gpu_launches": int(launches_per_step * args.steps),
-        "roofline": roofline,
-        "kernels": kernels,
+                   "launch": launch_kind},
     }
-    if rank == 0 and world == 1 and not args.no_scale_probe:
-        del copies, graphs
-        torch.cuda.empty_cache()
-        out["rooflines_at_scale"] = scale_probe(ctx, dev, peaks)
+
+
+def run_ours(args):
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    cfg = W.CONFIGS[args.config]
+    if args.batch > 0:
+        cfg = W.shrink(cfg, B=args.batch)
+    solo = rank == 0 and world == 1
+
+    # The CPU oracle legs run first, before this process touches CUDA: the all-core leg forks workers.
+    cpu = None
+    inp = None
+    if solo and not args.no_cpu_baseline:
+        wl = OracleWorkload(cfg)
+        cpu = cpu_baseline(cfg, budget_s=12.0, wl=wl)
+        inp = from_harness_inputs(wl.inp, cfg)               # the same seeded tensors, generated once
+        del wl
+
+    import torch
+    import torch.distributed as dist
+    from paper_2512_14069_b200 import binding as rb
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    dev = torch.device("cuda", local)
+    ctx = rb.Context(local)
+
+    m = measure_config(cfg, args, ctx, dev, rank, world, steps=args.steps, warmup=args.warmup, blocks=max(1, args.blocks),
+                       with_e2e=True, inp=inp, use_graph=not args.no_graph)
+    del inp
+    out = {
+        "metric": METRIC, "value": m["value"], "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": m["ms_per_step"], "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32" if cfg.kv_dtype == "f32" else "bf16", "data": "synthetic",
+        "config": m["config"],
+        "timed_blocks": {"blocks": len(m["block_ms"]), "steps_per_block": args.steps, "value_from": "median block",
+                         "ms_per_block": [round(x, 4) for x in m["block_ms"]],
+                         "ms_per_step_min_median_max": [min(m["block_ms"]) / args.steps, m["ms_per_step"], max(m["block_ms"]) / args.steps]},
+        "tree_tokens_per_s": m["value"] * m["tree_rows"],
+        "clocks": m["clocks"],
+        "e2e": m["e2e"],
+        "gpu_launches": int(m["launches_per_step"] * args.steps),
+        "roofline": m["roofline"],
+        "kernels": m["kernels"],
+    }
+    if solo and not args.no_per_config:
+        per = {}
+        for cid in sorted(W.CONFIGS):
+            if cid == cfg.cid and args.batch == 0:
+                r = m
+            else:
+                c2 = W.CONFIGS[cid]
+                r = measure_config(c2, args, ctx, dev, rank, world, steps=min(args.steps, 100), warmup=3, blocks=3, with_e2e=False)
+            rf = r["roofline"] or {}
+            per[str(cid)] = {"workload": r["config"]["workload"], "ms_per_step": r["ms_per_step"], "steps_per_s": r["value"],
+                             "draft_calls_per_seq": r["config"]["draft_calls_per_seq"],
+                             "accepted_draft_tokens_per_seq": r["config"]["accepted_draft_tokens_per_seq"],
+                             "dominant_kernel": rf.get("kernel"), "bound": rf.get("bound"), "frac": rf.get("frac"),
+                             "dominant_overall": rf.get("dominant_overall"),
+                             "kernel_us": {n: round(v["avg_us"] * v["launches_per_step"], 2) for n, v in r["kernels"].items()}}
+        out["per_config"] = per
+    if solo and not args.no_scale_probe:
+        out["rooflines_at_scale"] = scale_probe(ctx, dev, measured_peaks())
         out["next_rows"] = next_rows_probe(ctx, dev)
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        out["cpu_baseline"] = cpu_baseline(cfg, budget_s=15.0)
+    if cpu is not None:
+        out["cpu_baseline"] = cpu
     if rank == 0:
         print(json.dumps(out))
     if world > 1:
@@ -512,7 +592,8 @@ def run_ours(args):
 # ------------------------------------------------------------------------------------------------
 class OracleWorkload:
     """The oracle's whole step on rank 0's batch, with a knob that runs only a fraction of the three
-    heavy loops (draft rows, attention (sequence, head) pairs, target rows)."""
+    heavy loops (draft rows, attention (sequence, head) pairs, target rows), and of that fraction only
+    the share of one of several workers."""
 
     def __init__(self, cfg):
         sys.path.insert(0, os.path.join(ROOT, "tests"))
@@ -528,18 +609,21 @@ class OracleWorkload:
         H.oracle_attention(cfg, self.inp, trees)
         H.oracle_accept(cfg, self.inp, trees, self.target)
 
-    def sampled_step(self, frac):
-        """Fraction `frac` of the heavy units; the light parts (frontier, gate, tree, walk: well under 1 %
-        of the oracle's time) are not repeated."""
+    def sampled_step(self, frac, part=(0, 1)):
+        """Fraction `frac` of the heavy units, of which worker part[0] of part[1] takes every part[1]-th; the light
+        parts (frontier, gate, tree, walk: well under 1 % of the oracle's time) are not repeated."""
         from oracle import radar_oracle as O
         cfg, inp = self.cfg, self.inp
+        w, n = part
+        take = lambda xs: xs[: max(1, int(round(frac * len(xs))))][w::n]
         rows = [(b, r) for b in range(cfg.B) for r in range(1 + (len(self.traces[b]) - 1) * cfg.k)]
-        for b, r in rows[: max(1, int(round(frac * len(rows))))]:
+        for b, r in take(rows):
             O.vocab_topk(inp["draft"][b, r], cfg.k)
-        pairs = [(b, h) for b in range(cfg.B) for h in range(cfg.Hq)]
-        self.H.oracle_attention(cfg, inp, self.trees, pairs=pairs[: max(1, int(round(frac * len(pairs))))])
+        pairs = take([(b, h) for b in range(cfg.B) for h in range(cfg.Hq)])
+        if pairs:
+            self.H.oracle_attention(cfg, inp, self.trees, pairs=pairs)
         trows = [(b, i) for b in range(cfg.B) for i in range(self.trees[b]["n_nodes"])]
-        for b, i in trows[: max(1, int(round(frac * len(trows))))]:
+        for b, i in take(trows):
             if cfg.mode == "greedy":
                 int(np.argmax(self.target[b, i]))
             else:
@@ -621,35 +705,67 @@ def next_rows_probe(ctx, dev, reps=10):
     }
 
 
-def cpu_baseline(cfg, budget_s):
+_POOL_WL = None                      # the workload the forked workers of the all-core leg share (copy on write)
+
+
+def _pool_task(t):
+    frac, w, n = t
+    _POOL_WL.sampled_step(frac, part=(w, n))
+    return 0
+
+
+def cpu_baseline(cfg, budget_s, wl=None):
+    """The oracle as it stands, timed twice on this host: on one core, and with its heavy loops (which are
+    independent per row / per (sequence, head) pair) dealt out over one forked worker per core.  Must run
+    before the process initialises CUDA (the workers are forked)."""
+    global _POOL_WL
+    import multiprocessing as mp
+    ncpu = os.cpu_count() or 1
     with _single_thread():
-        wl = OracleWorkload(cfg)
+        wl = wl or OracleWorkload(cfg)
         t0 = time.perf_counter()
-        wl.full_step() if cfg.cid <= 2 else wl.sampled_step(0.02)
-        probe = time.perf_counter() - t0
-        full_est = probe if cfg.cid <= 2 else probe / 0.02
-        frac = 1.0 if full_est <= budget_s else max(budget_s / full_est, 1e-3)
-        reps = max(1, int(budget_s / max(full_est * frac, 1e-3))) if frac == 1.0 else 1
+        wl.sampled_step(0.02)
+        full_est = (time.perf_counter() - t0) / 0.02
+        frac = min(1.0, max(budget_s / full_est, 1e-3))
         t0 = time.perf_counter()
-        for _ in range(reps):
-            wl.full_step() if frac == 1.0 else wl.sampled_step(frac)
-        dt = (time.perf_counter() - t0) / reps
-    return {"value": frac / dt, "unit": UNIT, "cores": 1, "kind": "oracle",
-            "sample": ("whole step, %d repetitions" % reps) if frac == 1.0 else
-            ("fraction %.4f of the draft rows, attention (sequence, head) pairs and target rows of one step" % frac)}
+        wl.sampled_step(frac)
+        dt1 = time.perf_counter() - t0
+        single = {"value": frac / dt1, "cores": 1,
+                  "sample": "fraction %.4f of the draft rows, attention (sequence, head) pairs and target rows of one step" % frac}
+        # all cores: the same loops, a larger fraction, one worker per core
+        frac_n = min(1.0, frac * ncpu)
+        _POOL_WL = wl
+        try:
+            with mp.get_context("fork").Pool(ncpu) as pool:
+                pool.map(_pool_task, [(1e-4, w, ncpu) for w in range(ncpu)])         # start the workers
+                t0 = time.perf_counter()
+                pool.map(_pool_task, [(frac_n, w, ncpu) for w in range(ncpu)])
+                dtn = time.perf_counter() - t0
+            multi = {"value": frac_n / dtn, "cores": ncpu,
+                     "sample": "fraction %.4f of the same units, dealt out over %d forked workers" % (frac_n, ncpu)}
+        except Exception as e:  # pragma: no cover
+            multi = {"value": None, "cores": ncpu, "sample": "all-core leg failed: %s" % e}
+        _POOL_WL = None
+    best = multi if multi["value"] else single
+    return {"value": best["value"], "unit": UNIT, "cores": best["cores"], "kind": "oracle", "sample": best["sample"],
+            "host_cores": ncpu, "single_core": single, "all_cores": multi}
 
 
 def run_reference(args):
+    """The reference arm: the CPU oracle on the same configuration, one core (the all-core figure is part of
+    `cpu_baseline` of the GPU arm's line); each step is a bounded sample of the workload."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
     cfg = W.CONFIGS[args.config]
+    if args.batch > 0:
+        cfg = W.shrink(cfg, B=args.batch)
     with _single_thread():
         wl = OracleWorkload(cfg)
         t0 = time.perf_counter()
-        wl.sampled_step(0.05)
-        full_est = (time.perf_counter() - t0) / 0.05
-        budget = 150.0 / (args.steps + args.warmup)
+        wl.sampled_step(0.02)
+        full_est = (time.perf_counter() - t0) / 0.02
+        budget = 100.0 / (args.steps + args.warmup)
         frac = min(1.0, max(budget / full_est, 1e-4))
         stepf = (lambda: wl.full_step()) if frac >= 1.0 else (lambda: wl.sampled_step(frac))
         for _ in range(args.warmup):
@@ -666,9 +782,10 @@ def run_reference(args):
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": 1000.0 / value, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": "config %d (%s), CPU oracle" % (cfg.cid, cfg.name)},
+        "config": {"workload": workload_string(cfg, wl.inp["prefix_len"]), "arithmetic": "CPU oracle, fp64"},
         "tree_tokens_per_s": value * n_rows,
-        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample,
+                         "host_cores": os.cpu_count()},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }))
