@@ -247,6 +247,25 @@ def scale_probe(ctx, dev, peaks, reps=20):
     ctx.check_device_status()
     kp = ctx.kernel_stats()["tree_attention"]
     us_attn_paged = 1000.0 * kp[1] / kp[2]
+    # the multi-layer form: 32 layers of the same shapes in ONE launch (random K / V per layer, the same trees)
+    n_layers = 32
+    QL = torch.randn(n_layers, B, 64, Hq, d, device=dev, generator=g).bfloat16()
+    KtL, VtL = (torch.randn(n_layers, B, 64, Hkv, d, device=dev, generator=g).bfloat16() for _ in range(2))
+    KcL, VcL = (torch.randn(n_layers, B * P, Hkv, d, device=dev, generator=g).bfloat16() for _ in range(2))
+    OL = torch.zeros_like(QL)
+    ctx.profile_begin(16)
+    for i in range(3):
+        torch.cuda._sleep(2_000_000)
+        rb.radar_tree_attention(ctx, B=B, Hq=Hq, Hkv=Hkv, d=d, Q=QL, Kc=KcL, Vc=VcL, kv_start=kv_start, prefix_len=plen,
+                                max_prefix_len=P, Kt=KtL, Vt=VtL, mask=step.tree_mask, n_nodes=step.n_nodes, O=OL,
+                                workspace=step.ws_attn, n_layers=n_layers)
+        torch.cuda.synchronize()
+    ctx.profile_end()
+    ctx.check_device_status()
+    kl = ctx.kernel_stats()
+    us_attn_layers = 1000.0 * (kl["tree_attention"][1] + kl["tree_attention_combine"][1]) / kl["tree_attention"][2] / n_layers
+    del QL, KtL, VtL, KcL, VcL, OL
+    torch.cuda.empty_cache()
     kv_bytes = float(((P + n_nodes) * Hkv * d * 2 * 2).sum() + 2 * n_nodes.sum() * Hq * d * 2)
     flops = float((4 * n_nodes * Hq * (P + n_nodes) * d).sum())
     shapes = "LLaMA-3.3-70B shapes: B=8, Hq/Hkv/d=64/8/128, prefix 8192, V=128256, k=10, %d..%d tree rows" % (n_nodes.min(), n_nodes.max())
@@ -256,6 +275,9 @@ def scale_probe(ctx, dev, peaks, reps=20):
     kpg = {"avg_us": us_attn_paged, "alg_bytes_per_launch": kv_bytes, "gbs": kv_bytes / us_attn_paged / 1e3,
            "tflops": flops / us_attn_paged / 1e6}
     out.append(roofline_entry("tree_attention(paged cache, 16-token pages)", kpg, peaks, None))
+    kml = {"avg_us": us_attn_layers, "alg_bytes_per_launch": kv_bytes, "gbs": kv_bytes / us_attn_layers / 1e3,
+           "tflops": flops / us_attn_layers / 1e6}
+    out.append(roofline_entry("tree_attention(32 layers in one launch, per layer, combine included)", kml, peaks, None))
     b_acc = float(n_nodes.sum()) * V * 4
     out.append(roofline_entry("vocab_pass(accept)", {"avg_us": us_acc, "alg_bytes_per_launch": b_acc,
                                                      "gbs": b_acc / us_acc / 1e3}, peaks,

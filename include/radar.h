@@ -209,6 +209,11 @@ int radar_rerank_build_tree(radar_ctx* ctx, const radar_tree_args* args, void* s
  * A page index whose page does not lie inside [0, cache_rows) records RADAR_ERR_INVALID_ARG on the
  * device status word (the read goes to page 0).  The paper has no paged cache; this is the layout
  * serving systems keep their KV in, so that verification can read it in place.
+ * Multi-layer form (n_layers > 1; Sec. 3: the target model's one parallel pass runs every layer over the same
+ * tree): the same attention for n_layers sets of Q / K / V / O that share the tree, its masks and the prefix
+ * lengths - the verification pass of a whole model issues its layers' attention in one call.  On the
+ * tensor-core path all layers run in ONE persistent launch (the tile space of a layer is repeated per layer and
+ * cut into equal ranges as before); the FMA path launches layer by layer.  The workspace of one layer suffices.
  * Limits: d in {64, 128}; Hq a multiple of Hkv; cache_rows < 2^31.
  */
 typedef struct {
@@ -231,6 +236,15 @@ typedef struct {
     const int32_t* block_table;         /* [B][max_pages] page indices, or NULL for the contiguous layout */
     int page_size;                      /* tokens per page                                               */
     int max_pages;                      /* entries per sequence in block_table                           */
+    /* Several layers in one call (0 or 1: one layer, the strides are ignored).  Layer l uses Q, Kc / Vc, Kt / Vt, O
+     * and lse at l times the given stride (in ELEMENTS of the tensor's type; multiples of 8 elements); the tree
+     * (mask, n_nodes), prefix_len, kv_start, block_table, scale and the workspace are the same for all layers. */
+    int n_layers;
+    int64_t q_layer_stride;             /* also the stride of O                                          */
+    int64_t cache_layer_stride;         /* Kc and Vc                                                     */
+    int64_t tree_kv_layer_stride;       /* Kt and Vt                                                     */
+    int64_t o_layer_stride;
+    int64_t lse_layer_stride;
 } radar_attn_args;
 
 enum { RADAR_ATTN_PATH_FMA = 0, RADAR_ATTN_PATH_TENSOR_CORE = 1 };

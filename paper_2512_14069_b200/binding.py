@@ -60,6 +60,8 @@ class AttnArgs(ctypes.Structure):
         ("cache_rows", _c_i64), ("Kt", _vp), ("Vt", _vp), ("mask", _vp), ("n_nodes", _vp), ("scale", _c_f), ("O", _vp), ("lse", _vp),
         ("workspace", _vp), ("workspace_bytes", _sz),
         ("block_table", _vp), ("page_size", _c_int), ("max_pages", _c_int),
+        ("n_layers", _c_int), ("q_layer_stride", _c_i64), ("cache_layer_stride", _c_i64),
+        ("tree_kv_layer_stride", _c_i64), ("o_layer_stride", _c_i64), ("lse_layer_stride", _c_i64),
     ]
 
 
@@ -285,8 +287,16 @@ def radar_rerank_build_tree(ctx: Context, *, B, N, t_max, pool_capacity, pool_to
 
 
 def _attn_args(*, B, Hq, Hkv, d, Q, Kc, Vc, kv_start, prefix_len, max_prefix_len, Kt, Vt, mask, n_nodes, O, workspace,
-               lse=None, scale=0.0, block_table=None, page_size=0):
+               lse=None, scale=0.0, block_table=None, page_size=0, n_layers=1):
+    """With n_layers > 1 every tensor carries a leading layer dimension: Q, O [L, B, 64, Hq, d]; Kt, Vt [L, B, 64, Hkv, d];
+    Kc, Vc [L, cache_rows, Hkv, d]; lse [L, B, Hq, 64]."""
     a = AttnArgs()
+    if n_layers > 1:
+        a.n_layers = n_layers
+        a.q_layer_stride, a.o_layer_stride = Q[0].numel(), O[0].numel()
+        a.tree_kv_layer_stride = Kt[0].numel()
+        a.cache_layer_stride = 0 if Kc is None else Kc[0].numel()
+        a.lse_layer_stride = 0 if lse is None else lse[0].numel()
     a.B, a.Hq, a.Hkv, a.d, a.dtype = B, Hq, Hkv, d, dtype_code(Q)
     for t in (Kc, Vc, Kt, Vt, O):
         if t is not None and t.dtype != Q.dtype:
@@ -294,7 +304,7 @@ def _attn_args(*, B, Hq, Hkv, d, Q, Kc, Vc, kv_start, prefix_len, max_prefix_len
     a.Q, a.Kc, a.Vc = _ptr(Q), _ptr(Kc), _ptr(Vc)
     a.kv_start, a.prefix_len = _ptr(kv_start, torch.int64), _ptr(prefix_len, torch.int32)
     a.max_prefix_len = max_prefix_len
-    a.cache_rows = 0 if Kc is None else min(Kc.numel(), Vc.numel()) // (Hkv * d)      # token rows [Hkv][d]
+    a.cache_rows = 0 if Kc is None else min(Kc.numel(), Vc.numel()) // (Hkv * d * max(n_layers, 1))   # token rows [Hkv][d] per layer
     a.Kt, a.Vt, a.mask, a.n_nodes = _ptr(Kt), _ptr(Vt), _ptr(mask, torch.int64), _ptr(n_nodes, torch.int32)
     a.scale, a.O, a.lse = scale, _ptr(O), _ptr(lse, torch.float32)
     a.workspace, a.workspace_bytes = _ptr(workspace), workspace.numel() * workspace.element_size()

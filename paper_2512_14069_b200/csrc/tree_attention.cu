@@ -350,7 +350,30 @@ extern "C" int radar_tree_attention(radar_ctx* ctx, const radar_attn_args* a, vo
           reinterpret_cast<uintptr_t>(a->Kt) | reinterpret_cast<uintptr_t>(a->Vt) | reinterpret_cast<uintptr_t>(a->O)) & 15) != 0)
         return RADAR_ERR_INVALID_ARG;
     if (a->max_prefix_len > 0 && a->cache_rows <= 0) return RADAR_ERR_INVALID_ARG;
+    const int n_layers = a->n_layers > 1 ? a->n_layers : 1;
+    if (n_layers > 1 && (((a->q_layer_stride | a->cache_layer_stride | a->tree_kv_layer_stride | a->o_layer_stride) & 7) != 0 ||
+                         a->q_layer_stride <= 0 || a->tree_kv_layer_stride <= 0 || a->o_layer_stride <= 0 ||
+                         (a->max_prefix_len > 0 && a->cache_layer_stride <= 0) || (a->lse != nullptr && a->lse_layer_stride <= 0)))
+        return RADAR_ERR_INVALID_ARG;
     if (tree_attn_tc_supported(a)) return tree_attn_tc_launch(ctx, a, stream);
+    if (n_layers > 1) {
+        // the FMA kernel takes one layer per launch
+        const size_t es = a->dtype == RADAR_F32 ? 4 : 2;
+        for (int l = 0; l < n_layers; ++l) {
+            radar_attn_args one = *a;
+            one.n_layers = 1;
+            one.Q = reinterpret_cast<const char*>(a->Q) + (size_t)l * a->q_layer_stride * es;
+            one.Kt = reinterpret_cast<const char*>(a->Kt) + (size_t)l * a->tree_kv_layer_stride * es;
+            one.Vt = reinterpret_cast<const char*>(a->Vt) + (size_t)l * a->tree_kv_layer_stride * es;
+            if (a->Kc) one.Kc = reinterpret_cast<const char*>(a->Kc) + (size_t)l * a->cache_layer_stride * es;
+            if (a->Vc) one.Vc = reinterpret_cast<const char*>(a->Vc) + (size_t)l * a->cache_layer_stride * es;
+            one.O = reinterpret_cast<char*>(a->O) + (size_t)l * a->o_layer_stride * es;
+            if (a->lse) one.lse = a->lse + (size_t)l * a->lse_layer_stride;
+            const int rc = radar_tree_attention(ctx, &one, stream_);
+            if (rc != RADAR_OK) return rc;
+        }
+        return RADAR_OK;
+    }
 
     AttnParams P;
     P.a = *a;

@@ -50,6 +50,7 @@ constexpr float kRescaleThreshold = 8.f;   // in log2 units: P stays below 2^8
 struct CutUnit {
     int valid;           // 1: this CTA's last segment starts a unit that continues in the following CTAs
     int b, g, nt;        // the unit and its number of tiles
+    int layer;           // the layer it belongs to
     int slot;            // partial slot of that first piece in this CTA (0 or 1)
     int rows;            // live query rows of the unit
     int w;               // cost of one of its tiles
@@ -61,6 +62,8 @@ struct TcParams {
     radar_attn_args a;
     int G, nodes_per_rb;
     int pair_rows;       // query rows of a class's units: 256 (two row blocks share each K/V tile) or 128
+    int n_layers;        // layers run by this launch (the same tree, masks and prefix lengths for all)
+    long long o_ls, lse_ls;   // elements between consecutive layers of O and of lse
     int n_cls;           // classes = units per KV head
     int ncc;             // CTAs per class; grid = n_cls * ncc
     float scale_log2;
@@ -119,6 +122,7 @@ __device__ __forceinline__ int tiles_before(long long x, long long U, int nt, in
 template <bool PAGED>
 struct Cursor {
     int b, g, t0, t1;
+    int layer;           // layers follow one another in the space, each with the same sequence of units
     long long U, hi;     // start position of the current unit, end of the CTA's range
     SeqInfo s;
     __device__ __forceinline__ bool valid() const { return t1 > t0; }
@@ -128,7 +132,13 @@ struct Cursor {
         t0 = 0;
         if (++g == P.a.Hkv) {
             g = 0;
-            do { ++b; if (b >= P.a.B) { t1 = 0; return; } s = seq_info<PAGED>(P, b, pp); } while (s.rows == 0);
+            do {
+                if (++b >= P.a.B) {                               // the next layer starts over at the first sequence
+                    if (++layer >= P.n_layers) { t1 = 0; return; }
+                    b = 0;
+                }
+                s = seq_info<PAGED>(P, b, pp);
+            } while (s.rows == 0);
         }
         clip();
     }
@@ -176,13 +186,14 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     struct __align__(1024) Static {
         uint64_t bar_qfull, bar_qempty, bar_kfull[3], bar_kempty[3], bar_vfull[3], bar_vempty[3];
         uint64_t bar_sfull[2], bar_pready[2], bar_odone[2], bar_ofree[2];
-        long long range[4];      // this CTA's range [lo, hi), size of the class's space, start of its first unit
-        int start[2];            // sequence and KV head of the unit that contains lo
+        long long range[4];      // this CTA's range [lo, hi), size of the class's space (all layers), start of its first unit
+        int start[3];            // sequence, KV head and layer of the unit that contains lo
+        int start_pad;
         uint32_t tmem_base;
         int abort;
         float xm[128];           // group 1's running max at the end of a segment (one live row block)
         float mx[2][2][128];     // per group and column half: row maxima of a tile; row sums at the end of a segment
-        unsigned char pad[kStaticSmem - (22 * 8 + 4 * 8 + 2 * 4 + 4 + 4 + 128 * 4 + 2 * 2 * 128 * 4)];
+        unsigned char pad[kStaticSmem - (22 * 8 + 4 * 8 + 4 * 4 + 4 + 4 + 128 * 4 + 2 * 2 * 128 * 4)];
     };
     static_assert(sizeof(Static) == kStaticSmem, "static shared-memory block");
     __shared__ Static st;
@@ -207,7 +218,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     float (&s_mx)[2][2][128] = st.mx;
     float (&s_xl)[2][2][128] = st.mx;        // same storage: the two uses never overlap in time
     long long (&s_range)[4] = st.range;
-    int (&s_start)[2] = st.start;
+    int (&s_start)[3] = st.start;
     const bool smem_aligned = (smem_u32(smem_raw) & 1023u) == 0;
 
     // ---- set-up: warp 0 finds this CTA's range while the barriers and tensor memory are prepared ----
@@ -226,7 +237,11 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             for (int o = 16; o > 0; o >>= 1) sz += __shfl_xor_sync(kFull, sz, o);
             tot += sz;
         }
-        const long long lo = tot * ci / P.ncc, hi = tot * (ci + 1) / P.ncc;
+        // the space of all layers: layer l occupies [l * tot, (l + 1) * tot)
+        const long long tot_all = tot * P.n_layers;
+        const long long lo_all = tot_all * ci / P.ncc, hi = tot_all * (ci + 1) / P.ncc;
+        const int layer0 = tot > 0 ? (int)(lo_all / tot) : 0;
+        const long long lo = lo_all - (long long)layer0 * tot;
         long long cum = 0, fU = 0;
         int fb = -1, fg = 0;
         for (int b0 = 0; b0 < a.B && fb < 0; b0 += 32) {
@@ -251,8 +266,8 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             cum += __shfl_sync(kFull, incl, 31);
         }
         if (lane == 0) {
-            s_range[0] = lo; s_range[1] = hi; s_range[2] = tot; s_range[3] = fU;
-            s_start[0] = fb; s_start[1] = fg;
+            s_range[0] = lo_all; s_range[1] = hi; s_range[2] = tot_all; s_range[3] = fU + (long long)layer0 * tot;
+            s_start[0] = layer0 < P.n_layers ? fb : -1; s_start[1] = fg; s_start[2] = layer0;
         }
     } else if (warp == 1) {
         if (lane == 0) {
@@ -285,7 +300,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
 
     // first segment: the unit that contains the range's start, from its first tile starting at or after it
     Cursor<PAGED> cur;
-    cur.b = s_start[0]; cur.g = s_start[1];
+    cur.b = s_start[0]; cur.g = s_start[1]; cur.layer = s_start[2];
     cur.hi = s_range[1];
     cur.U = s_range[3];
     cur.t0 = cur.t1 = 0;
@@ -321,7 +336,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 const int b = cur.b, g = cur.g, n = cur.t1 - cur.t0;
                 const bool two = TWO && cur.two_rb();
                 if (cur.t0 == 0 && cur.t1 < cur.s.nt) {          // necessarily the last segment of this CTA
-                    cu.valid = 1; cu.b = b; cu.g = g; cu.nt = cur.s.nt; cu.slot = seg == 0 ? 0 : 1;
+                    cu.valid = 1; cu.b = b; cu.g = g; cu.nt = cur.s.nt; cu.slot = seg == 0 ? 0 : 1; cu.layer = cur.layer;
                     cu.rows = cur.s.rows; cu.w = cur.s.w; cu.u0 = cur.U; cu.tot = s_range[2];
                 }
                 if (lead) ok = ok && mbar_wait(&bar_qempty, (seg & 1) ^ 1, ab);
@@ -329,8 +344,8 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                     mbar_arrive_expect_tx(&bar_qfull, two ? 2 * SM::kQBlock : SM::kQBlock);
                     for (int q = 0; q < (two ? 2 : 1); ++q)
                         for (int h = 0; h < H; ++h)
-                            tma_load_3d(sQ + q * SM::kQBlock + h * (128 * 128), &tmQ, &bar_qfull, h * 64, g * G,
-                                        b * kMaxNodes + (pp * (P.pair_rows / 128) + q) * P.nodes_per_rb);
+                            tma_load_4d(sQ + q * SM::kQBlock + h * (128 * 128), &tmQ, &bar_qfull, h * 64, g * G,
+                                        b * kMaxNodes + (pp * (P.pair_rows / 128) + q) * P.nodes_per_rb, cur.layer);
                 }
                 auto load_tile = [&](int t, bool is_k) {
                     uint32_t& cnt = is_k ? kc : vc;
@@ -348,13 +363,13 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                         if (lead) {
                             mbar_arrive_expect_tx(full, kTreeKeys * D * 2);
                             for (int h = 0; h < H; ++h)
-                                tma_load_3d(dst + h * (kTreeKeys * 128), is_k ? &tmKt : &tmVt, full, h * 64, g, b * kMaxNodes);
+                                tma_load_4d(dst + h * (kTreeKeys * 128), is_k ? &tmKt : &tmVt, full, h * 64, g, b * kMaxNodes, cur.layer);
                         }
                     } else if (!PAGED) {
                         mbar_arrive_expect_tx(full, kTileKeys * D * 2);
                         const int row = (int)(cur.s.kv0 + (long long)t * kTileKeys);
                         for (int h = 0; h < H; ++h)
-                            tma_load_3d(dst + h * (kTileKeys * 128), is_k ? &tmKc : &tmVc, full, h * 64, g, row);
+                            tma_load_4d(dst + h * (kTileKeys * 128), is_k ? &tmKc : &tmVc, full, h * 64, g, row, cur.layer);
                     } else {
                         // paged cache: one box per page (or per tile when a page holds whole tiles); only pages
                         // that hold live keys are fetched, what stays stale in the slot is masked / never read
@@ -370,7 +385,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                             if (page < 0 || page >= n_cache_pages) { set_status(P.status, RADAR_ERR_INVALID_ARG); page = 0; }
                             const int row = (int)(page * ps + key % ps);
                             for (int h = 0; h < H; ++h)
-                                tma_load_3d(dst + h * (kTileKeys * 128) + p * per * 128, is_k ? &tmKc : &tmVc, full, h * 64, g, row);
+                                tma_load_4d(dst + h * (kTileKeys * 128) + p * per * 128, is_k ? &tmKc : &tmVc, full, h * 64, g, row, cur.layer);
                         }
                     }
                 };
@@ -735,7 +750,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                     }
                     if (row_live) {
                         if (final_rows) {
-                            __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(a.O) + out_row * D + col;
+                            __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(a.O) + cur.layer * P.o_ls + out_row * D + col;
 #pragma unroll
                             for (int q = 0; q < 4; ++q) {
                                 uint32_t w[4];
@@ -757,7 +772,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 if (row_live && half == 0) {
                     const float m_nat = m_safe * 0.6931471805599453f;
                     if (final_rows) {
-                        if (a.lse != nullptr) a.lse[((int64_t)b * a.Hq + hq) * kMaxNodes + node] = m_nat + logf(l_out);
+                        if (a.lse != nullptr) a.lse[cur.layer * P.lse_ls + ((int64_t)b * a.Hq + hq) * kMaxNodes + node] = m_nat + logf(l_out);
                     } else {
                         P.part_ml[rec] = make_float2(m_out == -CUDART_INF_F ? -CUDART_INF_F : m_nat, l_out);
                     }
@@ -824,10 +839,10 @@ __global__ void __launch_bounds__(256) tree_attn_tc_combine_kernel(const TcParam
         const float inv = 1.f / den;
         const int r_glob = pp * P.pair_rows + prow;
         const int node = r_glob / G, hq = cu.g * G + r_glob % G;
-        __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(a.O) + (((int64_t)cu.b * kMaxNodes + node) * a.Hq + hq) * D + lane * E;
+        __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(a.O) + cu.layer * P.o_ls + (((int64_t)cu.b * kMaxNodes + node) * a.Hq + hq) * D + lane * E;
 #pragma unroll
         for (int q = 0; q < E; q += 2) *reinterpret_cast<__nv_bfloat162*>(dst + q) = __floats2bfloat162_rn(o[q] * inv, o[q + 1] * inv);
-        if (a.lse != nullptr && lane == 0) a.lse[((int64_t)cu.b * a.Hq + hq) * kMaxNodes + node] = mx + logf(den);
+        if (a.lse != nullptr && lane == 0) a.lse[cu.layer * P.lse_ls + ((int64_t)cu.b * a.Hq + hq) * kMaxNodes + node] = mx + logf(den);
     };
 
     if (n_pieces <= 4) {
@@ -984,10 +999,10 @@ __global__ void __launch_bounds__(256) tree_attn_tc_combine_wide_kernel(const Tc
     const float inv = 1.f / den;
     const int r_glob = pp * P.pair_rows + prow;
     const int node = r_glob / G, hq = cu.g * G + r_glob % G;
-    __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(a.O) + (((int64_t)cu.b * kMaxNodes + node) * a.Hq + hq) * D + lane * (D / 32);
+    __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(a.O) + cu.layer * P.o_ls + (((int64_t)cu.b * kMaxNodes + node) * a.Hq + hq) * D + lane * (D / 32);
 #pragma unroll
     for (int q = 0; q < D / 32; ++q) dst[q] = __float2bfloat16(o[q] * inv);
-    if (a.lse != nullptr && lane == 0) a.lse[((int64_t)cu.b * a.Hq + hq) * kMaxNodes + node] = mx + logf(den);
+    if (a.lse != nullptr && lane == 0) a.lse[cu.layer * P.lse_ls + ((int64_t)cu.b * a.Hq + hq) * kMaxNodes + node] = mx + logf(den);
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -1004,15 +1019,18 @@ EncodeTiledFn encode_fn() {
     return fn;
 }
 
-// [rows][heads][d] bf16 tensor, box = (64 elements, box_heads, box_rows), 128-byte swizzle, zero fill
-bool make_map(CUtensorMap* tm, const void* base, int d, int heads, long long rows, int box_heads, int box_rows) {
+// [layers][rows][heads][d] bf16 tensor (layer_stride elements between layers), box = (64 elements, box_heads,
+// box_rows, one layer), 128-byte swizzle, zero fill
+bool make_map(CUtensorMap* tm, const void* base, int d, int heads, long long rows, int box_heads, int box_rows, int layers,
+              long long layer_stride) {
     EncodeTiledFn enc = encode_fn();
     if (!enc) return false;
-    cuuint64_t dims[3] = {(cuuint64_t)d, (cuuint64_t)heads, (cuuint64_t)rows};
-    cuuint64_t strides[2] = {(cuuint64_t)d * 2, (cuuint64_t)d * 2 * heads};
-    cuuint32_t box[3] = {64, (cuuint32_t)box_heads, (cuuint32_t)box_rows};
-    cuuint32_t es[3] = {1, 1, 1};
-    return enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, es,
+    if (layers <= 1) { layers = 1; layer_stride = rows * heads * d; }
+    cuuint64_t dims[4] = {(cuuint64_t)d, (cuuint64_t)heads, (cuuint64_t)rows, (cuuint64_t)layers};
+    cuuint64_t strides[3] = {(cuuint64_t)d * 2, (cuuint64_t)d * 2 * heads, (cuuint64_t)layer_stride * 2};
+    cuuint32_t box[4] = {64, (cuuint32_t)box_heads, (cuuint32_t)box_rows, 1};
+    cuuint32_t es[4] = {1, 1, 1, 1};
+    return enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, es,
                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
@@ -1066,11 +1084,14 @@ static int launch_tc(radar_ctx* ctx, TcParams& P, cudaStream_t stream) {
     const long long tree_rows = (long long)a.B * kMaxNodes;
     const bool have_prefix = a.Kc != nullptr && a.Vc != nullptr && a.cache_rows > 0;
     const int cache_box = a.block_table != nullptr && a.page_size < kTileKeys ? a.page_size : kTileKeys;   // rows per TMA box
-    if (!make_map(&tmQ, a.Q, D, a.Hq, tree_rows, P.G, P.nodes_per_rb) ||
-        !make_map(&tmKt, a.Kt, D, a.Hkv, tree_rows, 1, kTreeKeys) ||
-        !make_map(&tmVt, a.Vt, D, a.Hkv, tree_rows, 1, kTreeKeys) ||
-        !make_map(&tmKc, have_prefix ? a.Kc : a.Kt, D, a.Hkv, have_prefix ? a.cache_rows : tree_rows, 1, cache_box) ||
-        !make_map(&tmVc, have_prefix ? a.Vc : a.Vt, D, a.Hkv, have_prefix ? a.cache_rows : tree_rows, 1, cache_box))
+    const int L = P.n_layers;
+    if (!make_map(&tmQ, a.Q, D, a.Hq, tree_rows, P.G, P.nodes_per_rb, L, a.q_layer_stride) ||
+        !make_map(&tmKt, a.Kt, D, a.Hkv, tree_rows, 1, kTreeKeys, L, a.tree_kv_layer_stride) ||
+        !make_map(&tmVt, a.Vt, D, a.Hkv, tree_rows, 1, kTreeKeys, L, a.tree_kv_layer_stride) ||
+        !make_map(&tmKc, have_prefix ? a.Kc : a.Kt, D, a.Hkv, have_prefix ? a.cache_rows : tree_rows, 1, cache_box, L,
+                  have_prefix ? a.cache_layer_stride : a.tree_kv_layer_stride) ||
+        !make_map(&tmVc, have_prefix ? a.Vc : a.Vt, D, a.Hkv, have_prefix ? a.cache_rows : tree_rows, 1, cache_box, L,
+                  have_prefix ? a.cache_layer_stride : a.tree_kv_layer_stride))
         return RADAR_ERR_CUDA;
     RADAR_CUDA_CHECK(radar_opt_in_smem(ctx, RADAR_SMEM_ATTN_TC + 4 * (D == 128) + 2 * TWO + PAGED, tree_attn_tc_kernel<D, TWO, PAGED>,
                                        (size_t)Smem<D, TWO>::kDynamic));
@@ -1101,6 +1122,9 @@ int tree_attn_tc_launch(radar_ctx* ctx, const radar_attn_args* a, cudaStream_t s
     P.scale_log2 = scale * 1.4426950408889634f;
     P.cache_rows = a->cache_rows;
     P.status = ctx->d_status;
+    P.n_layers = a->n_layers > 1 ? a->n_layers : 1;
+    P.o_ls = P.n_layers > 1 ? a->o_layer_stride : 0;
+    P.lse_ls = P.n_layers > 1 ? a->lse_layer_stride : 0;
     plan_grid(ctx, a->B, a->Hq, a->Hkv, a->max_prefix_len, &P.pair_rows, &P.n_cls, &P.ncc);
     if (tree_attn_tc_workspace_bytes(ctx, a->B, a->Hq, a->Hkv, a->d, a->max_prefix_len) > a->workspace_bytes)
         return RADAR_ERR_WORKSPACE;

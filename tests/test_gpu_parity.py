@@ -463,3 +463,58 @@ def test_stochastic_acceptance_with_minus_inf_logits(ctx):
     g.inp = inp2
     g.accept(target)
     H.compare_accept(cfg, g, accepts)
+
+
+@pytest.mark.parametrize("kind", ["bf16_tensor_core", "bf16_two_row_blocks", "f32_fma"])
+def test_attention_several_layers_in_one_call(ctx, kind):
+    """The multi-layer form: L sets of Q / K / V that share one tree per sequence, every layer against the oracle.
+    On the tensor-core path all layers run in one persistent launch (units of a layer repeat per layer and the
+    ranges of the CTAs run across layer boundaries); the FMA path goes layer by layer."""
+    import torch
+    from paper_2512_14069_b200 import binding as rb
+    L = 3
+    if kind == "f32_fma":
+        base = W.shrink(W.CONFIGS[1], cid=150, B=2, Hq=4, Hkv=2, P=(100, 400), V=2000, k=4, t_max=4, N=30)
+    elif kind == "bf16_two_row_blocks":
+        base = W.shrink(W.CONFIGS[5], cid=151, B=3, Hq=16, Hkv=2, P=(200, 1500), V=2000, k=4, t_max=5, N=50)
+    else:
+        base = W.shrink(W.CONFIGS[5], cid=152, B=4, Hq=8, Hkv=8, P=(0, 900), V=2000, k=4, t_max=5, N=40)
+    inp0 = H.make_inputs(base)
+    if kind == "bf16_tensor_core":
+        inp0["prefix_len"][0] = 0
+    _, _, trees = H.oracle_expand_and_tree(base, inp0)
+    plen = inp0["prefix_len"]
+    layers = []
+    for l in range(L):                                  # every layer draws its own Q / K / V (another stream id), same lengths
+        c = W.shrink(base, cid=base.cid + 10 * (l + 1))
+        inp = {"Q": np.stack([W.attn_q(c, b) for b in range(c.B)]), "prefix_len": plen}
+        kt, vt = zip(*[W.attn_tree_kv(c, b) for b in range(c.B)])
+        inp["Kt"], inp["Vt"] = np.stack(kt), np.stack(vt)
+        kc, vc = zip(*[W.attn_prefix_kv(c, b, int(plen[b])) for b in range(c.B)])
+        inp["Kc"], inp["Vc"] = list(kc), list(vc)
+        layers.append(inp)
+    stack = lambda name: H.to_dev(np.stack([inp[name] for inp in layers]))
+    Q, Kt, Vt = stack("Q"), stack("Kt"), stack("Vt")
+    Kc = H.to_dev(np.stack([np.concatenate(inp["Kc"], 0) for inp in layers]))
+    Vc = H.to_dev(np.stack([np.concatenate(inp["Vc"], 0) for inp in layers]))
+    kv_start = H.to_dev(np.concatenate([[0], np.cumsum(plen)[:-1]]).astype(np.int64))
+    mask = H.to_dev(np.stack([t["mask"] for t in trees]).view(np.int64))
+    n_nodes = H.to_dev(np.array([t["n_nodes"] for t in trees], np.int32))
+    O = torch.zeros_like(Q)
+    lse = torch.zeros(L, base.B, base.Hq, 64, device="cuda")
+    maxp = int(max(plen))
+    wb = rb.radar_attn_workspace_bytes(ctx, base.B, base.Hq, base.Hkv, base.d, rb.dtype_code(Q), maxp)
+    ws = torch.zeros(wb + 256, dtype=torch.uint8, device="cuda")
+    off = (-ws.data_ptr()) % 256
+    kw = dict(B=base.B, Hq=base.Hq, Hkv=base.Hkv, d=base.d, Q=Q, Kc=Kc, Vc=Vc, kv_start=kv_start, prefix_len=H.to_dev(plen),
+              max_prefix_len=maxp, Kt=Kt, Vt=Vt, mask=mask, n_nodes=n_nodes, O=O, lse=lse, workspace=ws[off:off + wb], n_layers=L)
+    assert rb.radar_tree_attention_path(**kw) == (rb.RADAR_ATTN_PATH_FMA if kind == "f32_fma" else rb.RADAR_ATTN_PATH_TENSOR_CORE)
+    rb.radar_tree_attention(ctx, **kw)
+    ctx.check_device_status()
+    O_gpu, lse_gpu = O.float().cpu().numpy(), lse.cpu().numpy()
+    for l in range(L):
+        O_ref, lse_ref = H.oracle_attention(base, layers[l], trees)
+        H.compare_attention(base, O_gpu[l], lse_gpu[l], O_ref, lse_ref, trees)
+    # rows past a tree's end stay untouched in every layer
+    for b in range(base.B):
+        assert not O_gpu[:, b, trees[b]["n_nodes"]:].any()
