@@ -74,6 +74,11 @@ struct TcParams {
     int* status;
 };
 
+__device__ __forceinline__ float max3(float a, float b, float c) {
+    float y;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(y) : "f"(a), "f"(b), "f"(c));
+    return y;
+}
 __device__ __forceinline__ float ex2(float x) {
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -636,7 +641,8 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                         }
                         float mxa[4] = {-CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F};
 #pragma unroll
-                        for (int e = 0; e < 32; ++e) mxa[e & 3] = fmaxf(mxa[e & 3], __uint_as_float(sv[e]));
+                        for (int e = 0; e < 32; e += 2)                     // three-input maxima: half the instructions
+                            mxa[(e >> 1) & 3] = max3(mxa[(e >> 1) & 3], __uint_as_float(sv[e]), __uint_as_float(sv[e + 1]));
                         mx = fmaxf(mx, fmaxf(fmaxf(mxa[0], mxa[1]), fmaxf(mxa[2], mxa[3])));
                     }
                 }
@@ -656,7 +662,9 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                     }
                     const float m_use = m_run == -CUDART_INF_F ? 0.f : m_run;
                     // ---- P = exp2(s * scale - m), row sum, bf16 pairs back to tensor memory ----
-                    float ls[4] = {0.f, 0.f, 0.f, 0.f};
+                    // (the scaling and the row sum work on pairs: one packed fp32x2 instruction per two values)
+                    float2 ls[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
+                    const float2 sc2 = make_float2(P.scale_log2, P.scale_log2), nm2 = make_float2(-m_use, -m_use);
 #pragma unroll 1
                     for (int cc = 0; cc < nch; ++cc) {
                         uint32_t sv[32];
@@ -671,15 +679,15 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                         uint32_t pk[16];
 #pragma unroll
                         for (int e = 0; e < 16; ++e) {
-                            const float p0 = ex2(fmaf(__uint_as_float(sv[2 * e]), P.scale_log2, -m_use));
-                            const float p1 = ex2(fmaf(__uint_as_float(sv[2 * e + 1]), P.scale_log2, -m_use));
-                            ls[e & 3] += p0 + p1;
+                            const float2 t = __ffma2_rn(make_float2(__uint_as_float(sv[2 * e]), __uint_as_float(sv[2 * e + 1])), sc2, nm2);
+                            const float p0 = ex2(t.x), p1 = ex2(t.y);
+                            ls[e & 1] = __fadd2_rn(ls[e & 1], make_float2(p0, p1));
                             const __nv_bfloat162 v = __floats2bfloat162_rn(p0, p1);
                             pk[e] = *reinterpret_cast<const uint32_t*>(&v);
                         }
                         tmem_st16(tS + half * 64 + cc * 16, pk);
                     }
-                    l_run = l_run * factor + ((ls[0] + ls[1]) + (ls[2] + ls[3]));
+                    l_run = l_run * factor + ((ls[0].x + ls[0].y) + (ls[1].x + ls[1].y));
                     // ---- rescale this thread's half of the accumulator when some row of the warp moved its max ----
                     if (j > 0 && __any_sync(kFull, factor != 1.f)) {
 #pragma unroll 1
