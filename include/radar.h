@@ -108,6 +108,18 @@ int radar_reset_launch_counts(radar_ctx* ctx);
  * Everything else of the call (candidates, pool, frontier) is the same for the three.
  */
 enum { RADAR_POLICY_LSTM_SCORES = 0, RADAR_POLICY_MLP_SCORES = 1, RADAR_POLICY_LSTM_HIDDEN = 2 };
+/* `phase` lets a caller overlap the two halves of consecutive draft calls (the bandwidth-bound vocabulary pass of
+ * call t+1 next to the latency-bound select + gate block of call t, on two streams):
+ *   RADAR_EXPAND_ALL     both halves, back to back on the given stream (the default, value 0);
+ *   RADAR_EXPAND_VOCAB   only the vocabulary pass (and the input-side products of the hidden-state policy) into
+ *                        `workspace`.  `active` is only READ here, as the mask of sequences whose rows are worth
+ *                        reading: it may be an older mask than the one the select half will see (a sequence that has
+ *                        stopped since is read in vain, nothing else), or NULL for "all";
+ *   RADAR_EXPAND_SELECT  only the select + gate half, on the records a RADAR_EXPAND_VOCAB call with the same
+ *                        arguments left in the same `workspace`.  The caller orders it after that call and after the
+ *                        previous draft call's select half.
+ * Results are identical in the three forms. */
+enum { RADAR_EXPAND_ALL = 0, RADAR_EXPAND_VOCAB = 1, RADAR_EXPAND_SELECT = 2 };
 
 typedef struct {
     int B, F, V, k;
@@ -141,6 +153,7 @@ typedef struct {
     int policy;                         /* RADAR_POLICY_*                                    */
     int feat_dim;                       /* RADAR_POLICY_LSTM_HIDDEN: length of a feature row */
     const float* features;              /* RADAR_POLICY_LSTM_HIDDEN: [B][feat_dim], device   */
+    int phase;                          /* RADAR_EXPAND_*                                    */
 } radar_expand_args;
 
 size_t radar_expand_workspace_bytes(const radar_ctx* ctx, int B, int F, int V, int k);

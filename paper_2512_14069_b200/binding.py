@@ -19,6 +19,7 @@ RADAR_F32, RADAR_BF16 = 0, 1
 RADAR_GREEDY, RADAR_STOCHASTIC = 0, 1
 RADAR_POLICY_LSTM_SCORES, RADAR_POLICY_MLP_SCORES, RADAR_POLICY_LSTM_HIDDEN = 0, 1, 2
 RADAR_OK = 0
+RADAR_EXPAND_ALL, RADAR_EXPAND_VOCAB, RADAR_EXPAND_SELECT = 0, 1, 2
 RADAR_ATTN_PATH_FMA, RADAR_ATTN_PATH_TENSOR_CORE = 0, 1
 
 _c_int, _c_i64, _c_f, _vp, _sz = ctypes.c_int, ctypes.c_int64, ctypes.c_float, ctypes.c_void_p, ctypes.c_size_t
@@ -38,7 +39,7 @@ class ExpandArgs(ctypes.Structure):
         ("frontier_tok", _vp), ("frontier_score", _vp), ("frontier_pool_idx", _vp), ("frontier_src_row", _vp),
         ("topk_tok", _vp), ("topk_logp", _vp), ("gate_logits", _vp), ("cont", _vp),
         ("workspace", _vp), ("workspace_bytes", _sz),
-        ("policy", _c_int), ("feat_dim", _c_int), ("features", _vp),
+        ("policy", _c_int), ("feat_dim", _c_int), ("features", _vp), ("phase", _c_int),
     ]
 
 
@@ -239,7 +240,8 @@ def radar_expand_step(ctx: Context, *, B, F, V, k, t, t_max, logits, logits_row_
                       logits_offset_elems=0, parent_score, parent_pool_idx, active, force_calls=None, gate,
                       h, c, pool_capacity, pool_tok, pool_parent, pool_depth, pool_draft_row, pool_score, pool_len,
                       frontier_tok, frontier_score, frontier_pool_idx, frontier_src_row, topk_tok, topk_logp,
-                      gate_logits, cont, workspace, stream=None, policy=RADAR_POLICY_LSTM_SCORES, features=None):
+                      gate_logits, cont, workspace, stream=None, policy=RADAR_POLICY_LSTM_SCORES, features=None,
+                      phase=RADAR_EXPAND_ALL):
     """One draft call's expansion.  `logits` is a CUDA tensor; the rows of this call start
     `logits_offset_elems` elements into it.  `gate` is a dict of the weight tensors (all eight for the
     LSTM policies; w1, b1, w2, b2 for RADAR_POLICY_MLP_SCORES); `features` [B, feat_dim] float32 is the
@@ -254,7 +256,7 @@ def radar_expand_step(ctx: Context, *, B, F, V, k, t, t_max, logits, logits_row_
     a.active, a.force_calls = _ptr(active, u8), _ptr(force_calls, i32)
     for n in ("w_ih", "w_hh", "b_ih", "b_hh", "w1", "b1", "w2", "b2"):
         setattr(a, n, _ptr(gate.get(n), f32))
-    a.policy = policy
+    a.policy, a.phase = policy, phase
     if features is not None:
         a.features, a.feat_dim = _ptr(features, f32), features.shape[-1]
     a.h, a.c = _ptr(h, f32), _ptr(c, f32)

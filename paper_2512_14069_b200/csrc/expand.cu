@@ -20,6 +20,8 @@ struct SelectParams {
     VocabPassParams vp;
     int* status;
     int staged;                                      // 1: the block's chunk records fit the staging area
+    int split;                                       // 1: launched on its own (RADAR_EXPAND_SELECT): the stream predecessor
+                                                     //    is not this call's vocabulary pass, so nothing is read before the wait
     const float* feat_pre;                           // hidden-state policy: [B][4H] W_ih f and [B][H] W_1[:, H:] f,
     const float* feat_hid;                           // written by gate_features_kernel
 };
@@ -97,6 +99,7 @@ __global__ void __launch_bounds__(kSelThreads, 1) expand_select_gate_kernel(cons
     // the previous call's state (active, h, c, pool_len) is complete when this block starts.  Only
     // the chunk records need the pass itself, so the gate warps never wait for it.
     chain_trigger();
+    if (P.split) chain_sync();                         // the predecessor may be the previous call's select + gate block
     const radar_expand_args& a = P.a;
     const int b = blockIdx.x;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -435,7 +438,8 @@ extern "C" int radar_expand_step(radar_ctx* ctx, const radar_expand_args* a, voi
     if (a->k > RADAR_MAX_K || a->F > kMaxF || a->V < a->k) return RADAR_ERR_UNSUPPORTED;
     if (a->logits_dtype != RADAR_F32 && a->logits_dtype != RADAR_BF16) return RADAR_ERR_UNSUPPORTED;
     if (a->logits_row_stride < a->V) return RADAR_ERR_INVALID_ARG;
-    if (!a->logits || !a->parent_score || !a->parent_pool_idx || !a->active || !a->h || !a->c || !a->pool_tok ||
+    if (a->phase != RADAR_EXPAND_ALL && a->phase != RADAR_EXPAND_VOCAB && a->phase != RADAR_EXPAND_SELECT) return RADAR_ERR_INVALID_ARG;
+    if (!a->logits || !a->parent_score || !a->parent_pool_idx || (!a->active && a->phase != RADAR_EXPAND_VOCAB) || !a->h || !a->c || !a->pool_tok ||
         !a->pool_parent || !a->pool_depth || !a->pool_draft_row || !a->pool_score || !a->pool_len ||
         !a->frontier_tok || !a->frontier_score || !a->frontier_pool_idx || !a->frontier_src_row || !a->topk_tok ||
         !a->topk_logp || !a->gate_logits || !a->cont || !a->workspace)
@@ -470,7 +474,7 @@ extern "C" int radar_expand_step(radar_ctx* ctx, const radar_expand_args* a, voi
     vp.k = a->k;
     vp.n_chunks = vocab_pass_plan_chunks(ctx->sm_count, a->B * a->F, a->V, &vp.chunk);
     vp.want_lse = 1;
-    vp.seq_active = a->t > 1 ? a->active : nullptr;
+    vp.seq_active = a->t > 1 ? a->active : nullptr;          // RADAR_EXPAND_VOCAB: the caller's (possibly older) mask, or NULL
     vp.seq_rows = nullptr;
     vp.status = ctx->d_status;
     const size_t part_bytes = align_up(vocab_pass_partial_bytes(a->B * a->F, vp.n_chunks, a->k), 256);
@@ -479,14 +483,16 @@ extern "C" int radar_expand_step(radar_ctx* ctx, const radar_expand_args* a, voi
     float* feat_pre = reinterpret_cast<float*>(reinterpret_cast<char*>(a->workspace) + part_bytes);
     sp.feat_pre = feat_pre;
     sp.feat_hid = feat_pre + (size_t)a->B * 4 * kHidden;
-    if (gate_runs && a->policy == RADAR_POLICY_LSTM_HIDDEN) {
+    if (gate_runs && a->policy == RADAR_POLICY_LSTM_HIDDEN && a->phase != RADAR_EXPAND_SELECT) {
         radar_launch_scope scope(ctx, RADAR_K_GATE_FEATURES, stream);
         const int nseg = (a->feat_dim + kFeatSeg - 1) / kFeatSeg;
         RADAR_CUDA_CHECK(launch_chained(gate_features_kernel, dim3(5 * kHidden), dim3(nseg * 32), 0, stream, *a, feat_pre,
                                         feat_pre + (size_t)a->B * 4 * kHidden));
     }
 
-    RADAR_CUDA_CHECK(vocab_pass_launch(ctx, RADAR_K_VOCAB_EXPAND, vp, stream));
+    if (a->phase != RADAR_EXPAND_SELECT) RADAR_CUDA_CHECK(vocab_pass_launch(ctx, RADAR_K_VOCAB_EXPAND, vp, stream));
+    if (a->phase == RADAR_EXPAND_VOCAB) return RADAR_OK;
+    sp.split = a->phase == RADAR_EXPAND_SELECT ? 1 : 0;
     // The chunk records are staged in shared memory only if they fit next to the survivor lists and the gate
     // weights inside the 227 KB a block may have; otherwise the merge reads them from global memory.
     const size_t stage_bytes = (size_t)a->F * vp.n_chunks * a->k * 8;

@@ -4,7 +4,11 @@
 acceptance output, workspaces) and issues the library calls in order on the current
 stream: t_max expansion calls (sequences the prediction model has stopped are skipped on
 the device, so no decision ever returns to the host), rerank + tree build, tree
-attention, acceptance.  It contains no arithmetic of the method.
+attention, acceptance.  The expansion calls are issued as two overlapping chains: the
+bandwidth-bound vocabulary passes run ahead on a side stream while the latency-bound
+select + gate blocks follow on the main stream (the pass of call t+1 skips the sequences
+that had stopped before call t; one that stops at call t is read once in vain).
+It contains no arithmetic of the method.
 """
 from __future__ import annotations
 
@@ -58,17 +62,21 @@ class SpecStep:
         # workspaces
         wb = max(rb.radar_expand_workspace_bytes(ctx, B, 1, V, k), rb.radar_expand_workspace_bytes(ctx, B, k, V, k))
         self.ws_expand = z((wb + 255,), u8)
+        self.ws_expand2 = z((wb + 255,), u8)          # consecutive calls alternate, so a pass can run ahead of the select
         self.ws_attn = z((rb.radar_attn_workspace_bytes(ctx, B, Hq, Hkv, d, rb.dtype_code(self.O), max_prefix_len) + 255,), u8)
         self.ws_accept = z((rb.radar_accept_workspace_bytes(ctx, B, V, mode) + 255,), u8)
-        for n in ("ws_expand", "ws_attn", "ws_accept"):
+        self.side = torch.cuda.Stream(dev)            # the vocabulary passes of the pipelined expansion
+        for n in ("ws_expand", "ws_expand2", "ws_attn", "ws_accept"):
             t = getattr(self, n)
             off = (-t.data_ptr()) % 256
             setattr(self, n, t[off:off + t.numel() - 255])
 
     # ---- expansion -------------------------------------------------------------------
-    def expand(self, t, draft_logits, gate, force_calls=None, policy=rb.RADAR_POLICY_LSTM_SCORES, features=None):
+    def expand(self, t, draft_logits, gate, force_calls=None, policy=rb.RADAR_POLICY_LSTM_SCORES, features=None,
+               phase=rb.RADAR_EXPAND_ALL, vocab_mask=None, workspace=None, stream=None):
         """Draft call t (1-based) on draft_logits [B,R,V]: row 0 for t = 1, rows 1+(t-2)k.. for t >= 2.
-        `features` [t_max-1, B, feat_dim] feeds the hidden-state policy (row t-1 at call t)."""
+        `features` [t_max-1, B, feat_dim] feeds the hidden-state policy (row t-1 at call t).  `phase`, `vocab_mask`
+        (the mask a RADAR_EXPAND_VOCAB call reads rows by), `workspace` and `stream` serve the pipelined form."""
         k, B, V = self.k, self.B, self.V
         F = 1 if t == 1 else k
         row0 = 0 if t == 1 else 1 + (t - 2) * k
@@ -78,19 +86,43 @@ class SpecStep:
             logits_row_stride=V, logits_seq_stride=self.R * V, logits_offset_elems=row0 * V,
             parent_score=self.root_score if t == 1 else self.frontier_score[s - 1],
             parent_pool_idx=self.root_pool_idx if t == 1 else self.frontier_pool_idx[s - 1],
-            active=self.active, force_calls=force_calls, gate=gate, h=self.h, c=self.c,
+            active=vocab_mask if phase == rb.RADAR_EXPAND_VOCAB else self.active, force_calls=force_calls, gate=gate, h=self.h, c=self.c,
             pool_capacity=self.C, pool_tok=self.pool_tok, pool_parent=self.pool_parent, pool_depth=self.pool_depth,
             pool_draft_row=self.pool_draft_row, pool_score=self.pool_score, pool_len=self.pool_len,
             frontier_tok=self.frontier_tok[s], frontier_score=self.frontier_score[s],
             frontier_pool_idx=self.frontier_pool_idx[s], frontier_src_row=self.frontier_src_row[s],
             topk_tok=self.topk_tok1 if t == 1 else self.topk_tok[s],
             topk_logp=self.topk_logp1 if t == 1 else self.topk_logp[s],
-            gate_logits=self.gate_logits[s], cont=self.cont_hist[s], workspace=self.ws_expand, policy=policy,
-            features=None if features is None or t >= self.t_max else features[s])
+            gate_logits=self.gate_logits[s], cont=self.cont_hist[s], workspace=self.ws_expand if workspace is None else workspace,
+            policy=policy, features=None if features is None or t >= self.t_max else features[s], phase=phase, stream=stream)
 
-    def run_expansion(self, draft_logits, gate, force_calls=None, policy=rb.RADAR_POLICY_LSTM_SCORES, features=None):
-        for t in range(1, self.t_max + 1):          # call 1 restarts the state on the device
-            self.expand(t, draft_logits, gate, force_calls, policy, features)
+    def run_expansion(self, draft_logits, gate, force_calls=None, policy=rb.RADAR_POLICY_LSTM_SCORES, features=None,
+                      pipelined=True):
+        if not pipelined:
+            for t in range(1, self.t_max + 1):      # call 1 restarts the state on the device
+                self.expand(t, draft_logits, gate, force_calls, policy, features)
+            return
+        # Two chains.  The vocabulary pass of call t (side stream, workspace t % 2) needs the select + gate block
+        # of call t - 2 done: that block wrote the mask the pass skips rows by (cont of call t - 2; nothing for
+        # t <= 2) and was the last reader of the same workspace.  The select + gate block of call t (main stream)
+        # needs its pass and the block of call t - 1, which precedes it on the stream.
+        main, side = torch.cuda.current_stream(), self.side
+        ws = (self.ws_expand, self.ws_expand2)
+        args = (draft_logits, gate, force_calls, policy, features)
+        side.wait_stream(main)                      # fork: whatever produced the inputs is done
+        sel_done = {}
+        for t in range(1, self.t_max + 1):
+            if t - 2 in sel_done:
+                side.wait_event(sel_done[t - 2])
+            mask = self.cont_hist[t - 3] if t >= 3 else None
+            self.expand(t, *args, phase=rb.RADAR_EXPAND_VOCAB, vocab_mask=mask, workspace=ws[t % 2], stream=side)
+            voc = torch.cuda.Event()
+            voc.record(side)
+            main.wait_event(voc)
+            self.expand(t, *args, phase=rb.RADAR_EXPAND_SELECT, workspace=ws[t % 2], stream=main)
+            sel_done[t] = torch.cuda.Event()
+            sel_done[t].record(main)
+        main.wait_stream(side)                      # join (the last pass has been waited for already)
 
     # ---- tree, attention, acceptance ------------------------------------------------------
     def build_tree(self, root_tok, prefix_len, n_keep=None):
