@@ -518,3 +518,42 @@ def test_attention_several_layers_in_one_call(ctx, kind):
     # rows past a tree's end stay untouched in every layer
     for b in range(base.B):
         assert not O_gpu[:, b, trees[b]["n_nodes"]:].any()
+
+
+@pytest.mark.parametrize("Hq,Hkv,P", [(8, 2, (6000, 9000)), (4, 4, (5000, 7000)), (16, 2, (9000, 14000))])
+def test_attention_scores_far_above_the_running_maximum(ctx, Hq, Hkv, P):
+    """Keys that score 100 to 300 doublings above everything their row has seen before, one in almost every tile
+    (each aimed at another query row, at varying places of the tile), plus: both column halves of one tile for
+    one row, the same row in consecutive tiles with growing size, the last prefix key and the tree tile.  The
+    kernel's one-pass tiles cannot take them with the reference maximum the row has; the group has to settle a
+    new one and finish the tile.  Long prefixes, so that a CTA runs several tiles of a unit; units with two live
+    row blocks and with one."""
+    cfg = W.shrink(W.CONFIGS[5], cid=140 + Hq, B=3, Hq=Hq, Hkv=Hkv, d=128, P=P, V=2000, k=4, t_max=5, N=50)
+    inp = H.make_inputs(cfg)
+    _, _, trees = H.oracle_expand_and_tree(cfg, inp)
+    G = Hq // Hkv
+
+    def plant(b, key, node, head, alpha, tree=False):
+        q = W.bf16_bits_to_f32(inp["Q"][b][node, head])
+        dst = inp["Kt"][b] if tree else inp["Kc"][b]
+        dst[key, head // G] = W.f32_to_bf16_bits(alpha * q)
+
+    for b in range(cfg.B):
+        Pb, n = int(inp["prefix_len"][b]), trees[b]["n_nodes"]
+        assert Pb >= 5000 and n >= 4
+        for t in range(1, Pb // 128):
+            if t % 7 == 3:
+                continue                                       # some tiles stay ordinary
+            plant(b, t * 128 + (37 * t + 5 * b) % 128, t % n, (3 * t + b) % Hq, 8.0 + t % 3)
+        plant(b, 10 * 128 + 10, 3, 1, 14.0)                    # both halves of one tile, one row
+        plant(b, 10 * 128 + 70, 3, 1, 19.0)
+        plant(b, 11 * 128 + 40, 3, 1, 25.0)                    # and the same row again in the next tile
+        plant(b, Pb - 1, 0, Hq // 2, 16.0)                     # the last prefix key
+        plant(b, 0, n - 1, 0, 30.0, tree=True)                 # the root's key in the tree tile: every row sees it
+    g = H.CudaRun(cfg, inp, ctx)
+    g.upload_attention()
+    O_gpu, lse_gpu = g.attention(trees)
+    assert ctx.read_device_status() == 0
+    O_ref, lse_ref = H.oracle_attention(cfg, inp, trees)
+    assert float(np.max(lse_ref)) > 100.0                      # the planted keys do dominate their rows
+    H.compare_attention(cfg, O_gpu, lse_gpu, O_ref, lse_ref, trees)
