@@ -363,6 +363,57 @@ int radar_accept_length_distribution(radar_ctx* ctx, const radar_acclen_args* ar
 size_t radar_noalloc_scratch_bytes(void);
 int radar_verify_accept_greedy_noalloc(radar_ctx* ctx, const radar_accept_args* args, void* stream);
 
+/* ------------------------------------------------------------------------------------------
+ * radar_policy_train_step - one REINFORCE step of the prediction model on a batch of data points {S, D}.
+ * (Sec. 4.2: the MDP of Eq. 3-9 and the loss of Eq. 10; Sec. 4.3: the data point x = {S, D}, the acceptance
+ * length drawn from d_T; App. "Implementation Details": the network, learning rate 1e-4, batches of 256.  The
+ * optimiser is not named there: Adam is used.)
+ *
+ * For data point j: the prediction model of radar_expand_step (LSTM + MLP, the RADAR_POLICY_LSTM_SCORES
+ * network) is rolled out over the states s_t = exp(log_states[t-1][j][:]), t = 1, 2, ...; after draft call t
+ * it CONTINUES iff u_action[j][t-1] < pi(continue | s_1..s_t) (softmax of the two logits), else stops: T = t.
+ * A trajectory that reaches t_max ends there without a decision (T = t_max, t_max - 1 decisions).  The
+ * acceptance length l_acc is the smallest i with p_0 + .. + p_i > u_length[j] * total over d_T =
+ * dists[T-1][j][:] (the last i with mass if none).  Rewards (Eq. 6): r_t = -alpha for t < T,
+ * r_T = l_acc / T_gen(T), T_gen(t) = T_o + T_d t + T_p (t + 1 if t < t_max else t) (Eq. 7-8).  The decision
+ * after call t collects G_t = sum_{t' = t..T} gamma^(t' - t) r_t' (Eq. 9-10).  Loss = mean over j of
+ * - sum_t G_t log pi(a_t | .); its gradient by backpropagation through time (actions and l_acc are constants
+ * of the gradient); no baseline, no dropout.  With step >= 1 the parameters then take one Adam update
+ * (bias-corrected, no weight decay): m, v and theta are updated in place; step == 0 leaves them alone.
+ *
+ * Layouts (all device): log_states [t_max][n][k] fp32 = the frontier_score buffers of t_max draft calls;
+ * dists [t_max][n][t_max+1] fp64, slice i-1 = what radar_accept_length_distribution wrote for the trees of
+ * i draft calls; theta / adam_m / adam_v / grad [radar_policy_param_count(k)] fp32 in the order
+ * w_ih [4H][k] | w_hh [4H][H] | b_ih [4H] | b_hh [4H] | w1 [H][H+k] | b1 [H] | w2 [2][H] | b2 [2]
+ * (every tensor starts 16-byte aligned when theta is, so radar_expand_step can be pointed into it).
+ * Outputs: grad, loss [1], calls [n] (T), l_acc [n], actions [n][t_max] (0 / 1, 255 where no decision was taken).
+ * Limits: 1 <= k <= RADAR_MAX_K, 2 <= t_max <= 16, n >= 1; theta and the workspace 16-byte aligned.
+ * Workspace: radar_train_workspace_bytes. */
+typedef struct {
+    int n, k, t_max;
+    const float* log_states;
+    const double* dists;
+    const float* u_action;              /* [n][t_max] uniforms in [0,1) */
+    const float* u_length;              /* [n] */
+    float alpha, gamma, T_o, T_d, T_p;
+    float lr, beta1, beta2, eps;
+    int step;                           /* Adam step counted from 1; 0: loss and gradient only */
+    float* theta;
+    float* adam_m;
+    float* adam_v;
+    float* grad;
+    float* loss;
+    int32_t* calls;
+    int32_t* l_acc;
+    uint8_t* actions;
+    void* workspace;
+    size_t workspace_bytes;
+} radar_train_args;
+
+size_t radar_policy_param_count(int k);
+size_t radar_train_workspace_bytes(const radar_ctx* ctx, int n, int k, int t_max);
+int radar_policy_train_step(radar_ctx* ctx, const radar_train_args* args, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -87,6 +87,18 @@ class AccLenArgs(ctypes.Structure):
     ]
 
 
+class TrainArgs(ctypes.Structure):
+    _fields_ = [
+        ("n", _c_int), ("k", _c_int), ("t_max", _c_int),
+        ("log_states", _vp), ("dists", _vp), ("u_action", _vp), ("u_length", _vp),
+        ("alpha", _c_f), ("gamma", _c_f), ("T_o", _c_f), ("T_d", _c_f), ("T_p", _c_f),
+        ("lr", _c_f), ("beta1", _c_f), ("beta2", _c_f), ("eps", _c_f), ("step", _c_int),
+        ("theta", _vp), ("adam_m", _vp), ("adam_v", _vp), ("grad", _vp), ("loss", _vp),
+        ("calls", _vp), ("l_acc", _vp), ("actions", _vp),
+        ("workspace", _vp), ("workspace_bytes", _sz),
+    ]
+
+
 _lib = None
 
 
@@ -371,6 +383,42 @@ def radar_accept_length_distribution(ctx: Context, *, B, V, t_max, temperature, 
     a.workspace, a.workspace_bytes = _ptr(workspace), workspace.numel() * workspace.element_size()
     _check("radar_accept_length_distribution",
            lib().radar_accept_length_distribution(ctx.handle, ctypes.byref(a), _stream(stream)))
+
+
+def radar_policy_param_count(k: int) -> int:
+    L = lib()
+    L.radar_policy_param_count.restype = _sz
+    L.radar_policy_param_count.argtypes = [_c_int]
+    return int(L.radar_policy_param_count(k))
+
+
+def radar_train_workspace_bytes(ctx: Context, n: int, k: int, t_max: int) -> int:
+    L = lib()
+    L.radar_train_workspace_bytes.restype = _sz
+    L.radar_train_workspace_bytes.argtypes = [_vp, _c_int, _c_int, _c_int]
+    return int(L.radar_train_workspace_bytes(ctx.handle, n, k, t_max))
+
+
+def radar_policy_train_step(ctx: Context, *, n, k, t_max, log_states, dists, u_action, u_length, alpha, gamma, T_o, T_d,
+                            T_p, theta, grad, loss, calls, l_acc, actions, workspace, step=0, lr=1e-4, beta1=0.9,
+                            beta2=0.999, eps=1e-8, adam_m=None, adam_v=None, stream=None):
+    """One REINFORCE step of the prediction model on n data points {S, D}; see include/radar.h for layouts."""
+    f32, f64, i32, u8 = torch.float32, torch.float64, torch.int32, torch.uint8
+    L = lib()
+    L.radar_policy_train_step.restype = _c_int
+    L.radar_policy_train_step.argtypes = [_vp, ctypes.POINTER(TrainArgs), _vp]
+    a = TrainArgs()
+    a.n, a.k, a.t_max = n, k, t_max
+    a.log_states, a.dists = _ptr(log_states, f32), _ptr(dists, f64)
+    a.u_action, a.u_length = _ptr(u_action, f32), _ptr(u_length, f32)
+    a.alpha, a.gamma, a.T_o, a.T_d, a.T_p = alpha, gamma, T_o, T_d, T_p
+    a.lr, a.beta1, a.beta2, a.eps, a.step = lr, beta1, beta2, eps, step
+    a.theta, a.grad, a.loss = _ptr(theta, f32), _ptr(grad, f32), _ptr(loss, f32)
+    a.adam_m = _ptr(adam_m, f32) if adam_m is not None else None
+    a.adam_v = _ptr(adam_v, f32) if adam_v is not None else None
+    a.calls, a.l_acc, a.actions = _ptr(calls, i32), _ptr(l_acc, i32), _ptr(actions, u8)
+    a.workspace, a.workspace_bytes = _ptr(workspace), workspace.numel() * workspace.element_size()
+    _check("radar_policy_train_step", L.radar_policy_train_step(ctx.handle, ctypes.byref(a), _stream(stream)))
 
 
 def radar_noalloc_scratch_bytes() -> int:

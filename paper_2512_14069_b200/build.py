@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libradar_b200.so")
-SOURCES = ["api.cu", "vocab_pass.cu", "expand.cu", "tree_build.cu", "tree_attention.cu", "tree_attention_tc.cu", "verify_accept.cu"]
+SOURCES = ["api.cu", "vocab_pass.cu", "expand.cu", "tree_build.cu", "tree_attention.cu", "tree_attention_tc.cu", "verify_accept.cu", "train.cu"]
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",
          "-Xcompiler", "-fPIC", "--expt-relaxed-constexpr"]
 

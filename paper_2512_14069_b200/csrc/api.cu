@@ -96,6 +96,9 @@ extern "C" const char* radar_kernel_name(int id) {
         case RADAR_K_ACCLEN_NODES: return "accept_length_nodes";
         case RADAR_K_ACCLEN_DIST: return "accept_length_dist";
         case RADAR_K_GATE_FEATURES: return "gate_features";
+        case RADAR_K_TRAIN_ROLLOUT: return "train_rollout";
+        case RADAR_K_TRAIN_OUTER: return "train_outer";
+        case RADAR_K_TRAIN_ADAM: return "train_adam";
         default: return "?";
     }
 }

@@ -22,6 +22,9 @@ enum radar_kernel_id {
     RADAR_K_ACCLEN_NODES,       // per-row conditional acceptance probabilities (Eq. 13)
     RADAR_K_ACCLEN_DIST,        // path products and the length distribution (Eq. 11-12)
     RADAR_K_GATE_FEATURES,      // input-side products of the hidden-state policy (Table 3)
+    RADAR_K_TRAIN_ROLLOUT,      // REINFORCE step: rollout + backpropagation through time per data point
+    RADAR_K_TRAIN_OUTER,        // REINFORCE step: parameter gradients
+    RADAR_K_TRAIN_ADAM,         // REINFORCE step: batch loss + Adam update
     RADAR_K_COUNT
 };
 

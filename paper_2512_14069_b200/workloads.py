@@ -21,7 +21,7 @@ GATE_HIDDEN = 128
 
 # tensor ids (second word of every stream key)
 T_DRAFT, T_TARGET_NOISE, T_GATE, T_Q, T_KC, T_VC, T_KT, T_VT, T_UACC, T_USAMP, T_PLEN, T_DEPTH, \
-    T_NKEEP, T_PEAK, T_TARGET_FRESH, T_ROOT, T_POLICY, T_FEATURES = range(18)
+    T_NKEEP, T_PEAK, T_TARGET_FRESH, T_ROOT, T_POLICY, T_FEATURES, T_TRAIN = range(19)
 
 
 @dataclass(frozen=True)
@@ -239,3 +239,24 @@ def accept_uniforms(cfg: Config):
     ua = stream(cfg, T_UACC).random((cfg.B, M_MAX), dtype=np.float32)
     us = stream(cfg, T_USAMP).random(cfg.B, dtype=np.float32)
     return ua, us
+
+
+# ---- synthetic training data for the prediction model (Sec. 4.3: data points {S, D}) -------------
+def train_batch(cfg: Config, n: int, seed: int = 0):
+    """n synthetic data points.  log_states [t_max][n][k] float32: logs of k descending confidence scores per
+    draft call, shrinking with depth like cumulative path probabilities; dists [t_max][n][t_max+1] float64:
+    random distributions whose mass moves to longer acceptance lengths as the number of calls grows, with
+    p_j = 0 for j > i (a tree of i calls cannot accept more than i tokens); uniforms u_action [n][t_max],
+    u_length [n] float32.  Holds no arithmetic of the method: the rows only have the paper's shapes."""
+    g = stream(cfg, T_TRAIN, seed)
+    k, t_max = cfg.k, cfg.t_max
+    base = np.sort(g.uniform(0.02, 1.0, size=(t_max, n, k)), axis=2)[:, :, ::-1]
+    decay = np.cumprod(g.uniform(0.5, 1.0, size=(t_max, n, 1)), axis=0)
+    log_states = np.log(base * decay).astype(np.float32)
+    dists = np.zeros((t_max, n, t_max + 1), np.float64)
+    for i in range(1, t_max + 1):
+        w = g.gamma(1.0, size=(n, i + 1))
+        dists[i - 1, :, : i + 1] = w / w.sum(axis=1, keepdims=True)
+    u_action = g.random((n, t_max), dtype=np.float32)
+    u_length = g.random(n, dtype=np.float32)
+    return log_states, dists, u_action, u_length

@@ -38,7 +38,8 @@ def test_library_builds_and_exports_every_declared_symbol():
 def test_python_structs_match_the_header_layout(tmp_path):
     """Compile a C program that prints sizeof/offsetof of every field and compare with ctypes."""
     structs = {"radar_expand_args": rb.ExpandArgs, "radar_tree_args": rb.TreeArgs,
-               "radar_attn_args": rb.AttnArgs, "radar_accept_args": rb.AcceptArgs, "radar_acclen_args": rb.AccLenArgs}
+               "radar_attn_args": rb.AttnArgs, "radar_accept_args": rb.AcceptArgs, "radar_acclen_args": rb.AccLenArgs,
+               "radar_train_args": rb.TrainArgs}
     lines = ['#include <stdio.h>', '#include <stddef.h>', '#include "radar.h"', "int main(void){"]
     for cname, st in structs.items():
         lines.append('printf("%s %%zu\\n", sizeof(%s));' % (cname, cname))
