@@ -666,8 +666,8 @@ def _single_thread():
 
 def next_rows_probe(ctx, dev, reps=10):
     """Device times of the kernels beyond the step itself: the acceptance-length distribution (Eq. 11-13) on the
-    trees of the Vicuna-13B configuration, and the
-    input-side kernel of the hidden-state policy at the draft model's width."""
+    trees of the Vicuna-13B configuration, the input-side kernel of the hidden-state policy at the draft model's
+    width, and one REINFORCE step of the prediction model (Eq. 10) on a batch of 256."""
     import torch
     from paper_2512_14069_b200 import binding as rb
     from paper_2512_14069_b200.pipeline import SpecStep
@@ -706,15 +706,38 @@ def next_rows_probe(ctx, dev, reps=10):
     force4 = torch.full((cfg4.B,), cfg4.t_max, dtype=torch.int32, device=dev)
     step4.expand(1, draft4, w_hid, force4, rb.RADAR_POLICY_LSTM_HIDDEN, feats)
 
+    # one REINFORCE step of the prediction model on a batch of 256 synthetic data points (k = 10, t_max = 8)
+    cfg2 = W.CONFIGS[2]
+    n_tr = 256
+    tb = [torch.from_numpy(x).to(dev) for x in W.train_batch(cfg2, n_tr, 0)]
+    Pn = rb.radar_policy_param_count(cfg2.k)
+    theta = torch.cat([torch.from_numpy(v.reshape(-1)) for v in W.gate_weights(cfg2).values()]).to(dev)
+    assert theta.numel() == Pn
+    t_m, t_v, t_g = (torch.zeros(Pn, device=dev) for _ in range(3))
+    t_loss = torch.zeros(1, device=dev)
+    t_calls, t_len = torch.zeros(n_tr, dtype=torch.int32, device=dev), torch.zeros(n_tr, dtype=torch.int32, device=dev)
+    t_act = torch.zeros((n_tr, cfg2.t_max), dtype=torch.uint8, device=dev)
+    t_ws = torch.zeros(rb.radar_train_workspace_bytes(ctx, n_tr, cfg2.k, cfg2.t_max), dtype=torch.uint8, device=dev)
+    train_it = [0]
+
+    def run_train():
+        train_it[0] += 1
+        rb.radar_policy_train_step(
+            ctx, n=n_tr, k=cfg2.k, t_max=cfg2.t_max, log_states=tb[0], dists=tb[1], u_action=tb[2], u_length=tb[3],
+            alpha=0.05, gamma=0.99, T_o=68.0, T_d=2.7, T_p=0.4, theta=theta, grad=t_g, loss=t_loss, calls=t_calls,
+            l_acc=t_len, actions=t_act, workspace=t_ws, step=train_it[0], lr=1e-4, adam_m=t_m, adam_v=t_v)
+
     run_acclen()
+    run_train()
     torch.cuda.synchronize()
-    ctx.profile_begin(reps * 6)
+    ctx.profile_begin(reps * 10)
     torch.cuda._sleep(8_000_000)
     for _ in range(reps):
         run_acclen()
         step4.active.fill_(1)
         step4.pool_len.fill_(cfg4.k)
         step4.expand(2, draft4, w_hid, force4, rb.RADAR_POLICY_LSTM_HIDDEN, feats)
+        run_train()
     torch.cuda.synchronize()
     ctx.profile_end()
     ctx.check_device_status()
@@ -727,6 +750,10 @@ def next_rows_probe(ctx, dev, reps=10):
         "hidden_state_policy": {
             "workload": "8 sequences, feature width 4096: 640 x 4096 fp32 weights read once",
             "gate_features_us": round(ks.get("gate_features", 0.0), 1), "select_gate_us": round(ks.get("expand_select_gate", 0.0), 1)},
+        "reinforce_step": {
+            "workload": "256 synthetic data points {S, D}, k = 10, t_max = 8, mean draft calls %.2f" % float(t_calls.float().mean()),
+            "rollout_bptt_us": round(ks.get("train_rollout", 0.0), 1), "param_gradients_us": round(ks.get("train_outer", 0.0), 1),
+            "loss_adam_us": round(ks.get("train_adam", 0.0), 1), "loss": float(t_loss)},
     }
 
 

@@ -142,3 +142,52 @@ def test_train_step_argument_errors(ctx):
                                    theta=tr.theta, grad=tr.grad, loss=tr.loss, calls=tr.calls, l_acc=tr.l_acc,
                                    actions=tr.actions, workspace=tr.ws, step=1, **HP)
     assert e.value.status == -1
+
+
+def test_dataset_from_the_library_then_a_train_step(ctx):
+    """The offline data set of Sec. 4.3 built by the library itself, on device buffers end to end: for every number
+    of draft calls i the expansion is forced to i calls, the tree is built and Eq. 11-13 gives d_i, written straight
+    into slice i - 1 of `dists`; the states are the frontier scores of the t_max-call run.  Both are checked against
+    the oracle, then one REINFORCE step runs on them and is compared with the training oracle."""
+    import torch
+    from oracle import accept_oracle as A
+    from oracle import train_oracle as T
+    from paper_2512_14069_b200 import binding as rb
+    cfg = W.shrink(W.CONFIGS[3], cid=330, B=6, V=3001, P=(64, 64), Hq=4, Hkv=4, t_max=5, N=24)
+    k, t_max, n = cfg.k, cfg.t_max, cfg.B
+    inp = H.make_inputs(cfg, with_attention=False)
+    g = H.CudaRun(cfg, inp, ctx)
+    s = g.step
+    dists = torch.zeros((t_max, n, t_max + 1), dtype=torch.float64, device="cuda")
+    pacc = torch.zeros((n, 64), dtype=torch.float64, device="cuda")
+    wb = rb.radar_acclen_workspace_bytes(ctx, n, cfg.V)
+    ws = torch.zeros(wb + 256, dtype=torch.uint8, device="cuda")
+    off = (-ws.data_ptr()) % 256
+    d_ref = np.zeros((t_max, n, t_max + 1))
+    for i in range(1, t_max + 1):
+        inp["force_calls"] = np.full(n, i, np.int32)
+        g.force = H.to_dev(inp["force_calls"])
+        _, traces, trees = H.oracle_expand_and_tree(cfg, inp)
+        target = H.make_target(cfg, inp, trees)
+        g.expand_and_tree()
+        rb.radar_accept_length_distribution(
+            ctx, B=n, V=cfg.V, t_max=t_max, temperature=1.0, target_logits=H.to_dev(target), tree_tok=s.tree_tok,
+            tree_parent=s.tree_parent, tree_depth=s.tree_depth, tree_draft_row=s.tree_draft_row, n_nodes=s.n_nodes,
+            draft_logits=g.draft, R=s.R, dist=dists[i - 1], p_acc_node=pacc, workspace=ws[off:off + wb])
+        ctx.check_device_status()
+        for b in range(n):
+            d_ref[i - 1, b], _ = A.accept_length_distribution(target[b], inp["draft"][b], trees[b], 1.0, t_max)
+    assert np.max(np.abs(dists.cpu().numpy() - d_ref)) < 1e-9
+    assert np.all(d_ref[0, :, 2:] == 0.0)                       # one draft call cannot accept more than one token
+    log_states = s.frontier_score                               # [t_max][n][k], left by the run with t_max calls
+    ref_states = np.stack([np.stack([traces[b][t]["frontier_score"] for b in range(n)]) for t in range(t_max)])
+    assert np.max(np.abs(log_states.cpu().numpy() - ref_states)) <= 1e-5
+
+    w = dict(inp["gate"])
+    w["b2"] = w["b2"].copy()
+    w["b2"][1] += np.float32(0.5)
+    u_action, u_length = W.train_batch(cfg, n, 5)[2:]
+    loss, grad, infos = T.batch_loss_and_grad(w, log_states.cpu().numpy(), dists.cpu().numpy(), u_action, u_length, t_max, **HP)
+    tr = Trainer(ctx, n, k, t_max, _theta(w))
+    tr.step(log_states, dists, H.to_dev(u_action), H.to_dev(u_length), step=0)
+    _compare(tr, w, None, infos, loss, grad)
