@@ -13,20 +13,15 @@
 // there are several pairs per KV head, CTAs alternate between them so that they stream the same K/V
 // at the same time and all but the first read hit L2.
 //
-// Inside the CTA (18 warps):
-//   warp 16    TMA producer: per segment the Q rows, then K and V tiles into two rings (128-byte
+// Inside the CTA (10 warps):
+//   warp 8     TMA producer: per segment the Q rows, then K and V tiles into two rings (128-byte
 //              swizzle), in the order the MMA warp consumes them.
-//   warp 17    MMA issuer (the warp runs converged, one elected lane issues): S = Q K^T into one of two
-//              tensor-memory score buffers, and O (+)= P V with P read back from tensor memory (bf16,
-//              overlaying S) and V consumed N-major straight from the row-major tile.
-//   warps 0-7 / 8-15  softmax groups 0 / 1, two threads per query row (each owns one half of the 128
-//              score columns of a tile): prefix-boundary / ancestor-bit masking in registers, exp2
-//              against the row's reference maximum, P back to tensor memory, row sum.  The reference is
-//              the largest score of the segment's first tile (the two halves exchange maxima once); every
-//              later tile is one pass over the scores, and the exponentials may exceed 1.  Only a score
-//              more than 2^64 above the reference moves it: the warp that meets one leaves its chunk
-//              unwritten, the issuer wakes the group instead of running P V, the group agrees on a new
-//              reference, rescales what it has written and finishes the tile (exact for any input).
+//   warp 9     MMA issuer (one lane): S = Q K^T into one of two tensor-memory score buffers, and
+//              O (+)= P V with P read back from tensor memory (bf16, overlaying S) and V consumed
+//              N-major straight from the row-major tile.
+//   warps 0-3 / 4-7  softmax groups 0 / 1, one thread per query row: S row from tensor memory,
+//              prefix-boundary / ancestor-bit masking in registers, running max with lazy rescaling
+//              of the O accumulator, exp2, P back to tensor memory.
 //              Unit with two live row blocks: group s owns row block s and sees every tile, so each
 //              K/V tile is loaded once for 256 query rows.  Unit with one live row block: the
 //              groups take alternate tiles with separate (m, l, O) and are merged at the end.
@@ -49,7 +44,7 @@ constexpr int kStaticSmem = 3072;    // barriers and exchange arrays: with the t
 constexpr int kTileKeys = 128;       // keys per prefix tile
 constexpr int kTreeKeys = 64;        // keys of the tree tile (RADAR_MAX_NODES)
 constexpr int kPairRows = 256;       // query rows of a row-block pair (and the stride of partial records)
-constexpr float kFarAbove = 64.f;    // in log2 units: a score this far above its row's reference maximum moves the reference
+constexpr float kRescaleThreshold = 8.f;   // in log2 units: P stays below 2^8
 
 // Written by every CTA of the attention kernel, read by the combine kernel.
 struct CutUnit {
@@ -195,17 +190,15 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     // swizzled tiles need a 1024-byte boundary and there is no room left for alignment slack.
     struct __align__(1024) Static {
         uint64_t bar_qfull, bar_qempty, bar_kfull[3], bar_kempty[3], bar_vfull[3], bar_vempty[3];
-        uint64_t bar_sfull[2], bar_pready[2], bar_odone[2], bar_ofree[2], bar_fix[2];
+        uint64_t bar_sfull[2], bar_pready[2], bar_odone[2], bar_ofree[2];
         long long range[4];      // this CTA's range [lo, hi), size of the class's space (all layers), start of its first unit
         int start[3];            // sequence, KV head and layer of the unit that contains lo
         int start_pad;
         uint32_t tmem_base;
         int abort;
-        int far[2];              // per group: a warp met a score far above its row's reference and left its tile unfinished
-        int redo[2];             // per group, set by the issuing warp only: this wake-up asks for that tile to be finished
         float xm[128];           // group 1's running max at the end of a segment (one live row block)
         float mx[2][2][128];     // per group and column half: row maxima of a tile; row sums at the end of a segment
-        unsigned char pad[kStaticSmem - (24 * 8 + 4 * 8 + 4 * 4 + 4 + 4 + 4 * 4 + 128 * 4 + 2 * 2 * 128 * 4)];
+        unsigned char pad[kStaticSmem - (22 * 8 + 4 * 8 + 4 * 4 + 4 + 4 + 128 * 4 + 2 * 2 * 128 * 4)];
     };
     static_assert(sizeof(Static) == kStaticSmem, "static shared-memory block");
     __shared__ Static st;
@@ -224,7 +217,6 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     uint64_t (&bar_pready)[2] = st.bar_pready;
     uint64_t (&bar_odone)[2] = st.bar_odone;
     uint64_t (&bar_ofree)[2] = st.bar_ofree;
-    uint64_t (&bar_fix)[2] = st.bar_fix;
     uint32_t& s_tmem_base = st.tmem_base;
     int& s_abort = st.abort;
     float (&s_xm)[128] = st.xm;
@@ -294,9 +286,6 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             for (int i = 0; i < 2; ++i) {
                 mbar_init(&bar_sfull[i], 1); mbar_init(&bar_pready[i], 8);
                 mbar_init(&bar_odone[i], 1); mbar_init(&bar_ofree[i], 8);
-                mbar_init(&bar_fix[i], 8);
-                st.far[i] = 0;
-                st.redo[i] = 0;
             }
             fence_barrier_init();
         }
@@ -448,23 +437,6 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             uint32_t k_slot = 0, v_slot = 0;      // ring slots of the K and V tiles in use
             bool acc[2] = {false, false};         // accumulator holds a product of this segment
 
-            // A softmax warp that met a score far above its row's reference has left its part of the tile
-            // unwritten and raised the group's flag before arriving: the group is woken through the barrier it
-            // waits on next (the one of its next S, or of the finished accumulator after its last tile), settles
-            // a new reference, finishes the tile and arrives again.  The group tells such a wake-up from an
-            // ordinary one by a word that only this warp sets: the flag itself may already be up again, raised
-            // by a quick warp for the next tile, when a slow warp of the group looks.
-            auto unfinished = [&](const int q, const bool last) {
-                while (ok && *(volatile int*)&st.far[q] != 0) {
-                    if (elected) {
-                        *(volatile int*)&st.redo[q] = 1;
-                        mbar_arrive(last ? &bar_odone[q] : &bar_sfull[q]);
-                    }
-                    __syncwarp();
-                    ok = ok && mbar_wait(&bar_pready[q], p_par[q], ab);
-                    p_par[q] ^= 1;
-                }
-            };
             // ---- O[q] (+)= P[q] V for tile i (q is a literal at every call site) ----
             auto pv = [&](const int q, const int i, const bool fresh_v, const bool release_v) {
                 const bool tree = seg_t0 + i == nt_unit - 1;
@@ -473,7 +445,6 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 const int ksteps = (valid + 15) >> 4;
                 ok = ok && mbar_wait(&bar_pready[q], p_par[q], ab);
                 p_par[q] ^= 1;
-                unfinished(q, two ? i == n - 1 : i + 2 >= n);
                 if (fresh_v) {
                     v_slot = v_next;
                     ok = ok && mbar_wait(&bar_vfull[v_slot], v_par, ab);
@@ -541,7 +512,6 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             auto pv_full = [&](const int q, const bool fresh_v, const bool release_v) {
                 wait_all(&bar_pready[q], p_par[q]);
                 p_par[q] ^= 1;
-                unfinished(q, false);
                 if (fresh_v) {
                     v_slot = v_next;
                     wait_all(&bar_vfull[v_slot], v_par);
@@ -616,7 +586,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         const uint32_t tO = tmem + 256 + grp * 128 + lane_addr;
         const uint32_t tO_other = tmem + 256 + (grp ^ 1) * 128 + lane_addr;
         constexpr int DH = D / 2;                               // accumulator columns per thread
-        uint32_t sc = 0, oc = 0, fc = 0;         // S tiles, accumulators and exchanges of fix_tile this group has waited for
+        uint32_t sc = 0, oc = 0;                 // S tiles and accumulators this group has waited for
         bool ok = true;
         for (uint32_t seg = 0; cur.valid(); cur.next(P, pp), ++seg) {
             const int b = cur.b, g = cur.g, n = cur.t1 - cur.t0;
@@ -635,243 +605,112 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             const int n_my = two ? n : (n - grp + 1) >> 1;
             float m_run = -CUDART_INF_F, l_run = 0.f;            // l_run: this thread's columns only
 
-            // Shape of the group's tile jj: tree tile or prefix tile, this thread's chunks of 32 score columns
-            // (a prefix tile has four, two per thread; the tree tile two, one per thread), live keys.
-            // Half h of a row works in columns 64 h .. 64 h + 63 of the buffer only: its scores sit there (the
-            // tree tile's second chunk is read from columns 32 .. 63 but belongs to half 1 alone) and its P goes
-            // to columns 64 h + 16 cc, so the halves never touch each other's columns and a thread overwrites
-            // only scores it has already taken into registers.
-            struct Tile { bool tree, partial; int nch, c0, valid; };
-            auto tile_of = [&](int jj) {
-                const int t = cur.t0 + (two ? jj : 2 * jj + grp);
-                Tile T;
-                T.tree = t == nt_unit - 1;
-                T.nch = T.tree ? 1 : 2;
-                T.c0 = T.tree ? half : 2 * half;
-                T.valid = T.tree ? kTreeKeys : min(kTileKeys, Pb - t * kTileKeys);
-                T.partial = T.tree || T.valid < kTileKeys;
-                return T;
-            };
-            auto allowed_bits = [&](const Tile& T, int c) -> uint32_t {     // keys of chunk c this row may attend to
-                if (T.tree) return (uint32_t)(mask_bits >> (c * 32));
-                const int lim = T.valid - c * 32;
-                return lim >= 32 ? 0xffffffffu : (lim <= 0 ? 0u : ((1u << lim) - 1u));
-            };
-            auto load_scores = [&](const Tile& T, int cc, uint32_t (&sv)[32]) {
-                tmem_ld32(tS + (T.c0 + cc) * 32, sv);
-                tmem_wait_ld();
-                if (T.partial) {
-                    const uint32_t al = allowed_bits(T, T.c0 + cc);
-#pragma unroll
-                    for (int e = 0; e < 32; ++e)
-                        if (!((al >> e) & 1u)) sv[e] = 0xff800000u;         // -inf
-                }
-            };
-            auto max32 = [&](const uint32_t (&sv)[32]) {                    // three-input maxima: half the instructions
-                float mxa[4] = {-CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F};
-#pragma unroll
-                for (int e = 0; e < 32; e += 2)
-                    mxa[(e >> 1) & 3] = max3(mxa[(e >> 1) & 3], __uint_as_float(sv[e]), __uint_as_float(sv[e + 1]));
-                return fmaxf(fmaxf(mxa[0], mxa[1]), fmaxf(mxa[2], mxa[3]));
-            };
-            // P = exp2(x) of one chunk whose x = s * scale - m sit in sv; row sum into ls; bf16 pairs to tensor memory
-            auto exp_store = [&](int cc, const uint32_t (&x)[32], float2 (&ls)[2]) {
-                uint32_t pk[16];
-#pragma unroll
-                for (int e = 0; e < 16; ++e) {
-                    const float p0 = ex2(__uint_as_float(x[2 * e])), p1 = ex2(__uint_as_float(x[2 * e + 1]));
-                    ls[e & 1] = __fadd2_rn(ls[e & 1], make_float2(p0, p1));
-                    const __nv_bfloat162 v = __floats2bfloat162_rn(p0, p1);
-                    pk[e] = *reinterpret_cast<const uint32_t*>(&v);
-                }
-                tmem_st16(tS + half * 64 + cc * 16, pk);
-            };
-            auto scale_shift = [&](uint32_t (&sv)[32], float m_use) {      // x = s * scale - m, two values per instruction
-                const float2 sc2 = make_float2(P.scale_log2, P.scale_log2), nm2 = make_float2(-m_use, -m_use);
-#pragma unroll
-                for (int e = 0; e < 16; ++e) {
-                    const float2 t = __ffma2_rn(make_float2(__uint_as_float(sv[2 * e]), __uint_as_float(sv[2 * e + 1])), sc2, nm2);
-                    sv[2 * e] = __float_as_uint(t.x);
-                    sv[2 * e + 1] = __float_as_uint(t.y);
-                }
-            };
-            auto rescale_acc = [&](float factor) {                          // this thread's half of the accumulator
-#pragma unroll 1
-                for (int c = 0; c < DH / 32; ++c) {
-                    uint32_t o[32];
-                    tmem_ld32(tO + half * DH + c * 32, o);
-                    tmem_wait_ld();
-#pragma unroll
-                    for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * factor);
-                    tmem_st32(tO + half * DH + c * 32, o);
-                }
-            };
-            auto publish = [&]() {                                          // this warp's P of a tile is in tensor memory
-                tc_fence_before_sync();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&bar_pready[grp]);
-            };
-
-            // First tile of a segment: the reference maximum m_run of a row is the largest score of that tile
-            // (the two halves of the row exchange their maxima through shared memory).
-            auto first_tile = [&](const Tile& T) {
-                float mx = -CUDART_INF_F;
-                if (ok && warp_live) {
-#pragma unroll 1
-                    for (int cc = 0; cc < T.nch; ++cc) {
-                        uint32_t sv[32];
-                        load_scores(T, cc, sv);
-                        mx = fmaxf(mx, max32(sv));
-                    }
-                }
-                s_mx[grp][half][row] = mx;
-                if (grp == 0) asm volatile("bar.sync 1, 256;" ::: "memory"); else asm volatile("bar.sync 2, 256;" ::: "memory");
-                if (ok && warp_live) {
-                    m_run = fmaxf(mx, s_mx[grp][half ^ 1][row]) * P.scale_log2;
-                    const float m_use = m_run == -CUDART_INF_F ? 0.f : m_run;
-                    float2 ls[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
-#pragma unroll 1
-                    for (int cc = 0; cc < T.nch; ++cc) {
-                        uint32_t sv[32];
-                        load_scores(T, cc, sv);
-                        scale_shift(sv, m_use);
-                        exp_store(cc, sv, ls);
-                    }
-                    l_run = (ls[0].x + ls[0].y) + (ls[1].x + ls[1].y);
-                    tmem_wait_st();
-                }
-            };
-            // Every later tile in ONE pass against the reference the row already has: the exponentials may then
-            // exceed 1, which costs nothing in fp32 / bf16 as long as they stay far from the end of the range.  A warp
-            // that meets a score more than 2^kFarAbove above the reference drops the chunk it has just computed
-            // (its scores are still in tensor memory), raises the group's flag, and the tile is finished by
-            // fix_tile below with a new reference.  The maxima are off the path of the exponentials: their vote
-            // is needed only before the chunk is written.
-            int stored = 0;              // chunks of the last tile whose P this warp has written
-            float xseen = -CUDART_INF_F; // largest x = s * scale - reference among them
-            auto next_tile = [&](const Tile& T) {
-                stored = T.nch;
-                xseen = -CUDART_INF_F;
-                if (ok && warp_live) {
-                    const float m_use = m_run == -CUDART_INF_F ? 0.f : m_run;
-                    float2 ls[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
-#pragma unroll 1
-                    for (int cc = 0; cc < T.nch; ++cc) {
-                        uint32_t sv[32];
-                        load_scores(T, cc, sv);
-                        scale_shift(sv, m_use);
-                        const float cmx = max32(sv);
-                        float2 lc[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
-                        uint32_t pk[16];
-#pragma unroll
-                        for (int e = 0; e < 16; ++e) {
-                            const float p0 = ex2(__uint_as_float(sv[2 * e])), p1 = ex2(__uint_as_float(sv[2 * e + 1]));
-                            lc[e & 1] = __fadd2_rn(lc[e & 1], make_float2(p0, p1));
-                            const __nv_bfloat162 v = __floats2bfloat162_rn(p0, p1);
-                            pk[e] = *reinterpret_cast<const uint32_t*>(&v);
-                        }
-                        if (__any_sync(kFull, cmx > kFarAbove)) { stored = cc; break; }
-                        tmem_st16(tS + half * 64 + cc * 16, pk);
-                        xseen = fmaxf(xseen, cmx);
-                        ls[0] = __fadd2_rn(ls[0], lc[0]);
-                        ls[1] = __fadd2_rn(ls[1], lc[1]);
-                    }
-                    l_run += (ls[0].x + ls[0].y) + (ls[1].x + ls[1].y);
-                    if (stored < T.nch && lane == 0) *(volatile int*)&st.far[grp] = 1;
-                    tmem_wait_st();
-                }
-            };
-            // The issuing warp has found the flag up and woken the group instead of running P V.  All rows of the
-            // group agree on a new reference (the old one plus a whole number of doublings, so that what is already
-            // in tensor memory is rescaled exactly): chunks already written are scaled, the others are computed
-            // from their scores, the accumulator and the row sum follow.
-            auto fix_tile = [&](const Tile& T) {
-                float cand = -CUDART_INF_F;
-                if (ok && warp_live) {
-                    if (stored > 0 && m_run != -CUDART_INF_F) cand = m_run + xseen;
-#pragma unroll 1
-                    for (int cc = stored; cc < T.nch; ++cc) {
-                        uint32_t sv[32];
-                        load_scores(T, cc, sv);
-                        cand = fmaxf(cand, max32(sv) * P.scale_log2);
-                    }
-                }
-                s_mx[grp][half][row] = cand;
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&bar_fix[grp]);
-                ok = __all_sync(kFull, ok && mbar_wait(&bar_fix[grp], fc & 1, ab));      // bounded, unlike a bar.sync
-                ++fc;
-                if ((warp & 7) == 0 && lane == 0) {                                      // every warp has read them
-                    *(volatile int*)&st.far[grp] = 0;
-                    *(volatile int*)&st.redo[grp] = 0;
-                }
-                if (ok && warp_live) {
-                    const float m_new = fmaxf(cand, s_mx[grp][half ^ 1][row]);           // the same in both halves
-                    float factor = 1.f;
-                    if (m_run == -CUDART_INF_F) {
-                        factor = 0.f;                                                    // nothing of weight so far
-                        m_run = m_new;
-                    } else if (m_new > m_run + kFarAbove) {
-                        const float delta = ceilf(m_new - m_run);
-                        factor = ex2(-delta);
-                        m_run += delta;
-                    }
-                    const bool any_moved = __any_sync(kFull, factor != 1.f);
-                    const float m_use = m_run == -CUDART_INF_F ? 0.f : m_run;
-                    float2 ls[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
-#pragma unroll 1
-                    for (int cc = 0; cc < T.nch; ++cc) {
-                        if (cc < stored) {
-                            if (any_moved) {
-                                uint32_t pk[16];
-                                tmem_ld16(tS + half * 64 + cc * 16, pk);
-                                tmem_wait_ld();
-#pragma unroll
-                                for (int e = 0; e < 16; ++e) {
-                                    const float p0 = __uint_as_float(pk[e] << 16) * factor;
-                                    const float p1 = __uint_as_float(pk[e] & 0xffff0000u) * factor;
-                                    const __nv_bfloat162 v = __floats2bfloat162_rn(p0, p1);
-                                    pk[e] = *reinterpret_cast<const uint32_t*>(&v);
-                                }
-                                tmem_st16(tS + half * 64 + cc * 16, pk);
-                            }
-                        } else {
-                            uint32_t sv[32];
-                            load_scores(T, cc, sv);
-                            scale_shift(sv, m_use);
-                            exp_store(cc, sv, ls);
-                        }
-                    }
-                    l_run = l_run * factor + ((ls[0].x + ls[0].y) + (ls[1].x + ls[1].y));
-                    if (any_moved) rescale_acc(factor);
-                    tmem_wait_st();
-                }
-                stored = T.nch;
-            };
-
-            for (int j = 0; j < n_my;) {
+            for (int j = 0; j < n_my; ++j) {
+                const int i = two ? j : 2 * j + grp;             // local tile index
+                const int t = cur.t0 + i;
                 ok = __all_sync(kFull, ok && mbar_wait(&bar_sfull[grp], sc & 1, ab));    // warp-uniform: guards .aligned ops
                 ++sc;
                 tc_fence_after_sync();
-                if (j > 0 && ok && *(volatile int*)&st.redo[grp] != 0) {                 // woken to finish tile j - 1
-                    fix_tile(tile_of(j - 1));
-                    publish();
-                    continue;
+                // This thread's chunks of 32 score columns: a prefix tile has four (two per thread), the tree tile
+                // two (one per thread).  Half h of a row works in columns 64 h .. 64 h + 63 of the buffer only: its
+                // scores sit there (the tree tile's second chunk is read from columns 32 .. 63 but belongs to
+                // half 1 alone) and its P goes to columns 64 h + 16 cc, so the halves never touch each other's
+                // columns and a thread overwrites only scores it has already taken into registers.
+                const bool tree = t == nt_unit - 1;
+                const int nch = tree ? 1 : 2;
+                const int c0 = tree ? half : 2 * half;
+                const int valid = tree ? kTreeKeys : min(kTileKeys, Pb - t * kTileKeys);
+                const bool partial = tree || valid < kTileKeys;
+                auto allowed_bits = [&](int c) -> uint32_t {        // keys of chunk c this row may attend to
+                    if (tree) return (uint32_t)(mask_bits >> (c * 32));
+                    const int lim = valid - c * 32;
+                    return lim >= 32 ? 0xffffffffu : (lim <= 0 ? 0u : ((1u << lim) - 1u));
+                };
+                float mx = -CUDART_INF_F;
+                if (ok && warp_live) {
+#pragma unroll 1
+                    for (int cc = 0; cc < nch; ++cc) {
+                        uint32_t sv[32];
+                        tmem_ld32(tS + (c0 + cc) * 32, sv);
+                        tmem_wait_ld();
+                        if (partial) {
+                            const uint32_t al = allowed_bits(c0 + cc);
+#pragma unroll
+                            for (int e = 0; e < 32; ++e)
+                                if (!((al >> e) & 1u)) sv[e] = 0xff800000u;     // -inf
+                        }
+                        float mxa[4] = {-CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F};
+#pragma unroll
+                        for (int e = 0; e < 32; e += 2)                     // three-input maxima: half the instructions
+                            mxa[(e >> 1) & 3] = max3(mxa[(e >> 1) & 3], __uint_as_float(sv[e]), __uint_as_float(sv[e + 1]));
+                        mx = fmaxf(mx, fmaxf(fmaxf(mxa[0], mxa[1]), fmaxf(mxa[2], mxa[3])));
+                    }
                 }
-                const Tile T = tile_of(j);
-                if (j == 0) first_tile(T); else next_tile(T);
-                publish();
-                ++j;
+                // the two halves of a row exchange their maxima
+                s_mx[grp][half][row] = mx;
+                if (grp == 0) asm volatile("bar.sync 1, 256;" ::: "memory"); else asm volatile("bar.sync 2, 256;" ::: "memory");
+                if (ok && warp_live) {
+                    mx = fmaxf(mx, s_mx[grp][half ^ 1][row]);
+                    // ---- running max (log2 units), lazy rescale decision: the same in both halves of a row ----
+                    const float m_tile = mx * P.scale_log2;
+                    float factor = 1.f;
+                    if (j == 0) {
+                        m_run = m_tile;
+                    } else if (m_tile > m_run + kRescaleThreshold) {
+                        factor = ex2(m_run - m_tile);           // m_run may be -inf: factor 0 clears O and l
+                        m_run = m_tile;
+                    }
+                    const float m_use = m_run == -CUDART_INF_F ? 0.f : m_run;
+                    // ---- P = exp2(s * scale - m), row sum, bf16 pairs back to tensor memory ----
+                    // (the scaling and the row sum work on pairs: one packed fp32x2 instruction per two values)
+                    float2 ls[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
+                    const float2 sc2 = make_float2(P.scale_log2, P.scale_log2), nm2 = make_float2(-m_use, -m_use);
+#pragma unroll 1
+                    for (int cc = 0; cc < nch; ++cc) {
+                        uint32_t sv[32];
+                        tmem_ld32(tS + (c0 + cc) * 32, sv);
+                        tmem_wait_ld();
+                        if (partial) {
+                            const uint32_t al = allowed_bits(c0 + cc);
+#pragma unroll
+                            for (int e = 0; e < 32; ++e)
+                                if (!((al >> e) & 1u)) sv[e] = 0xff800000u;
+                        }
+                        uint32_t pk[16];
+#pragma unroll
+                        for (int e = 0; e < 16; ++e) {
+                            const float2 t = __ffma2_rn(make_float2(__uint_as_float(sv[2 * e]), __uint_as_float(sv[2 * e + 1])), sc2, nm2);
+                            const float p0 = ex2(t.x), p1 = ex2(t.y);
+                            ls[e & 1] = __fadd2_rn(ls[e & 1], make_float2(p0, p1));
+                            const __nv_bfloat162 v = __floats2bfloat162_rn(p0, p1);
+                            pk[e] = *reinterpret_cast<const uint32_t*>(&v);
+                        }
+                        tmem_st16(tS + half * 64 + cc * 16, pk);
+                    }
+                    l_run = l_run * factor + ((ls[0].x + ls[0].y) + (ls[1].x + ls[1].y));
+                    // ---- rescale this thread's half of the accumulator when some row of the warp moved its max ----
+                    if (j > 0 && __any_sync(kFull, factor != 1.f)) {
+#pragma unroll 1
+                        for (int c = 0; c < DH / 32; ++c) {
+                            uint32_t o[32];
+                            tmem_ld32(tO + half * DH + c * 32, o);
+                            tmem_wait_ld();
+#pragma unroll
+                            for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * factor);
+                            tmem_st32(tO + half * DH + c * 32, o);
+                        }
+                    }
+                    tmem_wait_st();
+                }
+                tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&bar_pready[grp]);
             }
 
             // ---- epilogue of the segment ----
-            while (n_my > 0) {
+            if (n_my > 0) {
                 ok = __all_sync(kFull, ok && mbar_wait(&bar_odone[grp], oc & 1, ab));
                 ++oc;
-                if (!(ok && *(volatile int*)&st.redo[grp] != 0)) break;
-                tc_fence_after_sync();
-                fix_tile(tile_of(n_my - 1));                                             // woken to finish the last tile
-                publish();
             }
             tc_fence_after_sync();
             const bool final_rows = cur.complete();

@@ -525,9 +525,9 @@ def test_attention_scores_far_above_the_running_maximum(ctx, Hq, Hkv, P):
     """Keys that score 100 to 300 doublings above everything their row has seen before, one in almost every tile
     (each aimed at another query row, at varying places of the tile), plus: both column halves of one tile for
     one row, the same row in consecutive tiles with growing size, the last prefix key and the tree tile.  The
-    kernel's one-pass tiles cannot take them with the reference maximum the row has; the group has to settle a
-    new one and finish the tile.  Long prefixes, so that a CTA runs several tiles of a unit; units with two live
-    row blocks and with one."""
+    running maximum of a row then jumps again and again, by far more than the lazy-rescaling threshold, and
+    everything accumulated before has to be scaled away exactly.  Long prefixes, so that a CTA runs several
+    tiles of a unit; units with two live row blocks and with one."""
     cfg = W.shrink(W.CONFIGS[5], cid=140 + Hq, B=3, Hq=Hq, Hkv=Hkv, d=128, P=P, V=2000, k=4, t_max=5, N=50)
     inp = H.make_inputs(cfg)
     _, _, trees = H.oracle_expand_and_tree(cfg, inp)
