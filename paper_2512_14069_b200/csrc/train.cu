@@ -7,9 +7,9 @@
 //                          every layer and the activations they multiply - goes to a record per (data point,
 //                          decision) in the workspace.
 //   train_outer_kernel     the parameter gradients: sums over all records of delta (x) activation, one output
-//                          tile per block, records in a fixed order (no atomics: the result does not depend
-//                          on scheduling).
-//   train_adam_kernel      batch loss (fixed-order sum) and the Adam update.
+//                          tile and one slice of the records per block, each slice in a fixed order into its own
+//                          partial buffer (no atomics: the result does not depend on scheduling).
+//   train_adam_kernel      adds the slices up (fixed order), batch loss (fixed-order sum) and the Adam update.
 // The network is the one expand.cu runs at inference; the forward arithmetic is fp32 like there.
 #include "common.cuh"
 
@@ -20,6 +20,7 @@ constexpr int H = kHidden;            // 128
 constexpr int kTrainThreads = 4 * H;  // one thread per LSTM gate row
 constexpr int kMaxSteps = 16;
 constexpr int kXPad = 32;             // room for the k scores behind h in the head's input
+constexpr int kSlices = 8;            // the records are summed in this many slices, one block each per output tile
 
 // record of one decision (floats)
 constexpr int R_DPRE = 0;                       // [4H] delta of the LSTM pre-activations
@@ -55,6 +56,7 @@ struct TrainParams {
     float* rec;          // [n][t_max - 1][R_STRIDE]
     int* ndec;           // [n] decisions taken
     float* point_loss;   // [n]
+    float* part;         // [kSlices][parameters] partial gradient sums
 };
 
 __device__ __forceinline__ float sigmoidf(float v) { return 1.f / (1.f + __expf(-v)); }
@@ -230,25 +232,28 @@ struct OuterParams {
     OuterJob job[8];
     const float* rec;
     const int* ndec;
-    float* grad;
+    float* part;                // [kSlices][count]
+    long long count;
     int n, steps;               // records per data point = t_max - 1
-    float scale;
 };
 
 __global__ void __launch_bounds__(256) train_outer_kernel(const OuterParams P) {
     chain_wait();
-    const OuterJob J = P.job[blockIdx.z];
+    const OuterJob J = P.job[blockIdx.z % 7];
+    const int slice = blockIdx.z / 7;
     const int m0 = blockIdx.y * 32, c0 = blockIdx.x * 32;
     if (m0 >= J.M || c0 >= J.N) return;
     __shared__ float As[32][33], Bs[32][33];
     const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;     // 32 x 8
     float acc[4] = {0.f, 0.f, 0.f, 0.f};
     const int K = P.n * P.steps;
-    for (int r0 = 0; r0 < K; r0 += 32) {
+    const int per = ((K + kSlices - 1) / kSlices + 31) / 32 * 32;
+    const int r_end = min(K, (slice + 1) * per);
+    for (int r0 = slice * per; r0 < r_end; r0 += 32) {
         // stage 32 records x 32 columns of each operand (invalid records and columns past the edge: zero)
         for (int e = ty; e < 32; e += 8) {
             const int r = r0 + e;
-            const bool live = r < K && (r % P.steps) < P.ndec[r / P.steps];
+            const bool live = r < r_end && (r % P.steps) < P.ndec[r / P.steps];
             const float* rec = P.rec + (size_t)r * R_STRIDE;
             As[e][tx] = live && m0 + tx < J.M ? rec[J.a_off + m0 + tx] : 0.f;
             Bs[e][tx] = live && c0 + tx < J.N ? (J.b_off < 0 ? 1.f : rec[J.b_off + c0 + tx]) : 0.f;
@@ -267,9 +272,9 @@ __global__ void __launch_bounds__(256) train_outer_kernel(const OuterParams P) {
         for (int i = 0; i < 4; ++i) {
             const int m = m0 + ty + 8 * i;
             if (m < J.M) {
-                const float v = acc[i] * P.scale;
-                P.grad[J.out_off + (long long)m * J.ld_out + c0 + tx] = v;
-                if (J.out_off2 >= 0) P.grad[J.out_off2 + (long long)m * J.ld_out + c0 + tx] = v;
+                float* out = P.part + (long long)slice * P.count;
+                out[J.out_off + (long long)m * J.ld_out + c0 + tx] = acc[i];
+                if (J.out_off2 >= 0) out[J.out_off2 + (long long)m * J.ld_out + c0 + tx] = acc[i];
             }
         }
     }
@@ -291,10 +296,15 @@ __global__ void __launch_bounds__(256) train_adam_kernel(const TrainParams P, si
         }
         if (threadIdx.x == 0) a.loss[0] = (float)(part[0] / a.n);
     }
-    if (a.step < 1) return;
-    const float c1 = 1.f - powf(a.beta1, (float)a.step), c2 = 1.f - powf(a.beta2, (float)a.step);
+    const float c1 = 1.f - powf(a.beta1, (float)max(a.step, 1)), c2 = 1.f - powf(a.beta2, (float)max(a.step, 1));
+    const float scale = 1.f / (float)a.n;
     for (size_t i = (size_t)blockIdx.x * 256 + threadIdx.x; i < count; i += (size_t)gridDim.x * 256) {
-        const float g = a.grad[i];
+        float g = 0.f;
+#pragma unroll
+        for (int sl = 0; sl < kSlices; ++sl) g += P.part[(size_t)sl * count + i];
+        g *= scale;
+        a.grad[i] = g;
+        if (a.step < 1) continue;
         const float m = a.beta1 * a.adam_m[i] + (1.f - a.beta1) * g;
         const float v = a.beta2 * a.adam_v[i] + (1.f - a.beta2) * g * g;
         a.adam_m[i] = m;
@@ -313,7 +323,7 @@ extern "C" size_t radar_policy_param_count(int k) { return k >= 1 && k <= RADAR_
 extern "C" size_t radar_train_workspace_bytes(const radar_ctx*, int n, int k, int t_max) {
     if (n < 1 || k < 1 || t_max < 2) return 0;
     return align_up((size_t)n * (t_max - 1) * R_STRIDE * sizeof(float), 256) + align_up((size_t)n * sizeof(int), 256) +
-           align_up((size_t)n * sizeof(float), 256);
+           align_up((size_t)n * sizeof(float), 256) + align_up((size_t)kSlices * param_count(k) * sizeof(float), 256);
 }
 
 extern "C" int radar_policy_train_step(radar_ctx* ctx, const radar_train_args* a, void* stream_) {
@@ -334,6 +344,8 @@ extern "C" int radar_policy_train_step(radar_ctx* ctx, const radar_train_args* a
     P.ndec = reinterpret_cast<int*>(w);
     w += align_up((size_t)a->n * sizeof(int), 256);
     P.point_loss = reinterpret_cast<float*>(w);
+    w += align_up((size_t)a->n * sizeof(float), 256);
+    P.part = reinterpret_cast<float*>(w);
     const int k = a->k;
     {
         radar_launch_scope scope(ctx, RADAR_K_TRAIN_ROLLOUT, stream);
@@ -344,7 +356,7 @@ extern "C" int radar_policy_train_step(radar_ctx* ctx, const radar_train_args* a
         const long long o_w_ih = 0, o_w_hh = o_w_ih + 4LL * H * k, o_b_ih = o_w_hh + 4LL * H * H, o_b_hh = o_b_ih + 4 * H;
         const long long o_w1 = o_b_hh + 4 * H, o_b1 = o_w1 + (long long)H * (H + k), o_w2 = o_b1 + H, o_b2 = o_w2 + 2 * H;
         OuterParams O = {};
-        O.rec = P.rec; O.ndec = P.ndec; O.grad = a->grad; O.n = a->n; O.steps = a->t_max - 1; O.scale = 1.f / (float)a->n;
+        O.rec = P.rec; O.ndec = P.ndec; O.part = P.part; O.count = (long long)param_count(k); O.n = a->n; O.steps = a->t_max - 1;
         O.job[0] = {R_DPRE, 4 * H, R_CAT + H, k, k, o_w_ih, -1};            // w_ih: dpre (x) x
         O.job[1] = {R_DPRE, 4 * H, R_HPREV, H, H, o_w_hh, -1};              // w_hh: dpre (x) h before the step
         O.job[2] = {R_DPRE, 4 * H, -1, 1, 1, o_b_ih, o_b_hh};         // both LSTM biases
@@ -353,7 +365,7 @@ extern "C" int radar_policy_train_step(radar_ctx* ctx, const radar_train_args* a
         O.job[5] = {R_DY, 2, R_HID, H, H, o_w2, -1};                        // w2: dy (x) relu output
         O.job[6] = {R_DY, 2, -1, 1, 1, o_b2, -1};
         radar_launch_scope scope(ctx, RADAR_K_TRAIN_OUTER, stream);
-        RADAR_CUDA_CHECK(launch_chained(train_outer_kernel, dim3((unsigned)((H + k + 31) / 32), (unsigned)(4 * H / 32), 7), dim3(256), 0,
+        RADAR_CUDA_CHECK(launch_chained(train_outer_kernel, dim3((unsigned)((H + k + 31) / 32), (unsigned)(4 * H / 32), 7 * kSlices), dim3(256), 0,
                                         stream, O));
     }
     {
