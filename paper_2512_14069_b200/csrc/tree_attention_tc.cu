@@ -66,6 +66,7 @@ struct TcParams {
     long long o_ls, lse_ls;   // elements between consecutive layers of O and of lse
     int n_cls;           // classes = units per KV head
     int ncc;             // CTAs per class; grid = n_cls * ncc
+    int cost_one, cost_two, unit_cost;   // tile_costs(n_cls)
     float scale_log2;
     long long cache_rows;
     float2* part_ml;     // [grid][2][256]     (m in natural-log units, l)
@@ -86,10 +87,16 @@ __device__ __forceinline__ float ex2(float x) {
 }
 
 // ---- the tile space of one class (unit index pp within a KV head) ---------------------------------
-// Positions are in cost units: a tile of a unit with two live row blocks (four MMAs) weighs kCostTwo,
-// a tile of a unit with one live row block weighs kCostOne; equal position ranges are then about
-// equal amounts of time.  A tile belongs to the CTA whose range contains the tile's start position.
-constexpr int kCostOne = 3, kCostTwo = 5;
+// Positions are in cost units: a tile of a unit with two live row blocks (four MMAs) weighs cost_two, a tile of
+// a unit with one live row block cost_one, and every unit books cost_unit in front of its first tile for what it
+// costs beside its tiles (pipeline fill, epilogue), so that a CTA whose range holds several unit starts gets fewer
+// tiles; equal position ranges are then about equal amounts of time.  A tile belongs to the CTA whose range
+// contains the tile's start position.  The weights are measured, not derived (attention kernel inside whole steps,
+// A/B on one GPU, against 3 : 5 without the unit term): with one class per KV head 2 : 4 + 12 (ragged batch of 32:
+// 605 -> 554 us; batch 1 is not of this kind), with several classes 3 : 5 + 15 (batch 1: 27.3 -> 23.3 us; batch 8 with
+// ragged trees: 167 -> 165 us, where 2 : 4 + 12 gave 175 us).
+struct TileCosts { int one, two, unit; };
+inline TileCosts tile_costs(int n_cls) { return n_cls == 1 ? TileCosts{2, 4, 12} : TileCosts{3, 5, 15}; }
 
 struct SeqInfo {
     int M, Pb, nt;       // tree rows, prefix length, tiles of a unit (prefix tiles + the tree tile)
@@ -108,18 +115,18 @@ __device__ __forceinline__ SeqInfo seq_info(const TcParams& P, int b, int pp) {
     const bool ok = s.Pb >= 0 && s.Pb <= a.max_prefix_len && s.kv0 >= 0 && s.kv0 + s.Pb <= P.cache_rows;
     s.rows = ok ? min(max(s.M * P.G - pp * P.pair_rows, 0), P.pair_rows) : 0;
     s.nt = (max(s.Pb, 0) + kTileKeys - 1) / kTileKeys + 1;
-    s.w = s.rows > 128 ? kCostTwo : kCostOne;
+    s.w = s.rows > 128 ? P.cost_two : P.cost_one;
     return s;
 }
 template <bool PAGED>
 __device__ __forceinline__ long long seq_cost(const TcParams& P, int b, int pp) {
     const SeqInfo s = seq_info<PAGED>(P, b, pp);
-    return s.rows > 0 ? (long long)P.a.Hkv * s.nt * s.w : 0;
+    return s.rows > 0 ? (long long)P.a.Hkv * (s.nt * s.w + P.unit_cost) : 0;
 }
 // number of tiles of a unit (start position U, nt tiles of cost w) that start before position x
-__device__ __forceinline__ int tiles_before(long long x, long long U, int nt, int w) {
-    if (x <= U) return 0;
-    const long long n = (x - U + w - 1) / w;
+__device__ __forceinline__ int tiles_before(long long x, long long U, int nt, int w, int unit_cost) {
+    if (x <= U + unit_cost) return 0;
+    const long long n = (x - U - unit_cost + w - 1) / w;
     return n > nt ? nt : (int)n;
 }
 
@@ -129,11 +136,12 @@ struct Cursor {
     int b, g, t0, t1;
     int layer;           // layers follow one another in the space, each with the same sequence of units
     long long U, hi;     // start position of the current unit, end of the CTA's range
+    int unit_cost;
     SeqInfo s;
     __device__ __forceinline__ bool valid() const { return t1 > t0; }
-    __device__ __forceinline__ void clip() { t1 = tiles_before(hi, U, s.nt, s.w); }
+    __device__ __forceinline__ void clip() { t1 = tiles_before(hi, U, s.nt, s.w, unit_cost); }
     __device__ __forceinline__ void next_unit(const TcParams& P, int pp) {
-        U += (long long)s.nt * s.w;
+        U += (long long)s.nt * s.w + unit_cost;
         t0 = 0;
         if (++g == P.a.Hkv) {
             g = 0;
@@ -264,7 +272,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 const long long before = cum + __shfl_sync(kFull, incl - sz, src);
                 fb = b0 + src;
                 const SeqInfo si = seq_info<PAGED>(P, fb, pp);
-                const long long unit = (long long)si.nt * si.w;
+                const long long unit = (long long)si.nt * si.w + P.unit_cost;
                 fg = (int)((lo - before) / unit);
                 fU = before + fg * unit;
             }
@@ -307,11 +315,12 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     Cursor<PAGED> cur;
     cur.b = s_start[0]; cur.g = s_start[1]; cur.layer = s_start[2];
     cur.hi = s_range[1];
+    cur.unit_cost = P.unit_cost;
     cur.U = s_range[3];
     cur.t0 = cur.t1 = 0;
     if (cur.b >= 0) {
         cur.s = seq_info<PAGED>(P, cur.b, pp);
-        cur.t0 = tiles_before(s_range[0], cur.U, cur.s.nt, cur.s.w);
+        cur.t0 = tiles_before(s_range[0], cur.U, cur.s.nt, cur.s.w, P.unit_cost);
         if (cur.t0 >= cur.s.nt) cur.next_unit(P, pp);       // every tile of that unit starts before the range
         else cur.clip();
     }
@@ -827,7 +836,7 @@ __global__ void __launch_bounds__(256) tree_attn_tc_combine_kernel(const TcParam
     if (!cu.valid) return;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int pp = blockIdx.x % P.n_cls, c0 = blockIdx.x / P.n_cls;
-    const long long u1 = cu.u0 + (long long)cu.nt * cu.w;
+    const long long u1 = cu.u0 + (long long)cu.nt * cu.w + P.unit_cost;
     const int row0 = blockIdx.y * 8 + warp;
     if (row0 >= cu.rows) return;                             // rows of a unit are live from 0 up
     // pieces: class-local CTAs c0, c0 + 1, ... while their range starts before the unit's end
@@ -840,8 +849,8 @@ __global__ void __launch_bounds__(256) tree_attn_tc_combine_kernel(const TcParam
         return ((int64_t)((c0 + j) * P.n_cls + pp) * 2 + slot) * kPairRows;
     };
     auto live = [&](int j) {                                 // a CTA whose range holds no tile start has no piece
-        return tiles_before(cu.tot * (c0 + j + 1) / P.ncc, cu.u0, cu.nt, cu.w) >
-               tiles_before(cu.tot * (c0 + j) / P.ncc, cu.u0, cu.nt, cu.w);
+        return tiles_before(cu.tot * (c0 + j + 1) / P.ncc, cu.u0, cu.nt, cu.w, P.unit_cost) >
+               tiles_before(cu.tot * (c0 + j) / P.ncc, cu.u0, cu.nt, cu.w, P.unit_cost);
     };
     auto store_row = [&](int prow, const float (&o)[E], float mx, float den) {
         const float inv = 1.f / den;
@@ -956,7 +965,7 @@ __global__ void __launch_bounds__(256) tree_attn_tc_combine_wide_kernel(const Tc
     if (!cu.valid) return;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int pp = blockIdx.x % P.n_cls, c0 = blockIdx.x / P.n_cls;
-    const long long u1 = cu.u0 + (long long)cu.nt * cu.w;
+    const long long u1 = cu.u0 + (long long)cu.nt * cu.w + P.unit_cost;
     // pieces: class-local CTAs c0, c0 + 1, ... while their range starts before the unit's end
     int n_pieces = 1;
     while (c0 + n_pieces < P.ncc && cu.tot * (c0 + n_pieces) / P.ncc < u1) ++n_pieces;
@@ -968,8 +977,8 @@ __global__ void __launch_bounds__(256) tree_attn_tc_combine_wide_kernel(const Tc
         return ((int64_t)((c0 + j) * P.n_cls + pp) * 2 + slot) * kPairRows + prow;
     };
     auto live = [&](int j) {                                 // a CTA whose range holds no tile start has no piece
-        return tiles_before(cu.tot * (c0 + j + 1) / P.ncc, cu.u0, cu.nt, cu.w) >
-               tiles_before(cu.tot * (c0 + j) / P.ncc, cu.u0, cu.nt, cu.w);
+        return tiles_before(cu.tot * (c0 + j + 1) / P.ncc, cu.u0, cu.nt, cu.w, P.unit_cost) >
+               tiles_before(cu.tot * (c0 + j) / P.ncc, cu.u0, cu.nt, cu.w, P.unit_cost);
     };
     float den = 0.f, mx = -CUDART_INF_F, o[D / 32];
 #pragma unroll
@@ -1134,6 +1143,8 @@ int tree_attn_tc_launch(radar_ctx* ctx, const radar_attn_args* a, cudaStream_t s
     P.o_ls = P.n_layers > 1 ? a->o_layer_stride : 0;
     P.lse_ls = P.n_layers > 1 ? a->lse_layer_stride : 0;
     plan_grid(ctx, a->B, a->Hq, a->Hkv, a->max_prefix_len, &P.pair_rows, &P.n_cls, &P.ncc);
+    const TileCosts tc = tile_costs(P.n_cls);
+    P.cost_one = tc.one; P.cost_two = tc.two; P.unit_cost = tc.unit;
     if (tree_attn_tc_workspace_bytes(ctx, a->B, a->Hq, a->Hkv, a->d, a->max_prefix_len) > a->workspace_bytes)
         return RADAR_ERR_WORKSPACE;
     const size_t rec = (size_t)P.n_cls * P.ncc * 2 * kPairRows;
