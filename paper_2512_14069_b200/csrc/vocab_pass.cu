@@ -70,10 +70,9 @@ __global__ void __launch_bounds__(kThreads, WANT_LSE ? (EPT == 32 ? 5 : 6) : 5) 
     using VT = Vec<T>;
     constexpr int N = VT::N;
     constexpr int NV = EPT / N;
-    const int row = blockIdx.x / p.n_chunks;
-    const int chunk_id = blockIdx.x - row * p.n_chunks;
-    const int seq = row / p.F;
-    const int f = row - seq * p.F;
+    // grid = (chunks, rows of a sequence, sequences): no division on the way to the block's data
+    const int chunk_id = blockIdx.x, f = blockIdx.y, seq = blockIdx.z;
+    const int row = seq * p.F + f;
     if (p.seq_active != nullptr && p.seq_active[seq] == 0) return;
     if (p.seq_rows != nullptr && f >= p.seq_rows[seq]) return;
 
@@ -95,14 +94,20 @@ __global__ void __launch_bounds__(kThreads, WANT_LSE ? (EPT == 32 ? 5 : 6) : 5) 
     // ---- every load of the chunk in flight ----
     float x[NV][N];
     const T* vbase = base + body0;
+    if (head == 0 && nvec == kThreads * NV) {        // a whole, aligned chunk (all but a row's last one): nothing to check
+        const T* vp = vbase + (int64_t)tid * N;
 #pragma unroll
-    for (int u = 0; u < NV; ++u) {
-        const int j = tid + u * kThreads;
-        if (j < nvec) {
-            VT::load(vbase + (int64_t)j * N, x[u]);
-        } else {
+        for (int u = 0; u < NV; ++u) VT::load(vp + (int64_t)u * (kThreads * N), x[u]);
+    } else {
 #pragma unroll
-            for (int e = 0; e < N; ++e) x[u][e] = -CUDART_INF_F;
+        for (int u = 0; u < NV; ++u) {
+            const int j = tid + u * kThreads;
+            if (j < nvec) {
+                VT::load(vbase + (int64_t)j * N, x[u]);
+            } else {
+#pragma unroll
+                for (int e = 0; e < N; ++e) x[u][e] = -CUDART_INF_F;
+            }
         }
     }
     // head and tail (each shorter than one vector): one value for threads 0..N-1 and N..2N-1
@@ -278,9 +283,9 @@ __global__ void __launch_bounds__(kThreads, WANT_LSE ? (EPT == 32 ? 5 : 6) : 5) 
 }
 
 template <typename T, bool WANT_LSE>
-cudaError_t launch_ept(const VocabPassParams& p, unsigned grid, cudaStream_t stream) {
-    if (p.chunk / kThreads == 16) return launch_chained(vocab_pass_kernel<T, 16, WANT_LSE>, dim3(grid), dim3(kThreads), 0, stream, p);
-    return launch_chained(vocab_pass_kernel<T, 32, WANT_LSE>, dim3(grid), dim3(kThreads), 0, stream, p);
+cudaError_t launch_ept(const VocabPassParams& p, dim3 grid, cudaStream_t stream) {
+    if (p.chunk / kThreads == 16) return launch_chained(vocab_pass_kernel<T, 16, WANT_LSE>, grid, dim3(kThreads), 0, stream, p);
+    return launch_chained(vocab_pass_kernel<T, 32, WANT_LSE>, grid, dim3(kThreads), 0, stream, p);
 }
 
 }  // namespace
@@ -320,9 +325,9 @@ cudaError_t vocab_pass_preload_argbest() {
 }
 
 cudaError_t vocab_pass_launch(radar_ctx* ctx, int kernel_id, const VocabPassParams& p, cudaStream_t stream) {
-    const int rows = p.n_seq * p.F;
-    const unsigned grid = (unsigned)rows * (unsigned)p.n_chunks;
-    if (grid == 0) return cudaSuccess;
+    if (p.n_seq <= 0 || p.F <= 0 || p.n_chunks <= 0) return cudaSuccess;
+    if (p.n_seq > 65535 || p.F > 65535) return cudaErrorInvalidValue;
+    const dim3 grid((unsigned)p.n_chunks, (unsigned)p.F, (unsigned)p.n_seq);
     if (!p.want_lse && p.k != 1) return cudaErrorInvalidValue;
     radar_launch_scope scope(ctx, kernel_id, stream);
     if (p.dtype == RADAR_F32) return p.want_lse ? launch_ept<float, true>(p, grid, stream) : launch_ept<float, false>(p, grid, stream);
