@@ -40,8 +40,8 @@ NCU_TRAFFIC_RATIO = {
     ("tree_attention", 5): 398.87 / 388.08,      # captured on the first four sequences of the configuration (--batch 4)
     ("tree_attention", 4): 455.14 / 284.58,
     ("tree_attention", 3): 355.25 / 343.57,
-    ("vocab_pass(expand)", 4): 41.088 / 41.042,
-    ("vocab_pass(accept)", 4): 228.72 / 224.70,
+    ("vocab_pass(expand)", 4): 41.142 / 41.042,
+    ("vocab_pass(accept)", 4): 228.67 / 224.70,
 }
 
 
