@@ -60,7 +60,7 @@ struct CutUnit {
 
 struct TcParams {
     radar_attn_args a;
-    int G, nodes_per_rb;
+    int G, g_log2, nodes_per_rb;   // G divides 128 on this path, so it is a power of two
     int pair_rows;       // query rows of a class's units: 256 (two row blocks share each K/V tile) or 128
     int n_layers;        // layers run by this launch (the same tree, masks and prefix lengths for all)
     long long o_ls, lse_ls;   // elements between consecutive layers of O and of lse
@@ -125,9 +125,10 @@ __device__ __forceinline__ long long seq_cost(const TcParams& P, int b, int pp) 
 }
 // number of tiles of a unit (start position U, nt tiles of cost w) that start before position x
 __device__ __forceinline__ int tiles_before(long long x, long long U, int nt, int w, int unit_cost) {
-    if (x <= U + unit_cost) return 0;
-    const long long n = (x - U - unit_cost + w - 1) / w;
-    return n > nt ? nt : (int)n;
+    const long long d = x - U - unit_cost;           // clamped first, so that the division is a 32-bit one
+    if (d <= 0) return 0;
+    if (d >= (long long)nt * w) return nt;
+    return ((int)d + w - 1) / w;
 }
 
 // One CTA's walk over its range [.., hi) of the class's space: segments (sequence b, KV head g, tiles [t0, t1)).
@@ -603,14 +604,16 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             const int M = cur.s.M, Pb = cur.s.Pb, nt_unit = cur.s.nt;
             const int prow = (two ? grp * 128 : 0) + row;        // row within the unit
             const int r_glob = pp * P.pair_rows + prow;
-            const int node = r_glob / G;
-            const int hq = g * G + r_glob % G;
+            const int node = r_glob >> P.g_log2;
+            const int hq = g * G + (r_glob & (G - 1));
             const bool row_live = prow < cur.s.rows;
             // A warp none of whose 32 rows is live does no arithmetic (the products of its rows are never read):
             // it only keeps the barriers going.
             const bool warp_live = prow - lane < cur.s.rows;
             const unsigned long long live_bits = M >= 64 ? ~0ull : ((1ull << M) - 1ull);
-            const unsigned long long mask_bits = row_live ? (a.mask[(int64_t)b * kMaxNodes + node] & live_bits) : 0ull;
+            // the row's ancestor word is needed by the tree tile only (the unit's last): it is loaded here and first
+            // touched there, so that the segment does not start with a wait for global memory
+            const unsigned long long mask_word = a.mask[(int64_t)b * kMaxNodes + min(node, kMaxNodes - 1)];
             const int n_my = two ? n : (n - grp + 1) >> 1;
             float m_run = -CUDART_INF_F, l_run = 0.f;            // l_run: this thread's columns only
 
@@ -631,7 +634,7 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 const int valid = tree ? kTreeKeys : min(kTileKeys, Pb - t * kTileKeys);
                 const bool partial = tree || valid < kTileKeys;
                 auto allowed_bits = [&](int c) -> uint32_t {        // keys of chunk c this row may attend to
-                    if (tree) return (uint32_t)(mask_bits >> (c * 32));
+                    if (tree) return row_live ? (uint32_t)((mask_word & live_bits) >> (c * 32)) : 0u;
                     const int lim = valid - c * 32;
                     return lim >= 32 ? 0xffffffffu : (lim <= 0 ? 0u : ((1u << lim) - 1u));
                 };
@@ -1134,6 +1137,8 @@ int tree_attn_tc_launch(radar_ctx* ctx, const radar_attn_args* a, cudaStream_t s
     TcParams P;
     P.a = *a;
     P.G = a->Hq / a->Hkv;
+    P.g_log2 = 0;
+    while ((1 << P.g_log2) < P.G) ++P.g_log2;
     P.nodes_per_rb = 128 / P.G;
     const float scale = a->scale > 0.f ? a->scale : 1.f / sqrtf((float)a->d);
     P.scale_log2 = scale * 1.4426950408889634f;
