@@ -80,6 +80,13 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
     asm("max.f32 %0, %1, %2, %3;" : "=f"(y) : "f"(a), "f"(b), "f"(c));
     return y;
 }
+// one 32-byte store: a whole sector per lane (the epilogue's lanes write to different rows, so every store
+// instruction is split into one transaction per lane; with 16-byte stores each of them filled half a sector)
+__device__ __forceinline__ void st_global_32b(void* p, const uint32_t (&w)[8]) {
+    asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(p), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]),
+                 "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7])
+                 : "memory");
+}
 __device__ __forceinline__ float ex2(float x) {
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -771,21 +778,31 @@ tree_attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                     if (row_live) {
                         if (final_rows) {
                             __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(a.O) + cur.layer * P.o_ls + out_row * D + col;
+                            const bool wide = (reinterpret_cast<uintptr_t>(dst) & 31) == 0;
 #pragma unroll
-                            for (int q = 0; q < 4; ++q) {
-                                uint32_t w[4];
+                            for (int q = 0; q < 2; ++q) {
+                                uint32_t w[8];
 #pragma unroll
-                                for (int e = 0; e < 4; ++e) {
-                                    const __nv_bfloat162 t2 = __floats2bfloat162_rn(v[q * 8 + 2 * e] * inv, v[q * 8 + 2 * e + 1] * inv);
+                                for (int e = 0; e < 8; ++e) {
+                                    const __nv_bfloat162 t2 = __floats2bfloat162_rn(v[q * 16 + 2 * e] * inv, v[q * 16 + 2 * e + 1] * inv);
                                     w[e] = *reinterpret_cast<const uint32_t*>(&t2);
                                 }
-                                *reinterpret_cast<uint4*>(dst + q * 8) = make_uint4(w[0], w[1], w[2], w[3]);
+                                if (wide) {
+                                    st_global_32b(dst + q * 16, w);
+                                } else {
+                                    *reinterpret_cast<uint4*>(dst + q * 16) = make_uint4(w[0], w[1], w[2], w[3]);
+                                    *reinterpret_cast<uint4*>(dst + q * 16 + 8) = make_uint4(w[4], w[5], w[6], w[7]);
+                                }
                             }
                         } else {
-                            float* dst = P.part_o + rec * D + col;
+                            float* dst = P.part_o + rec * D + col;          // 128-byte aligned (workspace carve)
 #pragma unroll
-                            for (int q = 0; q < 8; ++q)
-                                *reinterpret_cast<float4*>(dst + q * 4) = make_float4(v[q * 4], v[q * 4 + 1], v[q * 4 + 2], v[q * 4 + 3]);
+                            for (int q = 0; q < 4; ++q) {
+                                uint32_t w[8];
+#pragma unroll
+                                for (int e = 0; e < 8; ++e) w[e] = __float_as_uint(v[q * 8 + e]);
+                                st_global_32b(dst + q * 8, w);
+                            }
                         }
                     }
                 }
