@@ -37,9 +37,9 @@ L2_BYTES = 126 * 1024 * 1024
 # captures summarised under profiles/ (kernel name, config id); traffic of a launch at the same shapes =
 # ratio x its algorithmic bytes (both grow with the rows processed).  Absent = not captured.
 NCU_TRAFFIC_RATIO = {
-    ("tree_attention", 5): 398.47 / 388.08,      # captured on the first four sequences of the configuration (--batch 4)
-    ("tree_attention", 4): 454.48 / 284.58,
-    ("tree_attention", 3): 356.13 / 343.57,
+    ("tree_attention", 5): 398.90 / 388.08,      # captured on the first four sequences of the configuration (--batch 4)
+    ("tree_attention", 4): 457.37 / 284.58,
+    ("tree_attention", 3): 355.21 / 343.57,
     ("vocab_pass(expand)", 4): 41.142 / 41.042,
     ("vocab_pass(accept)", 4): 228.67 / 224.70,
 }
