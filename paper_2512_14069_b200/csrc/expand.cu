@@ -136,6 +136,7 @@ __global__ void __launch_bounds__(kSelThreads, 1) expand_select_gate_kernel(cons
     __shared__ int s_ti[kMergeWarps], s_ri[kMergeWarps][32];
 
     if (tid == 0) s_base = a.t > 1 ? a.pool_len[b] : 0;
+    const int forced = a.force_calls != nullptr ? a.force_calls[b] : -1;     // read now, needed at the very end
 
     if (warp < kMergeWarps) {
         // ---- 1a. chunk records -> shared memory (coalesced), then per row: top-k, log-normaliser, scores ----
@@ -176,8 +177,8 @@ __global__ void __launch_bounds__(kSelThreads, 1) expand_select_gate_kernel(cons
                     const float hv = lane < n_chunks ? pv[lane * k] : -CUDART_INF_F;
                     const int hi = lane < n_chunks ? pi[lane * k] : 0x7fffffff;
                     int rank = 0;
-#pragma unroll
-                    for (int o = 0; o < 32; ++o) {
+#pragma unroll 4
+                    for (int o = 0; o < n_chunks; ++o) {                 // lanes beyond the chunks hold (-inf, max): they precede nothing
                         const float ov = __shfl_sync(kFull, hv, o);
                         const int oi = __shfl_sync(kFull, hi, o);
                         rank += precedes(ov, oi, hv, hi) ? 1 : 0;
@@ -329,11 +330,18 @@ __global__ void __launch_bounds__(kSelThreads, 1) expand_select_gate_kernel(cons
     __syncthreads();      // draft_row = -1 must land before the survivors overwrite theirs
 
     // ---- 3. the k best candidates over all parents (score desc, flat index asc) ----
-    for (int e = tid; e < n_cand; e += kSelThreads) {
-        const double v = s_cand[e];
+    // eight threads share a candidate's rank count (n_cand <= 1024: at most 8 rounds)
+    for (int e0 = 0; e0 < n_cand; e0 += kSelThreads / 8) {
+        const int e = e0 + (tid >> 3), part = tid & 7;
+        const bool have = e < n_cand;
+        const double v = have ? s_cand[e] : 0.0;
         int rank = 0;
-        for (int j = 0; j < n_cand; ++j) rank += precedes(s_cand[j], j, v, e) ? 1 : 0;
-        if (rank < k) {
+        if (have)
+            for (int j = part; j < n_cand; j += 8) rank += precedes(s_cand[j], j, v, e) ? 1 : 0;
+        rank += __shfl_xor_sync(kFull, rank, 1);
+        rank += __shfl_xor_sync(kFull, rank, 2);
+        rank += __shfl_xor_sync(kFull, rank, 4);
+        if (have && part == 0 && rank < k) {
             const float sc = (float)v;
             const size_t o = (size_t)b * k + rank;
             a.frontier_tok[o] = s_ctok[e];
@@ -341,7 +349,7 @@ __global__ void __launch_bounds__(kSelThreads, 1) expand_select_gate_kernel(cons
             a.frontier_pool_idx[o] = base + e;
             a.frontier_src_row[o] = e / k;
             a.pool_draft_row[pb + e] = 1 + (a.t - 1) * k + rank;
-            s_x[rank] = (float)exp((double)sc);                  // confidence score in [0,1]
+            s_x[rank] = expf(sc);                                // confidence score in [0,1]
         }
     }
     if (tid == 0) a.pool_len[b] = base + n_cand;
@@ -366,7 +374,7 @@ __global__ void __launch_bounds__(kSelThreads, 1) expand_select_gate_kernel(cons
         __syncthreads();
         cont = s_y[1] > s_y[0];
         if (tid < 2) a.gate_logits[(size_t)b * 2 + tid] = s_y[tid];
-        if (a.force_calls != nullptr) cont = a.t < a.force_calls[b];
+        if (forced >= 0) cont = a.t < forced;
     } else if (run_gate) {
         if (tid < 4 * H) {
             float acc = s_pre[tid];
@@ -409,7 +417,7 @@ __global__ void __launch_bounds__(kSelThreads, 1) expand_select_gate_kernel(cons
         __syncthreads();
         cont = s_y[1] > s_y[0];
         if (tid < 2) a.gate_logits[(size_t)b * 2 + tid] = s_y[tid];
-        if (a.force_calls != nullptr) cont = a.t < a.force_calls[b];
+        if (forced >= 0) cont = a.t < forced;
     } else {
         if (tid < 2) a.gate_logits[(size_t)b * 2 + tid] = 0.f;
     }
