@@ -156,8 +156,9 @@ __global__ void __launch_bounds__(kSelThreads, 1) expand_select_gate_kernel(cons
         for (int f = warp; f < F; f += kMergeWarps) {
             const size_t row = row0 + f;
             // log-sum-exp over the chunks in fp64: the first loads are issued here and consumed after the merge
-            const float pm0 = lane < n_chunks ? P.vp.part_m[row * n_chunks + lane] : -CUDART_INF_F;
-            const float ps0 = lane < n_chunks ? P.vp.part_s[row * n_chunks + lane] : 0.f;
+            // (always from a valid address, and not looked at before the merge is done: nothing below waits for them)
+            const float pm0_raw = P.vp.part_m[row * n_chunks + min(lane, n_chunks - 1)];
+            const float ps0_raw = P.vp.part_s[row * n_chunks + min(lane, n_chunks - 1)];
             WarpTopList<float> top;
             top.reset();
             bool merged = false;
@@ -246,6 +247,8 @@ __global__ void __launch_bounds__(kSelThreads, 1) expand_select_gate_kernel(cons
                     }
                 }
             }
+            const float pm0 = lane < n_chunks ? pm0_raw : -CUDART_INF_F;
+            const float ps0 = lane < n_chunks ? ps0_raw : 0.f;
             float mloc = pm0;
             for (int c = lane + 32; c < n_chunks; c += 32) mloc = fmaxf(mloc, P.vp.part_m[row * n_chunks + c]);
             const float M = warp_max(mloc);
@@ -399,13 +402,32 @@ __global__ void __launch_bounds__(kSelThreads, 1) expand_select_gate_kernel(cons
             s_hn[tid] = hn;
         }
         __syncthreads();
-        for (int r = warp; r < H; r += kSelWarps) {
-            const float* w = s_w1 + r * (H + kx);
-            float acc = 0.f;
-            for (int c = lane; c < H; c += 32) acc = fmaf(w[c], s_hn[c], acc);
-            if (lane < kx) acc = fmaf(w[H + lane], s_x[lane], acc);
-            acc = warp_sum(acc);
-            if (lane == 0) s_hid[r] = fmaxf(acc + s_b1[r] + (policy == RADAR_POLICY_LSTM_HIDDEN ? P.feat_hid[(size_t)b * H + r] : 0.f), 0.f);
+        {
+            // a warp's four rows side by side: the inputs are read once and the four reductions run interleaved
+            static_assert(kHidden == 4 * kSelWarps, "four rows of the hidden layer per warp");
+            const float hv[4] = {s_hn[lane], s_hn[lane + 32], s_hn[lane + 64], s_hn[lane + 96]};
+            const float xv = lane < kx ? s_x[lane] : 0.f;
+            float acc[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const float* w = s_w1 + (warp + i * kSelWarps) * (H + kx);
+                float t = w[lane] * hv[0];
+                t = fmaf(w[lane + 32], hv[1], t);
+                t = fmaf(w[lane + 64], hv[2], t);
+                t = fmaf(w[lane + 96], hv[3], t);
+                if (lane < kx) t = fmaf(w[H + lane], xv, t);
+                acc[i] = t;
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+#pragma unroll
+                for (int i = 0; i < 4; ++i) acc[i] += __shfl_xor_sync(kFull, acc[i], o);
+            }
+            if (lane < 4) {
+                const int r = warp + lane * kSelWarps;
+                const float v = lane == 0 ? acc[0] : lane == 1 ? acc[1] : lane == 2 ? acc[2] : acc[3];
+                s_hid[r] = fmaxf(v + s_b1[r] + (policy == RADAR_POLICY_LSTM_HIDDEN ? P.feat_hid[(size_t)b * H + r] : 0.f), 0.f);
+            }
         }
         __syncthreads();
         if (warp < 2) {
