@@ -31,6 +31,7 @@ enum radar_kernel_id {
 // kernels that opt in to more than 48 KB of dynamic shared memory: one slot per instantiation
 enum radar_smem_slot {
     RADAR_SMEM_SELECT_GATE = 0,
+    RADAR_SMEM_SELECT_GATE_CLUSTER,   // the instantiation with helper blocks
     RADAR_SMEM_TREE_BUILD,
     RADAR_SMEM_ATTN_FMA,        // + 2 * (bf16) + (d == 128)
     RADAR_SMEM_ATTN_TC = RADAR_SMEM_ATTN_FMA + 4,   // + 4 * (d == 128) + 2 * two + paged

@@ -14,6 +14,8 @@ constexpr int kMergeWarps = 16;                      // warps 0..15 merge chunk 
 constexpr int kMaxF = 32;
 constexpr size_t kStageLimit = 96 * 1024;            // chunk records are staged in shared memory up to this size
 constexpr int kSurvCap = 256;                        // per-row survivor list of the parallel merge
+constexpr int kSelCluster = 4;                       // blocks per sequence when the recurrent product is shared out
+constexpr long long kShortPassLogits = 4 << 20;      // ... which is done while a vocabulary pass reads at most this many logits
 
 struct SelectParams {
     radar_expand_args a;
@@ -24,6 +26,8 @@ struct SelectParams {
                                                      //    is not this call's vocabulary pass, so nothing is read before the wait
     const float* feat_pre;                           // hidden-state policy: [B][4H] W_ih f and [B][H] W_1[:, H:] f,
     const float* feat_hid;                           // written by gate_features_kernel
+    int cluster;                                     // blocks per sequence: block 0 of a cluster does the work below,
+                                                     // the others hold W_hh in shared memory and multiply it by h
 };
 
 // Hidden-state policy (Table 3): the input-side products of the prediction model, W_ih f_b (4H rows) and the
@@ -89,20 +93,87 @@ __device__ __forceinline__ void cp_async16(void* smem, const void* gmem) {
 __device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
 __host__ __device__ inline size_t up16(size_t x) { return (x + 15) & ~(size_t)15; }
 
+// Thread-block cluster pieces of the select + gate block: stores and barrier arrivals into block 0's shared memory.
+__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void cluster_barrier() {
+    asm volatile("barrier.cluster.arrive.release;\n\tbarrier.cluster.wait.acquire;" ::: "memory");
+}
+__device__ __forceinline__ void st_cluster_f32(const float* local, uint32_t rank, float v) {
+    asm volatile("{\n\t.reg .b32 ra;\n\tmapa.shared::cluster.u32 ra, %0, %1;\n\tst.shared::cluster.f32 [ra], %2;\n\t}" ::"r"(
+                     smem_addr(local)), "r"(rank), "f"(v) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(const uint64_t* local, uint32_t rank) {
+    asm volatile("{\n\t.reg .b32 ra;\n\tmapa.shared::cluster.u32 ra, %0, %1;\n\t"
+                 "mbarrier.arrive.release.cluster.shared::cluster.b64 _, [ra];\n\t}" ::"r"(smem_addr(local)), "r"(rank) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait_cluster(const uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+                 "selp.u32 %0, 1, 0, p;\n\t}" : "=r"(ok) : "r"(smem_addr(bar)), "r"(parity) : "memory");
+    return ok != 0;
+}
+constexpr int kHelperRows(int n_help) { return (4 * kHidden + n_help - 1) / n_help; }
+
 // One block per sequence.  Phase 1 runs two things side by side: warps 0-15 merge the vocabulary pass's
 // chunk records into each row's top-k and log-normaliser, warps 16-31 do everything of the prediction
 // model that does not depend on this call's candidates (W_hh h + biases, weights into shared memory).
 // Phase 2 appends the candidates to the pool and selects the frontier; phase 3 finishes the LSTM cell
 // and the MLP head from shared memory only.
+template <bool kHelpers>
 __global__ void __launch_bounds__(kSelThreads, 1) expand_select_gate_kernel(const SelectParams P) {
     // The predecessor is this call's vocabulary pass, whose blocks wait for everything before them:
     // the previous call's state (active, h, c, pool_len) is complete when this block starts.  Only
     // the chunk records need the pass itself, so the gate warps never wait for it.
     chain_trigger();
-    if (P.split) chain_sync();                         // the predecessor may be the previous call's select + gate block
     const radar_expand_args& a = P.a;
-    const int b = blockIdx.x;
+    const int n_help = kHelpers ? P.cluster - 1 : 0;   // blocks of the cluster that only multiply W_hh by h
+    const int b = kHelpers ? blockIdx.x / P.cluster : blockIdx.x;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    extern __shared__ __align__(16) unsigned char sel_smem[];
+    __shared__ float s_pre[4 * kHidden];
+    __shared__ __align__(8) uint64_t s_pre_bar;        // block 0's: counts the helper warps that have delivered
+    uint32_t crank = 0;
+    if (kHelpers) asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(crank));
+
+    if (crank != 0) {
+        // ---- helper block: rows [hr0, hr1) of W_hh h + biases, into block 0's s_pre ----
+        // The weights are constants: they are in shared memory before the predecessor is done, so that the
+        // product costs block 0 no global-memory traffic at all once the state is there.
+        const int H = kHidden;
+        const int hr0 = ((int)crank - 1) * kHelperRows(n_help), hr1 = min(4 * H, hr0 + kHelperRows(n_help));
+        float* s_w = reinterpret_cast<float*>(sel_smem);
+        for (int e = tid; e < (hr1 - hr0) * H / 4; e += kSelThreads) cp_async16(s_w + 4 * e, a.w_hh + (size_t)hr0 * H + 4 * e);
+        cluster_barrier();                             // block 0 has started and its barrier word is initialised
+        if (P.split) chain_sync();
+        if (!(a.t > 1 && a.active[b] == 0)) {          // (block 0 takes the same decision and waits for nobody)
+            cp_async_wait_all();
+            __syncthreads();
+            const bool state = a.t > 1;
+            const float* hb = a.h + (size_t)b * H + lane * 4;
+            const float4 h4 = state ? make_float4(hb[0], hb[1], hb[2], hb[3]) : make_float4(0.f, 0.f, 0.f, 0.f);
+            for (int r = hr0 + warp; r < hr1; r += kSelWarps) {
+                const float4 w = *reinterpret_cast<const float4*>(s_w + (size_t)(r - hr0) * H + lane * 4);
+                float acc = w.x * h4.x;                // the same arithmetic, in the same order, as block 0's own loop
+                acc = fmaf(w.y, h4.y, acc);
+                acc = fmaf(w.z, h4.z, acc);
+                acc = fmaf(w.w, h4.w, acc);
+                acc = warp_sum(acc);
+                if (lane == 0) st_cluster_f32(&s_pre[r], 0, acc + a.b_ih[r] + a.b_hh[r]);
+            }
+            if (lane == 0) mbar_arrive_cluster(&s_pre_bar, 0);       // release: after this lane's stores
+        }
+        cp_async_wait_all();
+        chain_sync();
+        return;
+    }
+    if (n_help > 0) {
+        if (tid == 0) {
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(&s_pre_bar)), "r"(n_help * kSelWarps) : "memory");
+            asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        }
+        cluster_barrier();
+    }
+    if (P.split) chain_sync();                         // the predecessor may be the previous call's select + gate block
     if (a.t > 1 && a.active[b] == 0) {                 // call 1 always runs: it (re)starts every sequence
         chain_sync();
         if (tid == 0) a.cont[b] = 0;
@@ -115,7 +186,6 @@ __global__ void __launch_bounds__(kSelThreads, 1) expand_select_gate_kernel(cons
     const int policy = a.policy;
     const int kx = policy == RADAR_POLICY_LSTM_HIDDEN ? 0 : k;      // input columns the block itself multiplies
 
-    extern __shared__ __align__(16) unsigned char sel_smem[];
     const size_t stage_elems = P.staged ? (size_t)F * per_row : 0;
     float* st_v = reinterpret_cast<float*>(sel_smem);                              // [F][n_chunks][k] if staged
     int* st_i = reinterpret_cast<int*>(sel_smem + up16(stage_elems * 4));
@@ -128,7 +198,7 @@ __global__ void __launch_bounds__(kSelThreads, 1) expand_select_gate_kernel(cons
     __shared__ int s_ctok[kMaxF * RADAR_MAX_K];
     __shared__ float s_x[RADAR_MAX_K];                 // gate input
     __shared__ __align__(16) float s_h[kHidden];
-    __shared__ float s_hn[kHidden], s_pre[4 * kHidden], s_hid[kHidden], s_c[kHidden];
+    __shared__ float s_hn[kHidden], s_hid[kHidden], s_c[kHidden];
     __shared__ float s_b1[kHidden], s_w2[2 * kHidden], s_b2[2];
     __shared__ float s_y[2];
     __shared__ int s_base;
@@ -292,7 +362,7 @@ __global__ void __launch_bounds__(kSelThreads, 1) expand_select_gate_kernel(cons
         group_barrier(3);
         const float4 h4 = *reinterpret_cast<const float4*>(&s_h[lane * 4]);
         constexpr int kBatch = 8;
-        for (int r0 = gw * 32; policy != RADAR_POLICY_MLP_SCORES && r0 < gw * 32 + 32; r0 += kBatch) {
+        for (int r0 = gw * 32; n_help == 0 && policy != RADAR_POLICY_MLP_SCORES && r0 < gw * 32 + 32; r0 += kBatch) {
             float4 w[kBatch];
 #pragma unroll
             for (int i = 0; i < kBatch; ++i)
@@ -311,6 +381,11 @@ __global__ void __launch_bounds__(kSelThreads, 1) expand_select_gate_kernel(cons
         if (gt < 2 * H) s_w2[gt] = a.w2[gt];
         if (gt < 2) s_b2[gt] = a.b2[gt];
         cp_async_wait_all();
+        if (n_help > 0 && gt == 0) {                   // the helpers' rows of s_pre; the barrier below publishes them
+            bool ok = false;
+            for (uint32_t it = 0; it < (1u << 22) && !(ok = mbar_try_wait_cluster(&s_pre_bar, 0)); ++it) {}
+            if (!ok) set_status(P.status, RADAR_ERR_TIMEOUT);
+        }
     }
     __syncthreads();
     const int base = s_base;
@@ -530,10 +605,40 @@ extern "C" int radar_expand_step(radar_ctx* ctx, const radar_expand_args* a, voi
                               sizeof(float) * ((size_t)4 * kHidden * a->k + (size_t)kHidden * (kHidden + a->k));
     sp.staged = stage_bytes <= kStageLimit && 2 * up16(stage_bytes / 2) + fixed_smem <= 227 * 1024 ? 1 : 0;
     const size_t smem = 2 * up16(sp.staged ? stage_bytes / 2 : 0) + fixed_smem;
-    RADAR_CUDA_CHECK(radar_opt_in_smem(ctx, RADAR_SMEM_SELECT_GATE, expand_select_gate_kernel, smem));
+    // Blocks per sequence.  With a recurrent policy, three more blocks per sequence hold W_hh (256 KB, more than
+    // one block has room for) in their shared memory, loaded while the predecessor still runs, and deliver
+    // W_hh h + biases into block 0: the block then streams none of it after the wait (measured: 1.3 us less per
+    // draft call at B = 1 and B = 4).  That pays while the draft calls are a chain of short, latency-bound
+    // kernels.  Once the next call's vocabulary pass, which shares the device with this kernel, is long enough
+    // to be the slower of the two, the waiting helper blocks only take SMs from it (B = 8, V = 128256: 0.8 us
+    // MORE per call), so larger passes keep one block per sequence.
+    const bool recurrent = gate_runs && a->policy != RADAR_POLICY_MLP_SCORES;
+    const size_t helper_bytes = (size_t)kHelperRows(kSelCluster - 1) * kHidden * sizeof(float);
+    const bool short_pass = (long long)a->B * a->k * a->V <= kShortPassLogits;
+    sp.cluster = recurrent && short_pass && a->B * kSelCluster * 2 <= ctx->sm_count && smem >= helper_bytes ? kSelCluster : 1;
     {
         radar_launch_scope scope(ctx, RADAR_K_SELECT_GATE, stream);
-        RADAR_CUDA_CHECK(launch_chained(expand_select_gate_kernel, dim3(a->B), dim3(kSelThreads), smem, stream, sp));
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)(a->B * sp.cluster));
+        cfg.blockDim = dim3(kSelThreads);
+        cfg.dynamicSmemBytes = smem;
+        cfg.stream = stream;
+        cudaLaunchAttribute attr[2];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        attr[1].id = cudaLaunchAttributeClusterDimension;
+        attr[1].val.clusterDim.x = (unsigned)sp.cluster;
+        attr[1].val.clusterDim.y = 1;
+        attr[1].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = sp.cluster > 1 ? 2 : 1;
+        if (sp.cluster > 1) {
+            RADAR_CUDA_CHECK(radar_opt_in_smem(ctx, RADAR_SMEM_SELECT_GATE_CLUSTER, expand_select_gate_kernel<true>, smem));
+            RADAR_CUDA_CHECK(cudaLaunchKernelEx(&cfg, expand_select_gate_kernel<true>, sp));
+        } else {
+            RADAR_CUDA_CHECK(radar_opt_in_smem(ctx, RADAR_SMEM_SELECT_GATE, expand_select_gate_kernel<false>, smem));
+            RADAR_CUDA_CHECK(cudaLaunchKernelEx(&cfg, expand_select_gate_kernel<false>, sp));
+        }
     }
     RADAR_CUDA_CHECK(cudaGetLastError());
     return RADAR_OK;

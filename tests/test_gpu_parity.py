@@ -349,6 +349,21 @@ def test_expansion_edge_sizes(ctx, k, V):
     H.compare_tree(cfg, g, trees)
 
 
+@pytest.mark.parametrize("B", [2, 20])
+def test_gate_with_and_without_helper_blocks(ctx, B):
+    """The select + gate kernel runs as a cluster of four blocks per sequence while 8 B blocks fit the device (three
+    of them hold W_hh in shared memory and deliver W_hh h into the first), and as one block per sequence beyond
+    that.  B = 2 takes the first form, B = 20 the second; gate state and decisions must match the oracle in both."""
+    cfg = W.shrink(W.CONFIGS[1], cid=80 + B, B=B, V=5003, k=6, t_max=6, N=30, gate_b2_offset=0.5)   # every call runs
+    inp = H.make_inputs(cfg, with_attention=False)
+    pools, traces, trees = H.oracle_expand_and_tree(cfg, inp)
+    H.check_margins(cfg, traces, trees)
+    g = H.CudaRun(cfg, inp, ctx)
+    g.expand_and_tree()
+    H.compare_expansion(cfg, g, pools, traces)
+    H.compare_tree(cfg, g, trees)
+
+
 def test_minus_inf_logits_and_nan_status(ctx):
     import torch
     cfg = W.shrink(W.CONFIGS[1], cid=70, B=1)
