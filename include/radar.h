@@ -95,7 +95,8 @@ int radar_reset_launch_counts(radar_ctx* ctx);
  *   step needs no separate reset.
  * A NaN logit records RADAR_ERR_NUMERIC (outputs of that sequence unspecified).
  * Limits: 1 <= k <= RADAR_MAX_K, 1 <= F <= 32, V >= k, pool_len[b] + F*k <= pool_capacity;
- * w_ih, w_hh and w1 16-byte aligned.
+ * w_ih, w_hh and w1 16-byte aligned.  The gate's weights must not be written between call 1 of a step and
+ * its last call: calls t >= 2 may fetch them before the work queued ahead of them on the stream has finished.
  *
  * `policy` selects the policy networks of the paper's ablation (Table 3):
  *   RADAR_POLICY_LSTM_SCORES  the model above (the default, value 0);

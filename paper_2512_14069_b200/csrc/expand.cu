@@ -121,11 +121,17 @@ constexpr int kHelperRows(int n_help) { return (4 * kHidden + n_help - 1) / n_he
 // and the MLP head from shared memory only.
 template <bool kHelpers>
 __global__ void __launch_bounds__(kSelThreads, 1) expand_select_gate_kernel(const SelectParams P) {
-    // The predecessor is this call's vocabulary pass, whose blocks wait for everything before them:
-    // the previous call's state (active, h, c, pool_len) is complete when this block starts.  Only
-    // the chunk records need the pass itself, so the gate warps never wait for it.
-    chain_trigger();
+    // Launched behind its vocabulary pass in one call, the predecessor is that pass, whose blocks wait for
+    // everything before them: the previous call's state (active, h, c, pool_len) is complete when this block
+    // starts.  Only the chunk records need the pass itself, so the gate warps never wait for it.
+    // Launched on its own (split), the predecessor on the stream is the previous call's select + gate block, or,
+    // at call 1, anything at all.  The only thing read before the wait for it are the gate's weights, and only
+    // from call 2 on: they may not change during an expansion, and whoever wrote them before call 1 is complete
+    // when the block of call 2 starts, because the block of call 1 lets its successor start only after its own
+    // wait (the trigger below sits behind the wait in this form).
+    if (!P.split) chain_trigger();
     const radar_expand_args& a = P.a;
+    const bool early = !P.split || a.t >= 2;           // weights may be fetched before the wait
     const int n_help = kHelpers ? P.cluster - 1 : 0;   // blocks of the cluster that only multiply W_hh by h
     const int b = kHelpers ? blockIdx.x / P.cluster : blockIdx.x;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -142,9 +148,12 @@ __global__ void __launch_bounds__(kSelThreads, 1) expand_select_gate_kernel(cons
         const int H = kHidden;
         const int hr0 = ((int)crank - 1) * kHelperRows(n_help), hr1 = min(4 * H, hr0 + kHelperRows(n_help));
         float* s_w = reinterpret_cast<float*>(sel_smem);
-        for (int e = tid; e < (hr1 - hr0) * H / 4; e += kSelThreads) cp_async16(s_w + 4 * e, a.w_hh + (size_t)hr0 * H + 4 * e);
+        if (early)
+            for (int e = tid; e < (hr1 - hr0) * H / 4; e += kSelThreads) cp_async16(s_w + 4 * e, a.w_hh + (size_t)hr0 * H + 4 * e);
         cluster_barrier();                             // block 0 has started and its barrier word is initialised
-        if (P.split) chain_sync();
+        if (P.split) { chain_sync(); chain_trigger(); }
+        if (!early)
+            for (int e = tid; e < (hr1 - hr0) * H / 4; e += kSelThreads) cp_async16(s_w + 4 * e, a.w_hh + (size_t)hr0 * H + 4 * e);
         if (!(a.t > 1 && a.active[b] == 0)) {          // (block 0 takes the same decision and waits for nobody)
             cp_async_wait_all();
             __syncthreads();
@@ -166,19 +175,6 @@ __global__ void __launch_bounds__(kSelThreads, 1) expand_select_gate_kernel(cons
         chain_sync();
         return;
     }
-    if (n_help > 0) {
-        if (tid == 0) {
-            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(&s_pre_bar)), "r"(n_help * kSelWarps) : "memory");
-            asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        }
-        cluster_barrier();
-    }
-    if (P.split) chain_sync();                         // the predecessor may be the previous call's select + gate block
-    if (a.t > 1 && a.active[b] == 0) {                 // call 1 always runs: it (re)starts every sequence
-        chain_sync();
-        if (tid == 0) a.cont[b] = 0;
-        return;
-    }
     const int F = a.F, k = a.k, H = kHidden;
     const int n_chunks = P.vp.n_chunks;
     const int per_row = n_chunks * k;
@@ -194,6 +190,40 @@ __global__ void __launch_bounds__(kSelThreads, 1) expand_select_gate_kernel(cons
     float* s_wih = reinterpret_cast<float*>(sv_i + kMergeWarps * kSurvCap);         // [4H][k]
     float* s_w1 = s_wih + 4 * H * k;                                                // [H][H + k]
 
+    // The gate's weights are constants: their copies into shared memory are issued before the wait where that is
+    // allowed, so that they cross the SM's load path while the predecessor still runs and not beside the merge.
+    auto stage_weights = [&]() {
+        if (warp < kMergeWarps || !run_gate) return;
+        const int gt = tid - kMergeWarps * 32;          // 0..511
+        if (policy == RADAR_POLICY_MLP_SCORES) {
+            for (int e = gt; e < H * k / 4; e += 512) cp_async16(s_w1 + 4 * e, a.w1 + 4 * e);     // [H][k]
+        } else if (policy == RADAR_POLICY_LSTM_HIDDEN) {
+            // only the head's columns for the LSTM output; the input columns were applied by gate_features_kernel
+            for (int e = gt; e < H * H / 4; e += 512) {
+                const int r = e / (H / 4), c4 = e % (H / 4);
+                cp_async16(s_w1 + r * H + c4 * 4, a.w1 + (size_t)r * (H + a.feat_dim) + c4 * 4);
+            }
+        } else {
+            for (int e = gt; e < H * k; e += 512) cp_async16(s_wih + 4 * e, a.w_ih + 4 * e);          // 4H*k floats
+            for (int e = gt; e < H * (H + k) / 4; e += 512) cp_async16(s_w1 + 4 * e, a.w1 + 4 * e);
+        }
+    };
+    if (early) stage_weights();
+    if (n_help > 0) {
+        if (tid == 0) {
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(&s_pre_bar)), "r"(n_help * kSelWarps) : "memory");
+            asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        }
+        cluster_barrier();
+    }
+    if (P.split) { chain_sync(); chain_trigger(); }
+    if (!early) stage_weights();
+    if (a.t > 1 && a.active[b] == 0) {                 // call 1 always runs: it (re)starts every sequence
+        cp_async_wait_all();                           // nothing of this block is in flight when it leaves
+        chain_sync();
+        if (tid == 0) a.cont[b] = 0;
+        return;
+    }
     __shared__ double s_cand[kMaxF * RADAR_MAX_K];     // candidate scores, flat (f, j)
     __shared__ int s_ctok[kMaxF * RADAR_MAX_K];
     __shared__ float s_x[RADAR_MAX_K];                 // gate input
@@ -342,18 +372,6 @@ __global__ void __launch_bounds__(kSelThreads, 1) expand_select_gate_kernel(cons
         // ---- 1b. the part of the prediction model that only needs the previous state ----
         const int gt = tid - kMergeWarps * 32;          // 0..511
         const int gw = warp - kMergeWarps;              // 0..15
-        if (policy == RADAR_POLICY_MLP_SCORES) {
-            for (int e = gt; e < H * k / 4; e += 512) cp_async16(s_w1 + 4 * e, a.w1 + 4 * e);     // [H][k]
-        } else if (policy == RADAR_POLICY_LSTM_HIDDEN) {
-            // only the head's columns for the LSTM output; the input columns were applied by gate_features_kernel
-            for (int e = gt; e < H * H / 4; e += 512) {
-                const int r = e / (H / 4), c4 = e % (H / 4);
-                cp_async16(s_w1 + r * H + c4 * 4, a.w1 + (size_t)r * (H + a.feat_dim) + c4 * 4);
-            }
-        } else {
-            for (int e = gt; e < H * k; e += 512) cp_async16(s_wih + 4 * e, a.w_ih + 4 * e);          // 4H*k floats
-            for (int e = gt; e < H * (H + k) / 4; e += 512) cp_async16(s_w1 + 4 * e, a.w1 + 4 * e);
-        }
         if (gt < H) {
             const bool state = a.t > 1 && policy != RADAR_POLICY_MLP_SCORES;
             s_h[gt] = state ? a.h[(size_t)b * H + gt] : 0.f;
