@@ -114,6 +114,19 @@ __device__ __forceinline__ bool mbar_try_wait_cluster(const uint64_t* bar, uint3
 }
 constexpr int kHelperRows(int n_help) { return (4 * kHidden + n_help - 1) / n_help; }
 
+// (value, index) as one 64-bit word whose unsigned order is the merge's order: a precedes b (larger value, then
+// smaller index) exactly if key(a) > key(b).  -0 is folded into +0 first, as the comparison of values does.
+__device__ __forceinline__ unsigned long long order_key(float v, int i) {
+    uint32_t u = __float_as_uint(v + 0.f);
+    u = (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+    return ((unsigned long long)u << 32) | (uint32_t)(0x7fffffff - i);
+}
+__device__ __forceinline__ float key_value(unsigned long long key) {
+    const uint32_t u = (uint32_t)(key >> 32);
+    return __uint_as_float((u & 0x80000000u) ? (u ^ 0x80000000u) : ~u);
+}
+__device__ __forceinline__ int key_index(unsigned long long key) { return 0x7fffffff - (int)(uint32_t)key; }
+
 // One block per sequence.  Phase 1 runs two things side by side: warps 0-15 merge the vocabulary pass's
 // chunk records into each row's top-k and log-normaliser, warps 16-31 do everything of the prediction
 // model that does not depend on this call's candidates (W_hh h + biases, weights into shared memory).
@@ -267,23 +280,21 @@ __global__ void __launch_bounds__(kSelThreads, 1) expand_select_gate_kernel(cons
                 // best from below; what is not after it survives, and survivors are ranked by counting.
                 const float* pv = st_v + (size_t)f * per_row;
                 const int* pi = st_i + (size_t)f * per_row;
-                float* lv = sv_v + warp * kSurvCap;
-                int* li = sv_i + warp * kSurvCap;
+                // survivors as order keys, in the space of this warp's value and index lists
+                unsigned long long* lk = reinterpret_cast<unsigned long long*>(sv_v) + warp * kSurvCap;
                 if (lane == 0) { s_tv[warp] = -CUDART_INF_F; s_ti[warp] = 0x7fffffff; }
                 s_rv[warp][lane] = -CUDART_INF_F;
                 s_ri[warp][lane] = 0x7fffffff;
                 __syncwarp();
                 if (n_chunks <= 32) {
-                    // lane c holds the head of chunk c; its rank among the heads by 32 shuffles
+                    // lane c holds the head of chunk c; its rank among the heads by shuffling the heads' order keys
+                    // (one 64-bit comparison per pair: the warp's instruction count is what this phase costs)
                     const float hv = lane < n_chunks ? pv[lane * k] : -CUDART_INF_F;
                     const int hi = lane < n_chunks ? pi[lane * k] : 0x7fffffff;
+                    const unsigned long long hk = order_key(hv, hi);
                     int rank = 0;
 #pragma unroll 4
-                    for (int o = 0; o < n_chunks; ++o) {                 // lanes beyond the chunks hold (-inf, max): they precede nothing
-                        const float ov = __shfl_sync(kFull, hv, o);
-                        const int oi = __shfl_sync(kFull, hi, o);
-                        rank += precedes(ov, oi, hv, hi) ? 1 : 0;
-                    }
+                    for (int o = 0; o < n_chunks; ++o) rank += __shfl_sync(kFull, hk, o) > hk ? 1 : 0;
                     if (lane < n_chunks && rank == k - 1) { s_tv[warp] = hv; s_ti[warp] = hi; }
                 } else {
                     for (int c = lane; c < n_chunks; c += 32) {
@@ -311,17 +322,17 @@ __global__ void __launch_bounds__(kSelThreads, 1) expand_select_gate_kernel(cons
                     }
                     const int off = total + incl - cnt;
                     for (int e = 0; e < cnt; ++e)
-                        if (off + e < kSurvCap) { lv[off + e] = pv[c * k + e]; li[off + e] = pi[c * k + e]; }
+                        if (off + e < kSurvCap) lk[off + e] = order_key(pv[c * k + e], pi[c * k + e]);
                     total += __shfl_sync(kFull, incl, 31);
                 }
                 __syncwarp();
                 if (total <= kSurvCap) {
                     for (int e = lane; e < total; e += 32) {
-                        const float cv = lv[e];
-                        const int ci = li[e];
+                        const unsigned long long ck = lk[e];
                         int rank = 0;
-                        for (int j = 0; j < total; ++j) rank += precedes(lv[j], li[j], cv, ci) ? 1 : 0;
-                        if (rank < k) { s_rv[warp][rank] = cv; s_ri[warp][rank] = ci; }
+#pragma unroll 4
+                        for (int j = 0; j < total; ++j) rank += lk[j] > ck ? 1 : 0;
+                        if (rank < k) { s_rv[warp][rank] = key_value(ck); s_ri[warp][rank] = key_index(ck); }
                     }
                     __syncwarp();
                     top.v = s_rv[warp][lane];
