@@ -249,6 +249,8 @@ __global__ void __launch_bounds__(kSelThreads, 1) expand_select_gate_kernel(cons
     __shared__ int s_ti[kMergeWarps], s_ri[kMergeWarps][32];
 
     if (tid == 0) s_base = a.t > 1 ? a.pool_len[b] : 0;
+    // previous call's state, needed late: requested now so that nothing waits for it (F * k <= the block's threads)
+    const int my_parent = tid < F * k ? a.parent_pool_idx[(size_t)b * F + tid / k] : 0;
     const int forced = a.force_calls != nullptr ? a.force_calls[b] : -1;     // read now, needed at the very end
 
     if (warp < kMergeWarps) {
@@ -272,6 +274,7 @@ __global__ void __launch_bounds__(kSelThreads, 1) expand_select_gate_kernel(cons
             // (always from a valid address, and not looked at before the merge is done: nothing below waits for them)
             const float pm0_raw = P.vp.part_m[row * n_chunks + min(lane, n_chunks - 1)];
             const float ps0_raw = P.vp.part_s[row * n_chunks + min(lane, n_chunks - 1)];
+            const float parent_sc = a.parent_score[(size_t)b * F + f];
             WarpTopList<float> top;
             top.reset();
             bool merged = false;
@@ -372,7 +375,7 @@ __global__ void __launch_bounds__(kSelThreads, 1) expand_select_gate_kernel(cons
             const double lse = (double)M + log(S);
             if (lane < k) {
                 const double logp = (double)top.v - lse;
-                const double sc = (double)a.parent_score[(size_t)b * F + f] + logp;
+                const double sc = (double)parent_sc + logp;
                 a.topk_tok[row * k + lane] = top.i;
                 a.topk_logp[row * k + lane] = (float)logp;
                 s_cand[f * k + lane] = sc;
@@ -426,10 +429,11 @@ __global__ void __launch_bounds__(kSelThreads, 1) expand_select_gate_kernel(cons
 
     // ---- 2. append every candidate to the pool ----
     const size_t pb = (size_t)b * a.pool_capacity + base;
-    for (int e = tid; e < n_cand; e += kSelThreads) {
-        const int f = e / k;
+    static_assert(kMaxF * RADAR_MAX_K <= kSelThreads, "one candidate per thread");
+    if (tid < n_cand) {
+        const int e = tid;
         a.pool_tok[pb + e] = s_ctok[e];
-        a.pool_parent[pb + e] = a.parent_pool_idx[(size_t)b * F + f];
+        a.pool_parent[pb + e] = my_parent;
         a.pool_score[pb + e] = (float)s_cand[e];
         a.pool_depth[pb + e] = a.t;
         a.pool_draft_row[pb + e] = -1;
