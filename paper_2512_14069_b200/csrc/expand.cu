@@ -436,9 +436,7 @@ __global__ void __launch_bounds__(kSelThreads, 1) expand_select_gate_kernel(cons
         a.pool_parent[pb + e] = my_parent;
         a.pool_score[pb + e] = (float)s_cand[e];
         a.pool_depth[pb + e] = a.t;
-        a.pool_draft_row[pb + e] = -1;
-    }
-    __syncthreads();      // draft_row = -1 must land before the survivors overwrite theirs
+    }                     // (its draft row is written below, by the thread that knows whether it survives)
 
     // ---- 3. the k best candidates over all parents (score desc, flat index asc) ----
     // eight threads share a candidate's rank count (n_cand <= 1024: at most 8 rounds)
@@ -452,6 +450,7 @@ __global__ void __launch_bounds__(kSelThreads, 1) expand_select_gate_kernel(cons
         rank += __shfl_xor_sync(kFull, rank, 1);
         rank += __shfl_xor_sync(kFull, rank, 2);
         rank += __shfl_xor_sync(kFull, rank, 4);
+        if (have && part == 0) a.pool_draft_row[pb + e] = rank < k ? 1 + (a.t - 1) * k + rank : -1;
         if (have && part == 0 && rank < k) {
             const float sc = (float)v;
             const size_t o = (size_t)b * k + rank;
@@ -459,7 +458,6 @@ __global__ void __launch_bounds__(kSelThreads, 1) expand_select_gate_kernel(cons
             a.frontier_score[o] = sc;
             a.frontier_pool_idx[o] = base + e;
             a.frontier_src_row[o] = e / k;
-            a.pool_draft_row[pb + e] = 1 + (a.t - 1) * k + rank;
             s_x[rank] = expf(sc);                                // confidence score in [0,1]
         }
     }
