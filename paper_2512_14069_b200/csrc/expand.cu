@@ -536,15 +536,17 @@ __global__ void __launch_bounds__(kSelThreads, 1) expand_select_gate_kernel(cons
             }
         }
         __syncthreads();
-        if (warp < 2) {
-            float acc = 0.f;
-            for (int c = lane; c < H; c += 32) acc = fmaf(s_w2[warp * H + c], s_hid[c], acc);
-            acc = warp_sum(acc);
-            if (lane == 0) s_y[warp] = acc + s_b2[warp];
+        if (warp == 0) {                               // both logits in one warp: nothing else has to wait for them
+            float y0 = 0.f, y1 = 0.f;
+            for (int c = lane; c < H; c += 32) {
+                y0 = fmaf(s_w2[c], s_hid[c], y0);
+                y1 = fmaf(s_w2[H + c], s_hid[c], y1);
+            }
+            y0 = warp_sum(y0) + s_b2[0];
+            y1 = warp_sum(y1) + s_b2[1];
+            cont = y1 > y0;
+            if (lane < 2) a.gate_logits[(size_t)b * 2 + lane] = lane == 0 ? y0 : y1;
         }
-        __syncthreads();
-        cont = s_y[1] > s_y[0];
-        if (tid < 2) a.gate_logits[(size_t)b * 2 + tid] = s_y[tid];
         if (forced >= 0) cont = a.t < forced;
     } else {
         if (tid < 2) a.gate_logits[(size_t)b * 2 + tid] = 0.f;
