@@ -491,6 +491,7 @@ __global__ void __launch_bounds__(kSelThreads, 1) expand_select_gate_kernel(cons
                 acc += P.feat_pre[(size_t)b * 4 * H + tid];
             } else {
                 const float* w = s_wih + tid * k;
+#pragma unroll 4                                       // the loads of four terms at once, the sum in the order of before
                 for (int j = 0; j < k; ++j) acc = fmaf(w[j], s_x[j], acc);
             }
             s_pre[tid] = acc;
